@@ -1,0 +1,168 @@
+/*
+ * kve.h — C ABI of libkve: the RNN-gated chunked KV cache decode path on one B200 (sm_100a).
+ *
+ * The paper's module replaces a transformer layer's KV cache (Sec. 1, Sec. 3.1): history outside a
+ * recent window is cut into chunks of C tokens, each chunk is reduced to one summary key/value
+ * (Eq. 2), an LSTM scores the summaries in temporal order (Eq. 3), chunks with s_t >= tau are kept
+ * (Sec. 3.2), and decode attention (Eq. 1) runs over the kept chunks plus the raw window
+ * (Sec. 3.3, n' = W + M).
+ *
+ * Conventions for every entry point
+ *   - returns KVE_OK (0) or a negative kvE_status; never throws, never aborts.
+ *   - work is enqueued on the given CUDA stream (passed as void*, a cudaStream_t); the call does not
+ *     wait for it.  kvE_poll_status and kvE_create are the only calls that synchronise.
+ *   - no entry point allocates or frees device memory.  Every device buffer is owned by the caller
+ *     (allocate it with any allocator, e.g. PyTorch) and only borrowed; the handle owns host metadata.
+ *   - argument and geometry errors are found on the host before any launch.  Device-side problems
+ *     (a page id out of range, a wait that ran out) set *status_word to a kvE_status and the kernel
+ *     skips the access; nothing traps and no wait is unbounded.
+ *   - one stream at a time per handle; calls on one handle are not thread-safe.
+ *   - "bf16" is the 16-bit brain float bit pattern; matrices are row-major; S = B * Hkv sequences,
+ *     sequence index s = b * Hkv + h.  d (head dim) must be 128.
+ */
+#ifndef KVE_H_
+#define KVE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KVE_OK = 0,
+  KVE_ERR_ARG = -1,       /* null pointer, negative size, unknown enum value */
+  KVE_ERR_GEOMETRY = -2,  /* a size combination the kernels do not support (d != 128, d_g, ...) */
+  KVE_ERR_CAPACITY = -3,  /* append beyond max_tokens, workspace too small, page id out of range */
+  KVE_ERR_STATE = -4,     /* call order: chunk range not yet summarised / gated, ... */
+  KVE_ERR_CUDA = -5,      /* a CUDA runtime call failed (launch error text via kvE_last_cuda_error) */
+  KVE_ERR_TIMEOUT = -6    /* a bounded device-side wait ran out (reported through status_word) */
+} kvE_status;
+
+enum { KVE_AGG_MEAN = 0, KVE_AGG_MLP = 1, KVE_AGG_IDENTITY = 2 };   /* Eq. 2 aggregator */
+enum { KVE_ATTEND_SUMMARY = 0, KVE_ATTEND_RAW = 1 };                /* what a kept chunk contributes */
+
+/* Geometry, fixed at kvE_create. */
+typedef struct {
+  int32_t B;           /* batch */
+  int32_t Hq, Hkv;     /* query heads, KV heads; Hq == Hkv required */
+  int32_t d;           /* head dim, 128 */
+  int32_t C;           /* chunk size in tokens, 1..1024 (Sec. 3.2) */
+  int32_t W;           /* recent window in tokens, >= 0 (Sec. 3.3): never summarised */
+  int32_t max_tokens;  /* capacity of one sequence */
+  int32_t n_layers;    /* independent layers sharing the handle */
+  int32_t agg;         /* KVE_AGG_* ; IDENTITY needs C == 1 */
+  int32_t d_sum;       /* MLP hidden size (KVE_AGG_MLP), multiple of 8, <= 1024 */
+  int32_t d_g;         /* LSTM hidden size: 64, 128 or 256 */
+  int32_t attend;      /* KVE_ATTEND_* */
+} kvE_config;
+
+/* max_chunks = ceil(max_tokens / C) is the chunk stride of every per-chunk array below. */
+
+/* Caller-owned DEVICE buffers. */
+typedef struct {
+  void* k_pages;        /* bf16 [n_pages][C][d]: one page = one chunk of one (layer, b, h) */
+  void* v_pages;        /* bf16 [n_pages][C][d] */
+  int64_t n_pages;
+  int32_t* page_table;  /* [n_layers][S][max_chunks] page ids, filled by the caller */
+  int32_t* seq_len;     /* [n_layers][B] tokens stored; written by kvE_append / kvE_set_len */
+  float* ksum_f32;      /* [n_layers][S][max_chunks][d] chunk summaries, fp32 */
+  float* vsum_f32;
+  void* ksum_bf16;      /* same, rounded to bf16: what the gate and attention read */
+  void* vsum_bf16;
+  float* scores;        /* [n_layers][S][max_chunks] gate scores s_t */
+  int32_t* keep_idx;    /* [n_layers][S][max_chunks] ascending kept chunk ids, rest -1 */
+  int32_t* keep_cnt;    /* [n_layers][S] */
+  float* lstm_h;        /* [n_layers][S][d_g] carried hidden state */
+  float* lstm_c;        /* [n_layers][S][d_g] carried cell state */
+  void* workspace;      /* kvE_workspace_bytes(cfg) bytes, 256-byte aligned, zeroed by kvE_create */
+  size_t workspace_bytes;
+  int32_t* status_word; /* one int32, zeroed by kvE_create; first device-side error sticks */
+} kvE_buffers;
+
+/* Aggregator MLP_K / MLP_V of Eq. 2 (KVE_AGG_MLP): y = W2 gelu(W1 m + b1) + b2, m the chunk mean.
+ * DEVICE pointers; W1 [d_sum][d], W2 [d][d_sum] bf16; b1 [d_sum], b2 [d] fp32. */
+typedef struct {
+  const void *W1K, *W2K, *W1V, *W2V;
+  const float *b1K, *b2K, *b1V, *b2V;
+} kvE_agg_weights;
+
+/* LSTM gate of Eq. 3.  DEVICE pointers; W_ih [4 d_g][2 d], W_hh [4 d_g][d_g] bf16, gate rows in the
+ * order i, f, g, o; b_ih, b_hh [4 d_g], w_s [d_g] fp32; b_s by value. */
+typedef struct {
+  const void *W_ih, *W_hh;
+  const float *b_ih, *b_hh, *w_s;
+  float b_s;
+} kvE_lstm_weights;
+
+typedef struct kvE_store kvE_store;
+
+/* Bytes of workspace the handle needs (gate projection buffer + attention split partials). */
+size_t kvE_workspace_bytes(const kvE_config* cfg);
+
+/* Host-side handle.  Validates the geometry, zeroes workspace, status_word, seq_len and keep_cnt
+ * (synchronous memsets on the current device).  All layers start empty. */
+int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out);
+int kvE_destroy(kvE_store* st);
+
+/* Sec. 3.2 "stores the key-value pairs in temporal order": append n_new tokens to every sequence
+ * of `layer`.  k_new, v_new: DEVICE bf16 [S][n_new][d].  *n_ready (nullable, host) receives how
+ * many completed chunks now lie outside the window and have not been gated yet (the trigger of
+ * Sec. 3.3).  KVE_ERR_CAPACITY if the layer would exceed max_tokens. */
+int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new,
+               int* n_ready, void* stream);
+
+/* Set the stored length of `layer` (all sequences) to n tokens, n <= max_tokens; the pages keep
+ * their contents.  Chunks at or beyond the new stale range lose their summarised / gated /
+ * compacted marks.  Used to load a prefilled cache and to roll a decode step back. */
+int kvE_set_len(kvE_store* st, int layer, int n, void* stream);
+
+/* Eq. 2: summaries of chunks [chunk_begin, chunk_end) of every sequence of `layer`;
+ * chunk_end <= floor((n - W) / C).  w is NULL unless agg == KVE_AGG_MLP. */
+int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_end,
+                         const kvE_agg_weights* w, void* stream);
+
+/* Eq. 3: run the LSTM over summaries [chunk_begin, chunk_end) oldest first and write scores.
+ * chunk_begin == 0 starts from h = c = 0; otherwise chunk_begin must equal the number of chunks
+ * already gated (state carried in lstm_h / lstm_c).  The range must have been summarised. */
+int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
+             const kvE_lstm_weights* w, void* stream);
+
+/* Sec. 3.2 retention rule: keep chunk t iff scores[t] >= tau, over all gated chunks of `layer`;
+ * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw. */
+int kvE_compact(kvE_store* st, int layer, float tau, void* stream);
+
+/* Sec. 3.3 + Eq. 1: out = softmax(q K'^T * scale) V' over [kept chunks ; raw tail] of `layer`.
+ * q, out: DEVICE bf16 [S][d]; lse: DEVICE fp32 [S] or NULL (log-sum-exp of the scaled logits). */
+int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale,
+                    void* stream);
+
+/* Eq. 1 over all n stored tokens of `layer` (the full-cache baseline of Sec. 3.3). */
+int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse,
+                          float scale, void* stream);
+
+/* One whole decode step of `layer` from HOST memory: copies k_new, v_new, q (bf16 [S][d] each,
+ * ideally pinned) to the device, appends the token, brings summaries, gate and keep list up to
+ * date for every chunk that has left the window (from scratch if `from_scratch` != 0), runs
+ * kvE_decode_attn and copies out (bf16 [S][d]) back to host memory.  Staging uses the tail of the
+ * workspace.  Waits for the stream before returning. */
+int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host,
+                         const void* q_host, void* out_host, const kvE_agg_weights* aw,
+                         const kvE_lstm_weights* lw, float tau, float scale, int from_scratch,
+                         void* stream);
+
+/* Reads *status_word (synchronises the device) into *device_status and clears it. */
+int kvE_poll_status(kvE_store* st, int* device_status);
+
+/* Host-side view of a layer: tokens stored, chunks summarised, gated and covered by the keep list. */
+int kvE_layer_state(const kvE_store* st, int layer, int* n_tokens, int* n_summarised, int* n_gated,
+                    int* n_compacted);
+
+/* Text of the last CUDA runtime error seen by this handle's calls ("" if none). */
+const char* kvE_last_cuda_error(const kvE_store* st);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVE_H_ */

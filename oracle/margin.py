@@ -34,11 +34,13 @@ def centred_b_s(o: kvo.Oracle, wl: wlm.Workload, K, V, mlp, lstm, keep=0.5, n_ch
 
 
 def repair_margin(o: kvo.Oracle, wl: wlm.Workload, layer, K, V, mlp, lstm, tau=None, margin=1e-3,
-                  n_chunks=None, max_attempts=50):
+                  n_chunks=None, max_attempts=50, seq_ids=None):
     """Adjusts K, V in place.  Returns (summaries dict, scores [S, stride], h, c, redraws) as the
-    oracle `o` computes them on the repaired inputs; redraws = [(s, t, attempt), ...]."""
+    oracle `o` computes them on the repaired inputs; redraws = [(s, t, attempt), ...].
+    K, V may hold a subset of the workload's sequences: seq_ids[i] is the sequence id of row i."""
     tau = wl.tau if tau is None else tau
     S, n, d = K.shape
+    seq_ids = list(range(S)) if seq_ids is None else [int(x) for x in seq_ids]
     Nc = wl.n_stale_chunks(n) if n_chunks is None else n_chunks
     stride = max(wl.max_chunks, 1)
     agg = AGG_CODE[wl.agg]
@@ -61,7 +63,7 @@ def repair_margin(o: kvo.Oracle, wl: wlm.Workload, layer, K, V, mlp, lstm, tau=N
                 attempt[s] += 1
                 if attempt[s] > max_attempts:
                     raise RuntimeError("margin repair did not converge")
-                k, v = wlm.gen_chunk(wl, layer, s, t, attempt[s])
+                k, v = wlm.gen_chunk(wl, layer, seq_ids[s], t, attempt[s])
                 K[s, t * wl.C:(t + 1) * wl.C] = k
                 V[s, t * wl.C:(t + 1) * wl.C] = v
             # re-summarise and re-gate just the redrawn (sequence, chunk) pairs from the saved state
@@ -75,5 +77,5 @@ def repair_margin(o: kvo.Oracle, wl: wlm.Workload, layer, K, V, mlp, lstm, tau=N
             h[bad], c[bad], scores[bad, t] = hb, cb, sb[:, 0]
             still = np.abs(sb[:, 0].astype(np.float64) - tau) < margin
             bad = bad[still]
-        redraws.extend((s, t, a) for s, a in attempt.items())
+        redraws.extend((seq_ids[s], t, a) for s, a in attempt.items())
     return sm, scores, h, c, redraws

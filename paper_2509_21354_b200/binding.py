@@ -1,0 +1,325 @@
+"""Thin ctypes binding over libkve.so (C ABI in include/kve.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.  PyTorch is
+used for device memory and streams.  There is no CPU fallback: if the library is missing or no
+CUDA device is present, calls raise.
+
+The module-level functions carry the C entry points' names (kvE_append, kvE_summarize_chunks,
+kvE_gate, kvE_compact, kvE_decode_attn, ...) and take the same arguments with torch tensors in place
+of device pointers; `Store` bundles the caller-owned buffers a handle needs.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+AGG = {"mean": 0, "mlp": 1, "identity": 2}
+ATTEND = {"summary": 0, "raw": 1}
+STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_CAPACITY",
+          -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
+
+EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
+           "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_decode_attn", "kvE_decode_attn_dense",
+           "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error"]
+
+
+class KveError(RuntimeError):
+    def __init__(self, fn, rc, detail=""):
+        self.rc = rc
+        super().__init__(f"{fn} -> {STATUS.get(rc, rc)} {detail}".strip())
+
+
+class kvE_config(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("B", "Hq", "Hkv", "d", "C", "W", "max_tokens", "n_layers", "agg",
+                                         "d_sum", "d_g", "attend")]
+
+
+class kvE_buffers(C.Structure):
+    _fields_ = [("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("n_pages", C.c_int64),
+                ("page_table", C.c_void_p), ("seq_len", C.c_void_p),
+                ("ksum_f32", C.c_void_p), ("vsum_f32", C.c_void_p), ("ksum_bf16", C.c_void_p), ("vsum_bf16", C.c_void_p),
+                ("scores", C.c_void_p), ("keep_idx", C.c_void_p), ("keep_cnt", C.c_void_p),
+                ("lstm_h", C.c_void_p), ("lstm_c", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("status_word", C.c_void_p)]
+
+
+class kvE_agg_weights(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("W1K", "W2K", "W1V", "W2V", "b1K", "b2K", "b1V", "b2V")]
+
+
+class kvE_lstm_weights(C.Structure):
+    _fields_ = [("W_ih", C.c_void_p), ("W_hh", C.c_void_p), ("b_ih", C.c_void_p), ("b_hh", C.c_void_p),
+                ("w_s", C.c_void_p), ("b_s", C.c_float)]
+
+
+_lib = None
+
+
+def load_library(build_if_missing: bool = True) -> C.CDLL:
+    """dlopen libkve.so (building it first if its sources are newer).  Raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if build_if_missing:
+        path = _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run `python -m paper_2509_21354_b200.build`")
+    lib = C.CDLL(path)
+    lib.kvE_workspace_bytes.restype = C.c_size_t
+    lib.kvE_workspace_bytes.argtypes = [C.POINTER(kvE_config)]
+    lib.kvE_create.argtypes = [C.POINTER(kvE_config), C.POINTER(kvE_buffers), C.POINTER(C.c_void_p)]
+    lib.kvE_destroy.argtypes = [C.c_void_p]
+    lib.kvE_append.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p]
+    lib.kvE_set_len.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+    lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
+    lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
+    lib.kvE_compact.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_void_p]
+    lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
+    lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
+    lib.kvE_decode_step_host.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float,
+                                         C.c_float, C.c_int, C.c_void_p]
+    lib.kvE_poll_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
+    lib.kvE_layer_state.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_int)] * 4
+    lib.kvE_last_cuda_error.restype = C.c_char_p
+    lib.kvE_last_cuda_error.argtypes = [C.c_void_p]
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if name not in ("kvE_workspace_bytes", "kvE_last_cuda_error"):
+            fn.restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _stream(stream=None) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _p(t) -> C.c_void_p:
+    if t is None:
+        return C.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous()
+    return C.c_void_p(t.data_ptr())
+
+
+def _check(fn, rc, handle=None):
+    if rc != 0:
+        detail = ""
+        if rc == -5 and handle is not None:
+            detail = load_library().kvE_last_cuda_error(handle).decode()
+        raise KveError(fn, rc, detail)
+
+
+def bits_to_bf16(a: np.ndarray, device="cuda") -> torch.Tensor:
+    """numpy uint16 bf16 bit patterns -> torch.bfloat16 tensor on `device`."""
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def bf16_to_bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class AggWeights:
+    """Device copies of the aggregator MLP weights (bf16 matrices, fp32 biases)."""
+
+    def __init__(self, w: dict, device="cuda"):
+        self.t = {}
+        for k in ("W1K", "W2K", "W1V", "W2V"):
+            self.t[k] = torch.from_numpy(np.ascontiguousarray(w[k], np.float32)).to(device).to(torch.bfloat16).contiguous()
+        for k in ("b1K", "b2K", "b1V", "b2V"):
+            self.t[k] = torch.from_numpy(np.ascontiguousarray(w[k], np.float32)).to(device).contiguous()
+        self.c = kvE_agg_weights(**{k: self.t[k].data_ptr() for k in self.t})
+
+
+class LstmWeights:
+    """Device copies of the gate weights (bf16 W_ih, W_hh; fp32 biases and score head)."""
+
+    def __init__(self, w: dict, device="cuda"):
+        self.t = {}
+        for k in ("W_ih", "W_hh"):
+            self.t[k] = torch.from_numpy(np.ascontiguousarray(w[k], np.float32)).to(device).to(torch.bfloat16).contiguous()
+        for k in ("b_ih", "b_hh", "w_s"):
+            self.t[k] = torch.from_numpy(np.ascontiguousarray(w[k], np.float32)).to(device).contiguous()
+        self.c = kvE_lstm_weights(**{k: self.t[k].data_ptr() for k in self.t}, b_s=float(w["b_s"]))
+
+    def set_b_s(self, b_s: float):
+        self.c.b_s = float(b_s)
+
+
+class Store:
+    """A kvE_store handle plus the device buffers it borrows (allocated here with torch).
+
+    page_perm: None -> page id = flat (layer, s, chunk) index; "random" -> a seeded permutation of the
+    page ids (exercises the page-table indirection); or an explicit int32 array [n_layers, S, max_chunks].
+    """
+
+    def __init__(self, B, H, C_, W, max_tokens, d_g, agg="mean", d_sum=0, attend="summary", n_layers=1,
+                 page_perm=None, device="cuda", seed=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libkve needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.device = torch.device(device)
+        self.cfg = kvE_config(B=B, Hq=H, Hkv=H, d=128, C=C_, W=W, max_tokens=max_tokens, n_layers=n_layers,
+                              agg=AGG[agg], d_sum=d_sum, d_g=d_g, attend=ATTEND[attend])
+        self.B, self.H, self.S, self.C, self.W, self.d_g = B, H, B * H, C_, W, d_g
+        self.n_layers, self.max_tokens = n_layers, max_tokens
+        self.max_chunks = -(-max_tokens // C_)
+        S, mc, L, dev = self.S, self.max_chunks, n_layers, self.device
+        n_pages = L * S * mc
+        ws_bytes = int(self.lib.kvE_workspace_bytes(C.byref(self.cfg)))
+        if ws_bytes == 0:
+            raise KveError("kvE_workspace_bytes", -2, "unsupported geometry")
+        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
+        self.k_pages = z((n_pages, C_, 128), torch.bfloat16)
+        self.v_pages = z((n_pages, C_, 128), torch.bfloat16)
+        if page_perm is None:
+            pt = np.arange(n_pages, dtype=np.int32)
+        elif isinstance(page_perm, str) and page_perm == "random":
+            pt = np.random.default_rng(seed).permutation(n_pages).astype(np.int32)
+        else:
+            pt = np.asarray(page_perm, np.int32)
+        self.page_table = torch.from_numpy(pt.reshape(L, S, mc).copy()).to(dev)
+        self.seq_len = z((L, B), torch.int32)
+        self.ksum_f32 = z((L, S, mc, 128), torch.float32)
+        self.vsum_f32 = z((L, S, mc, 128), torch.float32)
+        self.ksum_bf16 = z((L, S, mc, 128), torch.bfloat16)
+        self.vsum_bf16 = z((L, S, mc, 128), torch.bfloat16)
+        self.scores = z((L, S, mc), torch.float32)
+        self.keep_idx = torch.full((L, S, mc), -1, dtype=torch.int32, device=dev)
+        self.keep_cnt = z((L, S), torch.int32)
+        self.lstm_h = z((L, S, d_g), torch.float32)
+        self.lstm_c = z((L, S, d_g), torch.float32)
+        self.workspace = z((ws_bytes + 256,), torch.uint8)
+        ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.status_word = z((1,), torch.int32)
+        self.buf = kvE_buffers(
+            k_pages=self.k_pages.data_ptr(), v_pages=self.v_pages.data_ptr(), n_pages=n_pages,
+            page_table=self.page_table.data_ptr(), seq_len=self.seq_len.data_ptr(),
+            ksum_f32=self.ksum_f32.data_ptr(), vsum_f32=self.vsum_f32.data_ptr(),
+            ksum_bf16=self.ksum_bf16.data_ptr(), vsum_bf16=self.vsum_bf16.data_ptr(),
+            scores=self.scores.data_ptr(), keep_idx=self.keep_idx.data_ptr(), keep_cnt=self.keep_cnt.data_ptr(),
+            lstm_h=self.lstm_h.data_ptr(), lstm_c=self.lstm_c.data_ptr(),
+            workspace=ws_ptr, workspace_bytes=ws_bytes, status_word=self.status_word.data_ptr())
+        torch.cuda.synchronize()
+        self.handle = C.c_void_p()
+        _check("kvE_create", self.lib.kvE_create(C.byref(self.cfg), C.byref(self.buf), C.byref(self.handle)))
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.kvE_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the C entry points, same names without the prefix ----
+    def append(self, layer, k_new, v_new, stream=None) -> int:
+        return kvE_append(self, layer, k_new, v_new, stream)
+
+    def set_len(self, layer, n, stream=None):
+        kvE_set_len(self, layer, n, stream)
+
+    def summarize_chunks(self, layer, chunk_begin, chunk_end, agg_weights=None, stream=None):
+        kvE_summarize_chunks(self, layer, chunk_begin, chunk_end, agg_weights, stream)
+
+    def gate(self, layer, chunk_begin, chunk_end, lstm_weights, stream=None):
+        kvE_gate(self, layer, chunk_begin, chunk_end, lstm_weights, stream)
+
+    def compact(self, layer, tau, stream=None):
+        kvE_compact(self, layer, tau, stream)
+
+    def decode_attn(self, layer, q, out=None, lse=None, scale=None, stream=None):
+        return kvE_decode_attn(self, layer, q, out, lse, scale, stream)
+
+    def decode_attn_dense(self, layer, q, out=None, lse=None, scale=None, stream=None):
+        return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)
+
+    def decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale=None,
+                         from_scratch=False, stream=None):
+        kvE_decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale, from_scratch, stream)
+
+    def poll_status(self) -> int:
+        return kvE_poll_status(self)
+
+    def layer_state(self, layer=0) -> dict:
+        return kvE_layer_state(self, layer)
+
+
+def kvE_append(st: Store, layer, k_new, v_new, stream=None) -> int:
+    """k_new, v_new: bf16 [S, n_new, 128] device tensors.  Returns the number of chunks ready to gate."""
+    assert k_new.dtype == torch.bfloat16 and k_new.shape == v_new.shape and k_new.shape[0] == st.S and k_new.shape[2] == 128
+    ready = C.c_int(0)
+    _check("kvE_append", st.lib.kvE_append(st.handle, layer, _p(k_new), _p(v_new), int(k_new.shape[1]),
+                                           C.byref(ready), _stream(stream)), st.handle)
+    return ready.value
+
+
+def kvE_set_len(st: Store, layer, n, stream=None):
+    _check("kvE_set_len", st.lib.kvE_set_len(st.handle, layer, int(n), _stream(stream)), st.handle)
+
+
+def kvE_summarize_chunks(st: Store, layer, chunk_begin, chunk_end, agg_weights=None, stream=None):
+    w = C.byref(agg_weights.c) if agg_weights is not None else None
+    _check("kvE_summarize_chunks", st.lib.kvE_summarize_chunks(st.handle, layer, int(chunk_begin), int(chunk_end), w,
+                                                               _stream(stream)), st.handle)
+
+
+def kvE_gate(st: Store, layer, chunk_begin, chunk_end, lstm_weights, stream=None):
+    _check("kvE_gate", st.lib.kvE_gate(st.handle, layer, int(chunk_begin), int(chunk_end), C.byref(lstm_weights.c),
+                                       _stream(stream)), st.handle)
+
+
+def kvE_compact(st: Store, layer, tau, stream=None):
+    _check("kvE_compact", st.lib.kvE_compact(st.handle, layer, C.c_float(tau), _stream(stream)), st.handle)
+
+
+def _attn(fn_name, st, layer, q, out, lse, scale, stream):
+    assert q.dtype == torch.bfloat16 and tuple(q.shape) == (st.S, 128)
+    if out is None:
+        out = torch.empty_like(q)
+    scale = 1.0 / np.sqrt(128.0) if scale is None else scale
+    _check(fn_name, getattr(st.lib, fn_name)(st.handle, layer, _p(q), _p(out), _p(lse), C.c_float(scale),
+                                              _stream(stream)), st.handle)
+    return out
+
+
+def kvE_decode_attn(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):
+    return _attn("kvE_decode_attn", st, layer, q, out, lse, scale, stream)
+
+
+def kvE_decode_attn_dense(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):
+    return _attn("kvE_decode_attn_dense", st, layer, q, out, lse, scale, stream)
+
+
+def kvE_decode_step_host(st: Store, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale=None,
+                         from_scratch=False, stream=None):
+    """k_new, v_new, q, out: HOST bf16 [S, 128] tensors (pinned for asynchronous copies)."""
+    for t in (k_new, v_new, q, out):
+        assert not t.is_cuda and t.dtype == torch.bfloat16 and tuple(t.shape) == (st.S, 128) and t.is_contiguous()
+    scale = 1.0 / np.sqrt(128.0) if scale is None else scale
+    aw = C.byref(agg_weights.c) if agg_weights is not None else None
+    _check("kvE_decode_step_host",
+           st.lib.kvE_decode_step_host(st.handle, layer, C.c_void_p(k_new.data_ptr()), C.c_void_p(v_new.data_ptr()),
+                                       C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), aw,
+                                       C.byref(lstm_weights.c), C.c_float(tau), C.c_float(scale),
+                                       1 if from_scratch else 0, _stream(stream)), st.handle)
+
+
+def kvE_poll_status(st: Store) -> int:
+    word = C.c_int(0)
+    _check("kvE_poll_status", st.lib.kvE_poll_status(st.handle, C.byref(word)), st.handle)
+    return word.value
+
+
+def kvE_layer_state(st: Store, layer=0) -> dict:
+    v = [C.c_int(0) for _ in range(4)]
+    _check("kvE_layer_state", st.lib.kvE_layer_state(st.handle, layer, *[C.byref(x) for x in v]))
+    return dict(zip(("n_tokens", "n_summarised", "n_gated", "n_compacted"), (x.value for x in v)))

@@ -1,0 +1,339 @@
+// Host side of libkve: the C ABI of include/kve.h.  Validates arguments, tracks per-layer progress
+// (tokens stored, chunks summarised / gated / compacted) and enqueues the kernels.  Allocates no
+// device memory.
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/kve.h"
+#include "kernels.h"
+
+using namespace kve;
+
+struct LayerState {
+  int n_tokens = 0;      // tokens stored (every sequence of the layer)
+  int n_summarised = 0;  // chunks [0, n_summarised) have summaries
+  int n_gated = 0;       // chunks [0, n_gated) have scores; LSTM state stands after chunk n_gated-1
+  int n_compacted = 0;   // keep list covers chunks [0, n_compacted); attention reads raw rows from there on
+};
+
+struct kvE_store {
+  kvE_config cfg;
+  kvE_buffers buf;
+  int S, max_chunks;
+  // workspace carve-up (byte offsets)
+  size_t off_P, off_partials, off_counters, off_stage, ws_needed;
+  int max_splits;
+  std::vector<LayerState> layers;
+  std::string cuda_error;
+};
+
+namespace {
+
+constexpr int MAX_SPLITS = 32;
+constexpr size_t ALIGN = 256;
+size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+int check_config(const kvE_config* c) {
+  if (!c) return KVE_ERR_ARG;
+  if (c->B <= 0 || c->Hq <= 0 || c->Hkv <= 0 || c->C <= 0 || c->W < 0 || c->max_tokens <= 0 || c->n_layers <= 0)
+    return KVE_ERR_ARG;
+  if (c->agg != KVE_AGG_MEAN && c->agg != KVE_AGG_MLP && c->agg != KVE_AGG_IDENTITY) return KVE_ERR_ARG;
+  if (c->attend != KVE_ATTEND_SUMMARY && c->attend != KVE_ATTEND_RAW) return KVE_ERR_ARG;
+  if (c->d != 128 || c->Hq != c->Hkv || c->C > 1024) return KVE_ERR_GEOMETRY;
+  if (c->agg == KVE_AGG_IDENTITY && c->C != 1) return KVE_ERR_GEOMETRY;
+  if (c->agg == KVE_AGG_MLP && (c->d_sum <= 0 || c->d_sum % 8 != 0 || c->d_sum > 1024)) return KVE_ERR_GEOMETRY;
+  if (c->d_g != 64 && c->d_g != 128 && c->d_g != 256) return KVE_ERR_GEOMETRY;
+  if ((long long)c->B * c->Hkv > 65535) return KVE_ERR_GEOMETRY;
+  return KVE_OK;
+}
+
+struct Carve {
+  size_t off_P, off_partials, off_counters, off_stage, total;
+};
+Carve carve(const kvE_config& c) {
+  const size_t S = (size_t)c.B * c.Hkv;
+  const size_t max_chunks = ((size_t)c.max_tokens + c.C - 1) / c.C;
+  Carve k;
+  size_t o = 0;
+  k.off_P = o;        o = align_up(o + S * max_chunks * 4 * (size_t)c.d_g * sizeof(float));
+  k.off_partials = o; o = align_up(o + S * MAX_SPLITS * ATTN_PARTIAL_FLOATS * sizeof(float));
+  k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
+  k.off_stage = o;    o = align_up(o + 4 * S * 128 * 2);   // k_new, v_new, q, out of kvE_decode_step_host
+  k.total = o;
+  return k;
+}
+
+int cuda_fail(kvE_store* st, cudaError_t e) {
+  st->cuda_error = cudaGetErrorString(e);
+  return KVE_ERR_CUDA;
+}
+
+LayerView view(const kvE_store* st, int layer) {
+  const kvE_config& c = st->cfg;
+  const kvE_buffers& b = st->buf;
+  const size_t S = st->S, mc = st->max_chunks, L = (size_t)layer;
+  LayerView v;
+  v.k_pages = static_cast<uint16_t*>(b.k_pages);
+  v.v_pages = static_cast<uint16_t*>(b.v_pages);
+  v.n_pages = b.n_pages;
+  v.page_table = b.page_table + L * S * mc;
+  v.seq_len = b.seq_len + L * c.B;
+  v.ksum_f32 = b.ksum_f32 + L * S * mc * 128;
+  v.vsum_f32 = b.vsum_f32 + L * S * mc * 128;
+  v.ksum_bf16 = static_cast<uint16_t*>(b.ksum_bf16) + L * S * mc * 128;
+  v.vsum_bf16 = static_cast<uint16_t*>(b.vsum_bf16) + L * S * mc * 128;
+  v.scores = b.scores + L * S * mc;
+  v.keep_idx = b.keep_idx + L * S * mc;
+  v.keep_cnt = b.keep_cnt + L * S;
+  v.lstm_h = b.lstm_h + L * S * c.d_g;
+  v.lstm_c = b.lstm_c + L * S * c.d_g;
+  v.status = b.status_word;
+  v.B = c.B; v.H = c.Hkv; v.S = st->S; v.C = c.C; v.max_chunks = st->max_chunks; v.max_tokens = c.max_tokens;
+  return v;
+}
+
+int stale_chunks(const kvE_config& c, int n) { return n > c.W ? (n - c.W) / c.C : 0; }
+
+bool bad_layer(const kvE_store* st, int layer) { return !st || layer < 0 || layer >= st->cfg.n_layers; }
+
+// rows per split and grid width for `n_rows_upper` logical rows per sequence
+AttnPlan plan_attention(const kvE_store* st, long long n_rows_upper) {
+  const long long target_ctas = 148LL * 2 * 2;     // about two waves at two CTAs per SM
+  long long splits = (target_ctas + st->S - 1) / st->S;
+  const long long max_useful = (n_rows_upper + 2 * ATTN_TILE_ROWS - 1) / (2 * ATTN_TILE_ROWS);   // >= 128 rows per split
+  if (splits > max_useful) splits = max_useful;
+  if (splits > MAX_SPLITS) splits = MAX_SPLITS;
+  if (splits < 1) splits = 1;
+  long long rows = (n_rows_upper + splits - 1) / splits;
+  rows = (rows + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS * ATTN_TILE_ROWS;
+  if (rows < ATTN_TILE_ROWS) rows = ATTN_TILE_ROWS;
+  AttnPlan p;
+  p.rows_per_split = (int)rows;
+  p.max_splits = (int)((n_rows_upper + rows - 1) / rows);
+  if (p.max_splits < 1) p.max_splits = 1;
+  return p;
+}
+
+int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* out, float* lse, float scale,
+                  cudaStream_t stream) {
+  const LayerState& ls = st->layers[layer];
+  long long rows_upper;
+  if (mode == ATTN_DENSE) rows_upper = ls.n_tokens;
+  else {
+    const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;
+    rows_upper = (long long)ls.n_compacted * per + (ls.n_tokens - (long long)ls.n_compacted * st->cfg.C);
+  }
+  AttnPlan plan = plan_attention(st, rows_upper);
+  char* ws = static_cast<char*>(st->buf.workspace);
+  cudaError_t e = launch_attn(view(st, layer), mode, ls.n_compacted, ls.n_tokens, plan, q, out, lse, scale,
+                              reinterpret_cast<float*>(ws + st->off_partials),
+                              reinterpret_cast<int32_t*>(ws + st->off_counters), stream);
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t kvE_workspace_bytes(const kvE_config* cfg) {
+  if (check_config(cfg) != KVE_OK) return 0;
+  return carve(*cfg).total;
+}
+
+int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
+  if (!out) return KVE_ERR_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc != KVE_OK) return rc;
+  if (!buf || !buf->k_pages || !buf->v_pages || !buf->page_table || !buf->seq_len || !buf->ksum_f32 ||
+      !buf->vsum_f32 || !buf->ksum_bf16 || !buf->vsum_bf16 || !buf->scores || !buf->keep_idx || !buf->keep_cnt ||
+      !buf->lstm_h || !buf->lstm_c || !buf->workspace || !buf->status_word || buf->n_pages <= 0)
+    return KVE_ERR_ARG;
+  const Carve k = carve(*cfg);
+  if (buf->workspace_bytes < k.total) return KVE_ERR_CAPACITY;
+  if (reinterpret_cast<uintptr_t>(buf->workspace) % ALIGN != 0) return KVE_ERR_ARG;
+  kvE_store* st = new (std::nothrow) kvE_store();
+  if (!st) return KVE_ERR_ARG;
+  st->cfg = *cfg;
+  st->buf = *buf;
+  st->S = cfg->B * cfg->Hkv;
+  st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
+  st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
+  st->off_stage = k.off_stage; st->ws_needed = k.total;
+  st->max_splits = MAX_SPLITS;
+  st->layers.assign(cfg->n_layers, LayerState());
+  cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.total - k.off_partials);
+  if (e == cudaSuccess) e = cudaMemset(buf->status_word, 0, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(buf->seq_len, 0, sizeof(int32_t) * (size_t)cfg->n_layers * cfg->B);
+  if (e == cudaSuccess) e = cudaMemset(buf->keep_cnt, 0, sizeof(int32_t) * (size_t)cfg->n_layers * st->S);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    delete st;
+    return KVE_ERR_CUDA;
+  }
+  *out = st;
+  return KVE_OK;
+}
+
+int kvE_destroy(kvE_store* st) {
+  delete st;
+  return KVE_OK;
+}
+
+int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new, int* n_ready, void* stream) {
+  if (bad_layer(st, layer) || !k_new || !v_new || n_new < 0) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
+  if (n_new > 0) {
+    cudaError_t e = launch_append(view(st, layer), k_new, v_new, n_new, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(st, e);
+    ls.n_tokens += n_new;
+  }
+  if (n_ready) *n_ready = stale_chunks(st->cfg, ls.n_tokens) - ls.n_gated;
+  return KVE_OK;
+}
+
+int kvE_set_len(kvE_store* st, int layer, int n, void* stream) {
+  if (bad_layer(st, layer) || n < 0) return KVE_ERR_ARG;
+  if (n > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
+  cudaError_t e = launch_set_len(view(st, layer), n, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  LayerState& ls = st->layers[layer];
+  ls.n_tokens = n;
+  const int nc = stale_chunks(st->cfg, n);
+  if (ls.n_summarised > nc) ls.n_summarised = nc;
+  if (ls.n_gated > nc) ls.n_gated = 0;          // the carried LSTM state is past the cut: gate again from chunk 0
+  if (ls.n_compacted > nc) ls.n_compacted = nc;
+  return KVE_OK;
+}
+
+int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE_agg_weights* w,
+                         void* stream) {
+  if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  if (chunk_end > stale_chunks(st->cfg, ls.n_tokens)) return KVE_ERR_STATE;   // the window is never summarised
+  const bool mlp = st->cfg.agg == KVE_AGG_MLP;
+  if (mlp && (!w || !w->W1K || !w->W2K || !w->W1V || !w->W2V || !w->b1K || !w->b2K || !w->b1V || !w->b2V))
+    return KVE_ERR_ARG;
+  if (chunk_end == chunk_begin) return KVE_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const LayerView v = view(st, layer);
+  cudaError_t e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, s);
+  if (e == cudaSuccess && mlp) {
+    MlpWeights mw;
+    mw.W1K = static_cast<const uint16_t*>(w->W1K); mw.W2K = static_cast<const uint16_t*>(w->W2K);
+    mw.W1V = static_cast<const uint16_t*>(w->W1V); mw.W2V = static_cast<const uint16_t*>(w->W2V);
+    mw.b1K = w->b1K; mw.b2K = w->b2K; mw.b1V = w->b1V; mw.b2V = w->b2V;
+    e = launch_chunk_mlp(v, chunk_begin, chunk_end, mw, st->cfg.d_sum, s);
+  }
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  if (chunk_begin <= ls.n_summarised && chunk_end > ls.n_summarised) ls.n_summarised = chunk_end;
+  return KVE_OK;
+}
+
+int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE_lstm_weights* w, void* stream) {
+  if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin) return KVE_ERR_ARG;
+  if (!w || !w->W_ih || !w->W_hh || !w->b_ih || !w->b_hh || !w->w_s) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  if (chunk_end > ls.n_summarised) return KVE_ERR_STATE;
+  if (chunk_begin != 0 && chunk_begin != ls.n_gated) return KVE_ERR_STATE;
+  if (chunk_end == chunk_begin) {
+    if (chunk_begin == 0) ls.n_gated = 0;
+    return KVE_OK;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const LayerView v = view(st, layer);
+  float* P = reinterpret_cast<float*>(static_cast<char*>(st->buf.workspace) + st->off_P);
+  cudaError_t e = launch_gate_proj(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_ih), w->b_ih, w->b_hh,
+                                   st->cfg.d_g, P, s);
+  if (e == cudaSuccess)
+    e = launch_gate_rnn(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_hh), w->w_s, w->b_s, st->cfg.d_g,
+                        P, chunk_begin == 0, s);
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  ls.n_gated = chunk_end;
+  if (ls.n_compacted > chunk_begin) ls.n_compacted = chunk_begin;   // scores changed under the keep list
+  return KVE_OK;
+}
+
+int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  cudaError_t e = launch_compact(view(st, layer), ls.n_gated, tau, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  ls.n_compacted = ls.n_gated;
+  return KVE_OK;
+}
+
+int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {
+  if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
+  return run_attention(st, layer, mode, q, out, lse, scale, static_cast<cudaStream_t>(stream));
+}
+
+int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {
+  if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  return run_attention(st, layer, ATTN_DENSE, q, out, lse, scale, static_cast<cudaStream_t>(stream));
+}
+
+int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host, const void* q_host,
+                         void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
+                         int from_scratch, void* stream) {
+  if (bad_layer(st, layer) || !k_new_host || !v_new_host || !q_host || !out_host || !lw) return KVE_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t row_bytes = (size_t)st->S * 128 * 2;
+  char* stage = static_cast<char*>(st->buf.workspace) + st->off_stage;
+  char *dk = stage, *dv = stage + row_bytes, *dq = stage + 2 * row_bytes, *dout = stage + 3 * row_bytes;
+  cudaError_t e = cudaMemcpyAsync(dk, k_new_host, row_bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_new_host, row_bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, row_bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  int rc = kvE_append(st, layer, dk, dv, 1, nullptr, stream);
+  if (rc != KVE_OK) return rc;
+  LayerState& ls = st->layers[layer];
+  const int nc = stale_chunks(st->cfg, ls.n_tokens);
+  const int s0 = from_scratch ? 0 : ls.n_summarised;
+  if (nc > s0) {
+    rc = kvE_summarize_chunks(st, layer, s0, nc, aw, stream);
+    if (rc != KVE_OK) return rc;
+  }
+  const int g0 = from_scratch ? 0 : ls.n_gated;
+  if (nc > g0 || from_scratch) {
+    rc = kvE_gate(st, layer, g0, nc, lw, stream);
+    if (rc != KVE_OK) return rc;
+  }
+  if (ls.n_compacted != ls.n_gated || from_scratch) {
+    rc = kvE_compact(st, layer, tau, stream);
+    if (rc != KVE_OK) return rc;
+  }
+  rc = kvE_decode_attn(st, layer, dq, dout, nullptr, scale, stream);
+  if (rc != KVE_OK) return rc;
+  e = cudaMemcpyAsync(out_host, dout, row_bytes, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+}
+
+int kvE_poll_status(kvE_store* st, int* device_status) {
+  if (!st || !device_status) return KVE_ERR_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  int32_t word = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&word, st->buf.status_word, sizeof(word), cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && word != 0) e = cudaMemset(st->buf.status_word, 0, sizeof(word));
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  *device_status = word;
+  return KVE_OK;
+}
+
+int kvE_layer_state(const kvE_store* st, int layer, int* n_tokens, int* n_summarised, int* n_gated, int* n_compacted) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  const LayerState& ls = st->layers[layer];
+  if (n_tokens) *n_tokens = ls.n_tokens;
+  if (n_summarised) *n_summarised = ls.n_summarised;
+  if (n_gated) *n_gated = ls.n_gated;
+  if (n_compacted) *n_compacted = ls.n_compacted;
+  return KVE_OK;
+}
+
+const char* kvE_last_cuda_error(const kvE_store* st) { return st ? st->cuda_error.c_str() : ""; }
+
+}  // extern "C"

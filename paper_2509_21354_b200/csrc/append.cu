@@ -1,0 +1,58 @@
+// kvE_append / kvE_set_len kernels: place new (k, v) rows at the tail of every sequence's paged
+// cache, in temporal order (Sec. 3.2), and keep the device-side length in step.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace kve {
+
+// One thread moves 16 bytes.  idx -> (row of k_new/v_new, K-or-V, 16-byte lane within the 256-byte row).
+__global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint4* __restrict__ k_new,
+                                                         const uint4* __restrict__ v_new, int n_new) {
+  const long long total = (long long)v.S * n_new * 32;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int lane16 = (int)(idx & 15);
+    const int is_v = (int)((idx >> 4) & 1);
+    const long long row = idx >> 5;              // s * n_new + i
+    const int s = (int)(row / n_new);
+    const int i = (int)(row - (long long)s * n_new);
+    const int b = s / v.H;
+    const int pos = v.seq_len[b] + i;
+    if (pos < 0 || pos >= v.max_tokens) { set_status(v.status, ERR_CAPACITY); continue; }
+    const int chunk = pos / v.C;
+    const int r = pos - chunk * v.C;
+    const long long page = v.page_table[(long long)s * v.max_chunks + chunk];
+    if (page < 0 || page >= v.n_pages) { set_status(v.status, ERR_CAPACITY); continue; }
+    uint4* dst = reinterpret_cast<uint4*>((is_v ? v.v_pages : v.k_pages) + (page * v.C + r) * D) + lane16;
+    const uint4* src = (is_v ? v_new : k_new) + row * 16 + lane16;
+    *dst = __ldg(src);
+  }
+}
+
+__global__ void kve_advance_len_kernel(int32_t* seq_len, int B, int n_new) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) seq_len[b] += n_new;
+}
+
+__global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) seq_len[b] = n;
+}
+
+cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st) {
+  const long long total = (long long)v.S * n_new * 32;
+  long long blocks = (total + 255) / 256;
+  if (blocks > 148LL * 32) blocks = 148LL * 32;   // grid-stride beyond 32 CTAs per SM
+  if (blocks < 1) blocks = 1;
+  kve_append_kernel<<<(unsigned)blocks, 256, 0, st>>>(v, static_cast<const uint4*>(k_new),
+                                                      static_cast<const uint4*>(v_new), n_new);
+  kve_advance_len_kernel<<<(v.B + 127) / 128, 128, 0, st>>>(v.seq_len, v.B, n_new);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st) {
+  kve_set_len_kernel<<<(v.B + 127) / 128, 128, 0, st>>>(v.seq_len, v.B, n);
+  return cudaGetLastError();
+}
+
+}  // namespace kve

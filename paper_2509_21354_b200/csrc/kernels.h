@@ -1,0 +1,58 @@
+// Internal launch interface between the host API (api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace kve {
+
+// Device pointers of ONE layer plus the geometry the kernels need.
+struct LayerView {
+  uint16_t* k_pages;          // bf16 [n_pages][C][128]
+  uint16_t* v_pages;
+  int64_t n_pages;
+  const int32_t* page_table;  // [S][max_chunks]
+  int32_t* seq_len;           // [B]
+  float* ksum_f32;            // [S][max_chunks][128]
+  float* vsum_f32;
+  uint16_t* ksum_bf16;
+  uint16_t* vsum_bf16;
+  float* scores;              // [S][max_chunks]
+  int32_t* keep_idx;          // [S][max_chunks]
+  int32_t* keep_cnt;          // [S]
+  float* lstm_h;              // [S][d_g]
+  float* lstm_c;
+  int32_t* status;
+  int B, H, S, C, max_chunks, max_tokens;
+};
+
+struct MlpWeights {
+  const uint16_t *W1K, *W2K, *W1V, *W2V;   // bf16
+  const float *b1K, *b2K, *b1V, *b2V;
+};
+
+enum AttnMode { ATTN_SUMMARY = 0, ATTN_RAW = 1, ATTN_DENSE = 2 };
+
+// attention split geometry chosen on the host
+struct AttnPlan {
+  int rows_per_split;   // multiple of the kernel's tile height
+  int max_splits;       // grid.x: upper bound of splits any sequence can need
+};
+constexpr int ATTN_TILE_ROWS = 64;
+constexpr int ATTN_PARTIAL_FLOATS = 128 + 2;   // acc[128], m, l
+
+cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st);
+cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st);
+cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, cudaStream_t st);
+cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st);
+cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t* W_ih, const float* b_ih,
+                             const float* b_hh, int d_g, float* P, cudaStream_t st);
+cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
+                            int d_g, const float* P, bool reset_state, cudaStream_t st);
+cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStream_t st);
+cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_tokens_upper, AttnPlan plan,
+                        const void* q, void* out, float* lse, float scale, float* partials, int32_t* counters,
+                        cudaStream_t st);
+int attn_smem_bytes();
+
+}  // namespace kve

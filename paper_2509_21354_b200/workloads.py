@@ -103,21 +103,28 @@ def _rng(*key) -> np.random.Generator:
 _TAG_KV, _TAG_CHUNK, _TAG_Q, _TAG_MLP, _TAG_LSTM, _TAG_NEW = 1, 2, 3, 4, 5, 6
 
 
-def gen_kv(wl: Workload, layer: int = 0, n=None):
-    """K, V [S, n, d] bf16 bits.  K rows get a per-(sequence, chunk) offset when the workload asks."""
+def gen_kv_seq(wl: Workload, layer: int, s: int, n=None):
+    """K, V [n, d] bf16 bits of sequence s alone (its own sub-seeded stream, so any subset of the
+    sequences can be drawn without the others).  K rows get a per-chunk offset when the workload asks."""
     n = wl.n if n is None else n
-    rng = _rng(wl.seed, _TAG_KV, layer)
-    K = np.empty((wl.S, n, wl.d), np.uint16)
-    V = np.empty((wl.S, n, wl.d), np.uint16)
-    n_chunks = -(-n // wl.C)
-    for s in range(wl.S):   # per sequence: bounded temporaries, same stream order at any size
-        k = rng.standard_normal((n, wl.d), dtype=np.float32)
-        v = rng.standard_normal((n, wl.d), dtype=np.float32)
-        if wl.key_offset_std > 0:
-            off = rng.standard_normal((n_chunks, wl.d), dtype=np.float32) * np.float32(wl.key_offset_std)
-            k += np.repeat(off, wl.C, axis=0)[:n]
-        K[s] = f32_to_bf16_bits(k)
-        V[s] = f32_to_bf16_bits(v)
+    rng = _rng(wl.seed, _TAG_KV, layer, s)
+    k = rng.standard_normal((n, wl.d), dtype=np.float32)
+    v = rng.standard_normal((n, wl.d), dtype=np.float32)
+    if wl.key_offset_std > 0:
+        n_chunks = -(-n // wl.C)
+        off = rng.standard_normal((n_chunks, wl.d), dtype=np.float32) * np.float32(wl.key_offset_std)
+        k += np.repeat(off, wl.C, axis=0)[:n]
+    return f32_to_bf16_bits(k), f32_to_bf16_bits(v)
+
+
+def gen_kv(wl: Workload, layer: int = 0, n=None, seqs=None):
+    """K, V [len(seqs), n, d] bf16 bits (all S sequences by default)."""
+    n = wl.n if n is None else n
+    seqs = range(wl.S) if seqs is None else seqs
+    K = np.empty((len(seqs), n, wl.d), np.uint16)
+    V = np.empty((len(seqs), n, wl.d), np.uint16)
+    for i, s in enumerate(seqs):
+        K[i], V[i] = gen_kv_seq(wl, layer, int(s), n)
     return K, V
 
 

@@ -1,0 +1,430 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the oracle on the same
+seeded inputs.  Index sets bit-exact; floating point within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kvo
+from paper_2509_21354_b200 import workloads as wlm
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2509_21354_b200 import binding
+    return binding
+
+
+def make_store(wl, attend="summary", page_perm="random", n_layers=1, S=None):
+    b = _binding()
+    return b.Store(B=wl.B, H=wl.H, C_=wl.C, W=wl.W, max_tokens=wl.max_tokens, d_g=wl.d_g, agg=wl.agg,
+                   d_sum=wl.d_sum, attend=attend, n_layers=n_layers, page_perm=page_perm, seed=wl.seed + 7)
+
+
+def load_kv(st, layer, K, V, pieces=(1.0,)):
+    """prefill through kvE_append, optionally in several ragged pieces"""
+    b = _binding()
+    n = K.shape[1]
+    cuts = sorted({0, n} | {int(n * f) for f in pieces})
+    for a, e in zip(cuts, cuts[1:]):
+        st.append(layer, b.bits_to_bf16(K[:, a:e]), b.bits_to_bf16(V[:, a:e]))
+
+
+def pages_to_plain(st, layer, n):
+    """read the paged store back into the plain [S, n, d] layout (host), via the page table"""
+    b = _binding()
+    pt = st.page_table[layer].cpu().numpy()
+    kp, vp = b.bf16_to_bits(st.k_pages), b.bf16_to_bits(st.v_pages)
+    nch = -(-n // st.C)
+    K = kp[pt[:, :nch]].reshape(st.S, nch * st.C, 128)[:, :n]
+    V = vp[pt[:, :nch]].reshape(st.S, nch * st.C, 128)[:, :n]
+    return K, V
+
+
+def run_gpu_pipeline(st, pb, layer=0, agg_w=None, lstm_w=None):
+    st.summarize_chunks(layer, 0, pb.Nc, agg_w)
+    st.gate(layer, 0, pb.Nc, lstm_w)
+    st.compact(layer, pb.tau)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+
+
+def check_summaries(st, pb, layer=0):
+    b = _binding()
+    Nc = pb.Nc
+    if Nc == 0:
+        return
+    kf = st.ksum_f32[layer, :, :Nc].cpu().numpy()
+    vf = st.vsum_f32[layer, :, :Nc].cpu().numpy()
+    kb = b.bf16_to_bits(st.ksum_bf16[layer, :, :Nc])
+    vb = b.bf16_to_bits(st.vsum_bf16[layer, :, :Nc])
+    if pb.wl.agg in ("mean", "identity"):
+        # same sequential fp32 sum and IEEE division as the f32 oracle: bit for bit
+        assert np.array_equal(kf, pb.sm32["ksum"][:, :Nc]) and np.array_equal(vf, pb.sm32["vsum"][:, :Nc])
+        assert np.array_equal(kb, pb.sm32["ksum_b16"][:, :Nc]) and np.array_equal(vb, pb.sm32["vsum_b16"][:, :Nc])
+    else:
+        # MLP: fp32 dot products in another order; erf from another library
+        for got, want in ((kf, pb.sm64["ksum"][:, :Nc]), (vf, pb.sm64["vsum"][:, :Nc])):
+            assert np.abs(got - want).max() <= 2e-5 * max(1.0, np.abs(want).max())
+        for got, want in ((kb, pb.sm32["ksum_b16"][:, :Nc]), (vb, pb.sm32["vsum_b16"][:, :Nc])):
+            dist = hz.bf16_ulp_distance(got, want)
+            assert dist.max() <= 1 and (dist > 0).mean() < 2e-3     # a rounding decision flips only at a tie
+    assert np.abs(kf - pb.sm64["ksum"][:, :Nc]).max() <= 2e-5 * max(1.0, np.abs(pb.sm64["ksum"]).max())
+
+
+def check_gate_and_keep(st, pb, layer=0):
+    Nc = pb.Nc
+    sc = st.scores[layer, :, :Nc].cpu().numpy()
+    assert np.abs(sc - pb.sc32[:, :Nc]).max() <= 2e-4
+    assert np.abs(sc - pb.sc64[:, :Nc]).max() <= 2e-4
+    assert np.abs(sc - pb.tau).min() >= 1e-3 if Nc else True     # the margin survived on the GPU side too
+    if Nc:
+        assert np.abs(st.lstm_h[layer].cpu().numpy() - pb.h64).max() <= 2e-4
+        assert np.abs(st.lstm_c[layer].cpu().numpy() - pb.c64).max() <= 4e-4
+    idx, cnt = st.keep_idx[layer].cpu().numpy(), st.keep_cnt[layer].cpu().numpy()
+    for want_idx, want_cnt in ((pb.idx32, pb.cnt32), (pb.idx64, pb.cnt64)):
+        assert np.array_equal(cnt, want_cnt)
+        assert np.array_equal(idx, want_idx)       # ascending kept ids, then -1 padding: bit-exact
+
+
+def check_attention(st, pb, attend, layer=0, step=0, K=None, V=None, n_chunks=None):
+    b = _binding()
+    q = wlm.gen_q(pb.wl, layer, step)[pb.seq_ids]
+    qd = b.bits_to_bf16(q)
+    lse = torch.zeros(st.S, dtype=torch.float32, device="cuda")
+    out = st.decode_attn(layer, qd, lse=lse)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    want, want_b, want_lse, n_eff = pb.oracle_attn(q, attend, "f64", K, V, n_chunks)
+    err = hz.check_output(b.bf16_to_bits(out), want, f"attn/{attend}")
+    assert np.abs(lse.cpu().numpy() - want_lse).max() <= 1e-3
+    return err, n_eff
+
+
+def check_dense(st, pb, layer=0, step=0, K=None, V=None):
+    b = _binding()
+    q = wlm.gen_q(pb.wl, layer, 100 + step)[pb.seq_ids]
+    lse = torch.zeros(st.S, dtype=torch.float32, device="cuda")
+    out = st.decode_attn_dense(layer, b.bits_to_bf16(q), lse=lse)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    want, _, want_lse = pb.oracle_dense(q, "f64", K, V)
+    hz.check_output(b.bf16_to_bits(out), want, "dense")
+    assert np.abs(lse.cpu().numpy() - want_lse).max() <= 1e-3
+
+
+def full_check(wl, attend="summary", pieces=(1.0,), keep=0.5):
+    b = _binding()
+    pb = hz.Problem(wl, keep=keep)
+    st = make_store(wl, attend)
+    load_kv(st, 0, pb.K, pb.V, pieces)
+    torch.cuda.synchronize()
+    Kp, Vp = pages_to_plain(st, 0, wl.n)
+    assert np.array_equal(Kp, pb.K) and np.array_equal(Vp, pb.V)          # append: byte-exact through the page table
+    assert st.seq_len[0].cpu().tolist() == [wl.n] * wl.B
+    agg_w = b.AggWeights(pb.mlp) if pb.mlp is not None else None
+    lstm_w = b.LstmWeights(pb.lstm)
+    run_gpu_pipeline(st, pb, 0, agg_w, lstm_w)
+    check_summaries(st, pb)
+    check_gate_and_keep(st, pb)
+    check_attention(st, pb, attend)
+    check_dense(st, pb)
+    return st, pb, agg_w, lstm_w
+
+
+# ------------------------------------------------------------------------------------------------
+def test_config1_full(request):
+    full_check(wlm.CFG1, "summary")
+    full_check(wlm.CFG1, "raw", pieces=(0.37, 0.9))
+
+
+@pytest.mark.parametrize("attend", ["summary", "raw"])
+def test_small_mlp_ragged(attend):
+    # S = 15 (not a multiple of the gate's 8 sequences per cluster), n ragged against C and the 64-row tiles
+    wl = wlm.Workload("ragged", B=3, H=5, n=1000 + 37, C=32, W=100, d_g=256, agg="mlp", d_sum=64, key_offset_std=0.5, seed=3)
+    full_check(wl, attend, pieces=(0.5,))
+
+
+@pytest.mark.parametrize("d_g", [64, 128, 256])
+@pytest.mark.parametrize("C", [32, 128, 256])
+def test_gate_sizes_and_chunk_sizes(d_g, C):
+    wl = wlm.Workload("sizes", B=2, H=9, n=6 * C + 150, C=C, W=128, d_g=d_g, agg="mean", key_offset_std=0.5, seed=d_g + C)
+    full_check(wl, "summary")
+
+
+def test_chunk_of_one_identity_keep_all_is_dense():
+    # C = 1 with identity aggregation and tau = 0: the summary path reproduces dense attention
+    b = _binding()
+    wl = wlm.Workload("ident", B=1, H=4, n=300, C=1, W=44, d_g=64, agg="identity", seed=11, tau=0.0)
+    pb = hz.Problem(wl, keep=None, tau=0.0, margin_eps=0.0)
+    st = make_store(wl, "summary")
+    load_kv(st, 0, pb.K, pb.V)
+    run_gpu_pipeline(st, pb, 0, None, b.LstmWeights(pb.lstm))
+    assert np.array_equal(b.bf16_to_bits(st.ksum_bf16[0, :, :pb.Nc]), pb.K[:, :pb.Nc])
+    assert st.keep_cnt[0].cpu().tolist() == [pb.Nc] * wl.S
+    q = wlm.gen_q(wl)
+    out = st.decode_attn(0, b.bits_to_bf16(q))
+    dense = st.decode_attn_dense(0, b.bits_to_bf16(q))
+    want, _, _ = pb.oracle_dense(q)
+    hz.check_output(b.bf16_to_bits(out), want, "identity keep-all")
+    hz.check_output(b.bf16_to_bits(dense), want, "dense")
+
+
+def test_keep_everything_raw_equals_dense_and_keep_nothing_is_window_only():
+    b = _binding()
+    wl = wlm.CFG1.small(n=1500, seed=5)
+    pb = hz.Problem(wl)
+    st = make_store(wl, "raw")
+    load_kv(st, 0, pb.K, pb.V)
+    lw = b.LstmWeights(pb.lstm)
+    st.summarize_chunks(0, 0, pb.Nc)
+    st.gate(0, 0, pb.Nc, lw)
+    q = wlm.gen_q(wl)
+    qd = b.bits_to_bf16(q)
+    st.compact(0, 0.0)                                   # tau = 0 keeps every chunk
+    assert st.keep_cnt[0].cpu().tolist() == [pb.Nc] * wl.S
+    want, _, _ = pb.oracle_dense(q)
+    hz.check_output(b.bf16_to_bits(st.decode_attn(0, qd)), want, "raw keep-all == dense")
+    st.compact(0, 1.5)                                   # tau > 1 keeps nothing
+    assert st.keep_cnt[0].cpu().tolist() == [0] * wl.S
+    R = wl.n - pb.Nc * wl.C
+    want, _, _ = pb.o64.attn_dense(q, np.ascontiguousarray(pb.K[:, -R:]), np.ascontiguousarray(pb.V[:, -R:]), hz.SCALE)
+    hz.check_output(b.bf16_to_bits(st.decode_attn(0, qd)), want, "keep-nothing == window only")
+    assert st.poll_status() == 0
+
+
+def test_no_stale_chunks_and_empty_cache():
+    b = _binding()
+    wl = wlm.Workload("short", B=2, H=3, n=100, C=64, W=256, d_g=128, seed=2)      # n < W: nothing to gate
+    pb = hz.Problem(wl, keep=None)
+    assert pb.Nc == 0
+    st = make_store(wl)
+    q = wlm.gen_q(wl)
+    qd = b.bits_to_bf16(q)
+    lse = torch.zeros(wl.S, device="cuda")
+    out = st.decode_attn(0, qd, lse=lse)                 # empty cache: zeros, lse = -inf
+    assert torch.all(out.float() == 0) and torch.all(torch.isneginf(lse))
+    load_kv(st, 0, pb.K, pb.V)
+    lw = b.LstmWeights(pb.lstm)
+    st.summarize_chunks(0, 0, 0)
+    st.gate(0, 0, 0, lw)
+    st.compact(0, 0.5)
+    check_attention(st, pb, "summary")
+    check_dense(st, pb)
+
+
+def test_incremental_gate_equals_from_scratch_and_append_decode_steps():
+    """Gate the first chunks, append tokens until more chunks leave the window, gate only the new
+    ones with the carried (h, c): scores and keep list equal the from-scratch oracle.  Then a few
+    append + decode steps (the cache grows, no chunk completes) against the oracle."""
+    b = _binding()
+    wl = wlm.CFG3.small(B=2, H=4, n_layers=1, n=64 + 5 * 256, seed=9)
+    pb = hz.Problem(wl)
+    st = make_store(wl)
+    aw, lw = b.AggWeights(pb.mlp), b.LstmWeights(pb.lstm)
+    n1 = 64 + 3 * 256 + 17
+    st.append(0, b.bits_to_bf16(pb.K[:, :n1]), b.bits_to_bf16(pb.V[:, :n1]))
+    nc1 = wl.n_stale_chunks(n1)
+    st.summarize_chunks(0, 0, nc1, aw)
+    st.gate(0, 0, nc1, lw)
+    ready = st.append(0, b.bits_to_bf16(pb.K[:, n1:]), b.bits_to_bf16(pb.V[:, n1:]))
+    assert ready == pb.Nc - nc1 and ready > 0
+    st.summarize_chunks(0, nc1, pb.Nc, aw)
+    st.gate(0, nc1, pb.Nc, lw)
+    st.compact(0, pb.tau)
+    check_summaries(st, pb)
+    check_gate_and_keep(st, pb)
+    K, V = pb.K, pb.V
+    for step in range(wl.n_append):
+        kn, vn = wlm.gen_new_tokens(wl, 0, step)
+        st.append(0, b.bits_to_bf16(kn), b.bits_to_bf16(vn))
+        K, V = np.concatenate([K, kn], axis=1), np.concatenate([V, vn], axis=1)
+        check_attention(st, pb, "summary", step=step, K=K, V=V)
+    check_dense(st, pb, K=K, V=V)
+    assert st.layer_state(0) == dict(n_tokens=wl.n + wl.n_append, n_summarised=pb.Nc, n_gated=pb.Nc, n_compacted=pb.Nc)
+
+
+def test_layers_are_independent():
+    b = _binding()
+    wl = wlm.CFG1.small(n=1024, B=2, H=4, n_layers=3)
+    st = make_store(wl, n_layers=3)
+    pbs = [hz.Problem(wl.small(seed=wl.seed + L), layer=L) for L in range(3)]
+    for L in (2, 0, 1):
+        load_kv(st, L, pbs[L].K, pbs[L].V)
+    for L in range(3):
+        lw = b.LstmWeights(pbs[L].lstm)
+        run_gpu_pipeline(st, pbs[L], L, None, lw)
+    for L in range(3):
+        check_summaries(st, pbs[L], L)
+        check_gate_and_keep(st, pbs[L], L)
+        check_attention(st, pbs[L], "summary", L)
+
+
+def test_decode_step_host_matches_stepwise_calls():
+    b = _binding()
+    wl = wlm.CFG1.small(n=1024 - 1, seed=4)
+    pb0 = hz.Problem(wl.small(n=1024), keep=0.5)          # oracle on the cache AFTER the step's append
+    st = make_store(wl.small(n=1024))
+    lw = b.LstmWeights(pb0.lstm)
+    load_kv(st, 0, pb0.K[:, :-1], pb0.V[:, :-1])
+    q = wlm.gen_q(wl)
+    pin = lambda a: b.bits_to_bf16(a, "cpu").pin_memory()
+    out = torch.zeros(wl.S, 128, dtype=torch.bfloat16).pin_memory()
+    st.decode_step_host(0, pin(pb0.K[:, -1]), pin(pb0.V[:, -1]), pin(q), out, None, lw, pb0.tau, from_scratch=True)
+    want, _, _, _ = pb0.oracle_attn(q, "summary")
+    hz.check_output(b.bf16_to_bits(out), want, "step_host")
+    check_gate_and_keep(st, pb0)
+
+
+def test_host_side_errors():
+    b = _binding()
+    wl = wlm.CFG1.small(n=512)
+    st = make_store(wl)
+    pb = hz.Problem(wl)
+    lw = b.LstmWeights(pb.lstm)
+    with pytest.raises(b.KveError) as e:                  # nothing stored yet: no chunk may be summarised
+        st.summarize_chunks(0, 0, 1)
+    assert e.value.rc == -4
+    load_kv(st, 0, pb.K, pb.V)
+    with pytest.raises(b.KveError) as e:                  # gate before summarize
+        st.gate(0, 0, pb.Nc, lw)
+    assert e.value.rc == -4
+    with pytest.raises(b.KveError) as e:                  # capacity
+        st.append(0, b.bits_to_bf16(pb.K[:, :1]), b.bits_to_bf16(pb.V[:, :1]))
+    assert e.value.rc == -3
+    with pytest.raises(b.KveError) as e:                  # bad layer
+        st.compact(5, 0.5)
+    assert e.value.rc == -1
+    st.summarize_chunks(0, 0, pb.Nc)
+    with pytest.raises(b.KveError) as e:                  # gate must continue where it stopped
+        st.gate(0, 2, pb.Nc, lw)
+    assert e.value.rc == -4
+    with pytest.raises(b.KveError):                       # unsupported geometry is refused at create
+        b.Store(B=1, H=1, C_=64, W=0, max_tokens=128, d_g=100)
+    assert st.poll_status() == 0
+
+
+def test_bad_page_id_sets_status_word_without_fault():
+    b = _binding()
+    wl = wlm.CFG1.small(n=512)
+    pt = np.arange(wl.S * wl.max_chunks, dtype=np.int32).reshape(1, wl.S, wl.max_chunks)
+    pt[0, 1, 2] = 10 ** 6                                 # beyond n_pages: the kernels must skip it
+    st = make_store(wl, page_perm=pt)
+    pb = hz.Problem(wl)
+    load_kv(st, 0, pb.K, pb.V)
+    torch.cuda.synchronize()
+    assert st.poll_status() == -3
+    assert st.poll_status() == 0                          # cleared by the poll
+
+
+# ------------------------------------------------------------------------------------------------ full sizes
+def test_config2_full_size():
+    """Llama-2-7B-shaped layer at the size bench.py times (B 8, H 32, n 4096, MLP aggregator, d_g 256)."""
+    st, pb, aw, lw = full_check(wlm.CFG2, "summary")
+    keep = st.keep_cnt[0].float().mean().item() / pb.Nc
+    assert 0.4 < keep < 0.6
+    # the RAW reading on the same store contents
+    st2 = make_store(wlm.CFG2, "raw")
+    load_kv(st2, 0, pb.K, pb.V)
+    run_gpu_pipeline(st2, pb, 0, aw, lw)
+    check_gate_and_keep(st2, pb)
+    check_attention(st2, pb, "raw")
+
+
+def _sampled_full_size(wl, n_sample, attend="summary", n_steps=0):
+    """Full-size launch, oracle on a sample of the sequences: the sampled sequences carry seeded,
+    margin-repaired inputs, the others carry device-generated filler of the same distribution."""
+    b = _binding()
+    rng = np.random.default_rng(wl.seed)
+    seqs = sorted(rng.choice(wl.S, n_sample, replace=False).tolist())
+    pb = hz.Problem(wl, seq_ids=seqs)
+    st = make_store(wl, attend, page_perm=None)
+    g = torch.Generator(device="cuda").manual_seed(wl.seed)
+    for b0 in range(0, wl.S, 64):                           # filler, 64 sequences at a time
+        shape = (min(64, wl.S - b0), wl.n, 128)
+        kf = torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        vf = torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        pages = st.page_table[0, b0:b0 + shape[0]].long()   # [s, max_chunks]
+        nch = wl.n // wl.C
+        st.k_pages[pages[:, :nch].reshape(-1)] = kf[:, :nch * wl.C].reshape(-1, wl.C, 128)
+        st.v_pages[pages[:, :nch].reshape(-1)] = vf[:, :nch * wl.C].reshape(-1, wl.C, 128)
+        del kf, vf
+    for i, s in enumerate(seqs):                            # the sampled sequences' real data
+        pages = st.page_table[0, s].long()
+        nch = -(-wl.n // wl.C)
+        pad = nch * wl.C - wl.n
+        kk = np.pad(pb.K[i], ((0, pad), (0, 0)))
+        vv = np.pad(pb.V[i], ((0, pad), (0, 0)))
+        st.k_pages[pages[:nch]] = b.bits_to_bf16(kk).reshape(nch, wl.C, 128)
+        st.v_pages[pages[:nch]] = b.bits_to_bf16(vv).reshape(nch, wl.C, 128)
+    st.set_len(0, wl.n)
+    aw, lw = (b.AggWeights(pb.mlp) if pb.mlp else None), b.LstmWeights(pb.lstm)
+    run_gpu_pipeline(st, pb, 0, aw, lw)
+    sel = torch.tensor(seqs, device="cuda")
+    Nc = pb.Nc
+    sc = st.scores[0, sel, :Nc].cpu().numpy()
+    assert np.abs(sc - pb.sc64[:, :Nc]).max() <= 2e-4
+    assert np.array_equal(st.keep_cnt[0, sel].cpu().numpy(), pb.cnt64)
+    assert np.array_equal(st.keep_idx[0, sel].cpu().numpy(), pb.idx64)
+    kb = b.bf16_to_bits(st.ksum_bf16[0, sel, :Nc])
+    assert hz.bf16_ulp_distance(kb, pb.sm32["ksum_b16"][:, :Nc]).max() <= 1
+    # properties that hold for every sequence at any size
+    cnt = st.keep_cnt[0].cpu().numpy()
+    idx = st.keep_idx[0].cpu().numpy()
+    scores = st.scores[0, :, :Nc].cpu().numpy()
+    assert np.array_equal(cnt, (scores >= np.float32(pb.tau)).sum(axis=1))
+    for s in range(0, wl.S, 7):
+        assert np.array_equal(idx[s, :cnt[s]], np.nonzero(scores[s] >= np.float32(pb.tau))[0]) and np.all(idx[s, cnt[s]:] == -1)
+    K, V = pb.K, pb.V
+    for step in range(max(1, n_steps)):
+        if n_steps:
+            kn, vn = wlm.gen_new_tokens(wl, 0, step)
+            st.append(0, b.bits_to_bf16(kn), b.bits_to_bf16(vn))
+            K, V = np.concatenate([K, kn[seqs]], axis=1), np.concatenate([V, vn[seqs]], axis=1)
+        q = wlm.gen_q(wl, 0, step)
+        out = st.decode_attn(0, b.bits_to_bf16(q))
+        want, _, _, _ = pb.oracle_attn(q[seqs], attend, "f64", K, V)
+        hz.check_output(b.bf16_to_bits(out[sel]), want, f"sampled attn step {step}")
+        assert torch.isfinite(out.float()).all()
+    dense = st.decode_attn_dense(0, b.bits_to_bf16(q))
+    want, _, _ = pb.oracle_dense(q[seqs], "f64", K, V)
+    hz.check_output(b.bf16_to_bits(dense[sel]), want, "sampled dense")
+    assert st.poll_status() == 0
+
+
+def test_config3_one_layer_full_size_sampled():
+    _sampled_full_size(wlm.CFG3.small(n_layers=1), n_sample=8, n_steps=wlm.CFG3.n_append)
+
+
+def test_config4_one_layer_full_size_sampled():
+    _sampled_full_size(wlm.CFG4.small(n_layers=1), n_sample=6)
+
+
+@pytest.mark.parametrize("B,n,C,keep", [(1, 2048, 32, 0.25), (4, 8192, 64, 0.75), (2, 32768, 256, 1.0), (64, 2048, 128, 0.5)])
+def test_sweep_points_sampled(B, n, C, keep):
+    wl = wlm.Workload(f"sweep_b{B}_n{n}_c{C}", B=B, H=32, n=n, C=C, W=512, d_g=256, agg="mean", key_offset_std=0.5, seed=B + n + C)
+    b = _binding()
+    rng = np.random.default_rng(1)
+    seqs = sorted(rng.choice(wl.S, min(4, wl.S), replace=False).tolist())
+    if keep >= 1.0:
+        pb = hz.Problem(wl, seq_ids=seqs, keep=None, tau=0.0, margin_eps=0.0)
+    else:
+        pb = hz.Problem(wl, seq_ids=seqs, keep=keep)
+    for attend in ("summary", "raw"):
+        st = make_store(wl, attend, page_perm=None)
+        for i, s in enumerate(seqs):
+            pages = st.page_table[0, s].long()
+            nch = wl.n // wl.C
+            st.k_pages[pages[:nch]] = b.bits_to_bf16(pb.K[i]).reshape(nch, wl.C, 128)
+            st.v_pages[pages[:nch]] = b.bits_to_bf16(pb.V[i]).reshape(nch, wl.C, 128)
+        st.set_len(0, wl.n)
+        run_gpu_pipeline(st, pb, 0, None, b.LstmWeights(pb.lstm))
+        sel = torch.tensor(seqs, device="cuda")
+        assert np.array_equal(st.keep_idx[0, sel].cpu().numpy(), pb.idx64)
+        q = wlm.gen_q(wl)
+        out = st.decode_attn(0, b.bits_to_bf16(q))
+        want, _, _, _ = pb.oracle_attn(q[seqs], attend)
+        hz.check_output(b.bf16_to_bits(out[sel]), want, f"sweep {attend}")
+        del st
+        torch.cuda.empty_cache()
