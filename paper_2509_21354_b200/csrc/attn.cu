@@ -37,7 +37,7 @@ struct AttnArgs {
   uint16_t* out;
   float* lse;
   float scale;
-  float* partials;     // [S][max_splits][130]
+  float* partials;     // [S][max_splits][132]
   int32_t* counters;   // [S], zero between launches
 };
 
@@ -86,8 +86,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   extern __shared__ __align__(128) unsigned char smem[];
   uint16_t* Ks = reinterpret_cast<uint16_t*>(smem);
   uint16_t* Vs = Ks + AT_STAGES * AT_STAGE_ELEMS;
-  float* comb = reinterpret_cast<float*>(Vs + AT_STAGES * AT_STAGE_ELEMS);          // [AT_CWARPS][130]
-  uint64_t* full = reinterpret_cast<uint64_t*>(comb + AT_CWARPS * ATTN_PARTIAL_FLOATS + 2);   // 8-byte aligned
+  float* comb = reinterpret_cast<float*>(Vs + AT_STAGES * AT_STAGE_ELEMS);          // [AT_CWARPS][132]
+  uint64_t* full = reinterpret_cast<uint64_t*>(comb + AT_CWARPS * ATTN_PARTIAL_FLOATS);   // 16-byte aligned
   uint64_t* empty = full + AT_STAGES;
 
   const LayerView& v = a.v;

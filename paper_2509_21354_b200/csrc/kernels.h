@@ -39,7 +39,7 @@ struct AttnPlan {
   int max_splits;       // grid.x: upper bound of splits any sequence can need
 };
 constexpr int ATTN_TILE_ROWS = 64;
-constexpr int ATTN_PARTIAL_FLOATS = 128 + 2;   // acc[128], m, l
+constexpr int ATTN_PARTIAL_FLOATS = 132;       // acc[128], m, l, 2 pad: keeps every record 16-byte aligned
 
 cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st);
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st);

@@ -68,8 +68,11 @@ def check_summaries(st, pb, layer=0):
         for got, want in ((kf, pb.sm64["ksum"][:, :Nc]), (vf, pb.sm64["vsum"][:, :Nc])):
             assert np.abs(got - want).max() <= 2e-5 * max(1.0, np.abs(want).max())
         for got, want in ((kb, pb.sm32["ksum_b16"][:, :Nc]), (vb, pb.sm32["vsum_b16"][:, :Nc])):
-            dist = hz.bf16_ulp_distance(got, want)
-            assert dist.max() <= 1 and (dist > 0).mean() < 2e-3     # a rounding decision flips only at a tie
+            # a rounding decision flips only next to a tie: at most one bf16 step (2^-7 relative; near
+            # zero the fp32 noise itself spans several tiny steps), and rarely
+            g, w = wlm.bf16_bits_to_f32(got).astype(np.float64), wlm.bf16_bits_to_f32(want).astype(np.float64)
+            assert np.all(np.abs(g - w) <= 2.0 ** -7 * np.abs(w) + 1e-5)
+            assert (got != want).mean() < 2e-3
     assert np.abs(kf - pb.sm64["ksum"][:, :Nc]).max() <= 2e-5 * max(1.0, np.abs(pb.sm64["ksum"]).max())
 
 
@@ -368,7 +371,8 @@ def _sampled_full_size(wl, n_sample, attend="summary", n_steps=0):
     assert np.array_equal(st.keep_cnt[0, sel].cpu().numpy(), pb.cnt64)
     assert np.array_equal(st.keep_idx[0, sel].cpu().numpy(), pb.idx64)
     kb = b.bf16_to_bits(st.ksum_bf16[0, sel, :Nc])
-    assert hz.bf16_ulp_distance(kb, pb.sm32["ksum_b16"][:, :Nc]).max() <= 1
+    kg, kw = (wlm.bf16_bits_to_f32(x).astype(np.float64) for x in (kb, pb.sm32["ksum_b16"][:, :Nc]))
+    assert np.all(np.abs(kg - kw) <= 2.0 ** -7 * np.abs(kw) + 1e-5)
     # properties that hold for every sequence at any size
     cnt = st.keep_cnt[0].cpu().numpy()
     idx = st.keep_idx[0].cpu().numpy()
