@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the gated chunked-KV decode path (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+
+A *step* is one pass of the whole hot path over one layer of the workload, from scratch:
+append one token to every sequence, summarise every chunk that lies outside the window, run the
+LSTM gate over all of them, compact the keep list, run the gated decode attention.  `value` is
+whole-job steps per second with all inputs resident in HBM; `e2e` is the same step through
+kvE_decode_step_host with pinned HOST buffers (H2D of k_new, v_new, q and D2H of the output inside
+the timed region).  Under torchrun every rank runs the same per-GPU workload on its own batch
+shard (weak scaling, no data-path collective: (layer, batch, head) units are independent).
+
+`--impl reference` times the CPU oracle (oracle/, as it stands) on the host cores on a bounded
+sample of the same workload.
+"""
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2509_21354_b200 import workloads as wlm  # noqa: E402
+
+METRIC = "gated_decode_attention_steps_per_sec"
+UNIT = "steps/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+SCALE = 1.0 / math.sqrt(128.0)
+KERNELS_PER_STEP = 9   # set_len, append (copy + length), chunk mean, chunk MLP, gate projection, gate recurrence, compact, attention
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def shard_batch(B_per_gpu: int, rank: int, world: int):
+    """Weak scaling: every rank owns B_per_gpu sequences-batches of its own; returns the global batch
+    range [lo, hi) this rank stands for (used to derive its data seed).  No collective is needed:
+    the gated cache of one (layer, batch, head) never reads another's."""
+    lo = rank * B_per_gpu
+    return lo, lo + B_per_gpu
+
+
+# ---------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs (read-only NVML)."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz, self._stop, self._thr = None, threading.Event(), None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------------- GPU arm
+def fill_cache(st, wl, seed):
+    """Synthetic cache of the workload's shape, generated on the device: N(0,1) keys and values, keys
+    shifted by a per-(sequence, chunk) offset ~ N(0, key_offset_std^2); stored through kvE_append."""
+    import torch
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    slab = max(wl.C, (512 // wl.C) * wl.C)
+    n_fill = wl.n - 1                      # the step appends the last token itself
+    for a in range(0, n_fill, slab):
+        m = min(slab, n_fill - a)
+        k = torch.randn((wl.S, m, 128), generator=g, device="cuda", dtype=torch.float32)
+        v = torch.randn((wl.S, m, 128), generator=g, device="cuda", dtype=torch.float32)
+        if wl.key_offset_std > 0:
+            nch = -(-m // wl.C)
+            off = torch.randn((wl.S, nch, 128), generator=g, device="cuda", dtype=torch.float32) * wl.key_offset_std
+            k += off.repeat_interleave(wl.C, dim=1)[:, :m]
+        st.append(0, k.to(torch.bfloat16).contiguous(), v.to(torch.bfloat16).contiguous())
+    return g
+
+
+def algorithmic_bytes(wl, Nc, keep_mean, R):
+    """Bytes each kernel must move per launch (per-unit figures x units; bf16 rows are 256 bytes)."""
+    S, d_g = wl.S, wl.d_g
+    by = {}
+    by["chunk_mean"] = S * Nc * (2 * wl.C * 256 + 2 * 128 * 4)            # every stale K and V row once; fp32 means out
+    by["chunk_mlp"] = S * Nc * 2 * (128 * 4 + 128 * 4 + 128 * 2)          # means in, fp32 + bf16 summaries out
+    by["gate_proj"] = S * Nc * (2 * 256 + 4 * d_g * 4)                    # bf16 summaries in, fp32 P out
+    by["gate_rnn"] = S * Nc * (4 * d_g * 4 + 4)                           # P in, scores out
+    by["compact"] = S * (Nc * 4 + Nc * 4 + 4)
+    by["attn_gated"] = S * (2 * (R + keep_mean) * 256 + 2 * 256)          # retained rows of K and V once (+ q, out)
+    by["attn_dense"] = S * (2 * wl.n * 256 + 2 * 256)
+    return by
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_21354_b200 import binding as b
+
+    torch.cuda.set_device(local_rank)
+    wl = wlm.CONFIGS[args.workload].small(n_layers=1)
+    lo, _ = shard_batch(wl.B, rank, world)
+    seed = 1000 + lo
+    st = b.Store(B=wl.B, H=wl.H, C_=wl.C, W=wl.W, max_tokens=wl.n, d_g=wl.d_g, agg=wl.agg, d_sum=wl.d_sum,
+                 attend=args.attend, page_perm="random", seed=seed)
+    g = fill_cache(st, wl, seed)
+    mlp = wlm.gen_mlp_weights(wl)
+    lstm = wlm.gen_lstm_weights(wl)
+    aw = b.AggWeights(mlp) if mlp is not None else None
+    lw = b.LstmWeights(lstm)
+    S = wl.S
+    rnd = lambda: torch.randn((S, 128), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16).contiguous()
+    k_new, v_new, q = rnd(), rnd(), rnd()
+    k3, v3 = k_new.view(S, 1, 128), v_new.view(S, 1, 128)
+    out = torch.empty_like(q)
+    n0 = wl.n
+    Nc = wl.n_stale_chunks(n0)
+
+    def step():
+        st.set_len(0, n0 - 1)
+        st.append(0, k3, v3)
+        st.summarize_chunks(0, 0, Nc, aw)
+        st.gate(0, 0, Nc, lw)
+        st.compact(0, wl.tau)
+        st.decode_attn(0, q, out)
+
+    # head bias that retains about half of the chunks (deterministic given the seed)
+    step()
+    torch.cuda.synchronize()
+    sc = st.scores[0, :, :Nc].double().clamp(1e-9, 1 - 1e-9)
+    lw.set_b_s(float(-torch.median(torch.log(sc / (1 - sc))).item()) + lstm["b_s"])
+    step()
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    keep_mean = st.keep_cnt[0].float().mean().item()
+    R = n0 - Nc * wl.C
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local_rank) as clk:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    assert st.poll_status() == 0
+
+    # ---- end to end: the same step through kvE_decode_step_host, host buffers, copies timed ----
+    hk, hv, hq = (t.cpu().pin_memory() for t in (k_new, v_new, q))
+    hout = torch.zeros((S, 128), dtype=torch.bfloat16).pin_memory()
+
+    def step_e2e():
+        st.set_len(0, n0 - 1)
+        st.decode_step_host(0, hk, hv, hq, hout, aw, lw, wl.tau, from_scratch=True)
+
+    for _ in range(min(args.warmup, 3)):
+        step_e2e()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step_e2e()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    same = bool(torch.equal(hout.cuda(), out))
+
+    if world > 1:
+        t = torch.tensor([ms_total, e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, e2e_s = t[0].item(), t[1].item()
+    if rank != 0:
+        return None
+
+    # ---- per-kernel timing (rank 0): the library brackets every launch with CUDA events on its stream ----
+    peaks, peak_kind = load_peaks()
+    hbm = peaks["hbm_gbs"]
+    st.profile(True)
+    in_step = {k: [] for k in b.KERNEL_IDS}
+    for _ in range(min(args.steps, 30)):          # same step as the timed region
+        step()
+        for k, v in st.profile_read().items():
+            if v is not None and k != "attn_dense":
+                in_step[k].append(v)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    cold = {"attn": [], "attn_dense": []}
+    for _ in range(10):                            # attention alone, L2 flushed before every launch
+        for name, fn in (("attn", st.decode_attn), ("attn_dense", st.decode_attn_dense)):
+            flush.fill_(1)
+            fn(0, q, out)
+            cold[name].append(st.profile_read()[name])
+    st.profile(False)
+    us = {k: float(np.mean(v)) for k, v in in_step.items() if v}
+    us["attn_dense"] = float(np.mean(cold["attn_dense"]))
+    us_attn_cold = float(np.mean(cold["attn"]))
+    by = algorithmic_bytes(wl, Nc, keep_mean, R)
+    by_kernel = {"append": S * 4 * 256, "chunk_mean": by["chunk_mean"], "chunk_mlp": by["chunk_mlp"],
+                 "gate_proj": by["gate_proj"], "gate_rnn": by["gate_rnn"], "compact": by["compact"],
+                 "attn": by["attn_gated"], "attn_dense": by["attn_dense"]}
+    kern = {}
+    for k, t in us.items():
+        kern[k] = {"us": t, "bytes": by_kernel[k], "GB/s": by_kernel[k] / (t * 1e-6) / 1e9}
+        kern[k]["frac_of_hbm_peak"] = kern[k]["GB/s"] / hbm
+    kern["attn"]["us_l2_flushed"] = us_attn_cold
+    kern["attn"]["GB/s_l2_flushed"] = by_kernel["attn"] / (us_attn_cold * 1e-6) / 1e9
+    dominant = max((k for k in kern if k != "attn_dense"), key=lambda k: kern[k]["us"])
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tp):
+        with open(tp) as f:
+            traffic = json.load(f).get(dominant)
+    roofline = {"kernel": dominant, "bound": "hbm", "achieved": kern[dominant]["GB/s"], "peak": hbm, "unit": "GB/s",
+                "frac": kern[dominant]["GB/s"] / hbm, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes": kern[dominant]["bytes"], "us_per_launch": kern[dominant]["us"]}
+    us["attn_gated"] = us_attn_cold
+
+    ms_step = ms_total / args.steps
+    res = {
+        "metric": METRIC, "value": world * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
+        "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "d": 128, "n": wl.n, "C": wl.C, "W": wl.W,
+                   "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend, "n_layers_timed": 1,
+                   "stale_chunks": Nc, "kept_chunks_mean": keep_mean, "n_eff": R + keep_mean,
+                   "memory_ratio_n_over_n_eff": n0 / (R + keep_mean),
+                   "l2": "inputs larger than L2 (each step streams 0.45 GB of stale KV + 0.06 GB window); per-kernel timings flush L2 before every launch"},
+        "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * S * 256,
+                "d2h_bytes_per_step": S * 256, "matches_device_path": same},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "clocks": clk.summary(),
+        "roofline": roofline,
+        "kernels": kern,
+        "attention_vs_dense": {"note": "attention kernels alone, L2 flushed before every launch",
+                               "gated_us": us["attn_gated"], "dense_us": us["attn_dense"],
+                               "speedup": us["attn_dense"] / us["attn_gated"],
+                               "kv_bytes_gated": by["attn_gated"], "kv_bytes_dense": by["attn_dense"],
+                               "gated_GB/s": kern["attn"]["GB/s_l2_flushed"], "dense_GB/s": kern["attn_dense"]["GB/s"],
+                               "gated_frac_of_measured_peak": kern["attn"]["GB/s_l2_flushed"] / hbm,
+                               "dense_frac_of_measured_peak": kern["attn_dense"]["GB/s"] / hbm,
+                               "gated_frac_of_nominal_8TBps": kern["attn"]["GB/s_l2_flushed"] / 8000.0,
+                               "dense_frac_of_nominal_8TBps": kern["attn_dense"]["GB/s"] / 8000.0},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        res["cpu_baseline"] = cpu_baseline(wl, args.attend, budget_s=15.0)
+    return res
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_step_time(wl, attend, n_seq, repeat=1):
+    """Seconds the oracle (f64 build, OpenMP over sequences) needs for the whole path on n_seq sequences."""
+    from oracle import kvo, margin
+    o = kvo.Oracle("f64")
+    seqs = list(range(n_seq))
+    K, V = wlm.gen_kv(wl, 0, seqs=seqs)
+    mlp, lstm = wlm.gen_mlp_weights(wl), wlm.gen_lstm_weights(wl)
+    q = wlm.gen_q(wl)[seqs]
+    Nc = wl.n_stale_chunks()
+    agg = margin.AGG_CODE[wl.agg]
+    att = kvo.ATTEND_RAW if attend == "raw" else kvo.ATTEND_SUMMARY
+    best = float("inf")
+    for _ in range(repeat):
+        t0 = time.perf_counter()
+        sm = o.summarize(K, V, wl.C, 0, Nc, agg, mlp, stride=max(wl.max_chunks, 1))
+        sc, _, _ = o.gate(sm["ksum_b16"], sm["vsum_b16"], 0, Nc, lstm)
+        idx, cnt = o.compact(sc, Nc, wl.tau)
+        o.attn(q, K, V, wl.C, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"], att, SCALE)
+        best = min(best, time.perf_counter() - t0)
+    return best
+
+
+def cpu_baseline(wl, attend, budget_s=15.0):
+    cores = os.cpu_count() or 1
+    n_probe = min(wl.S, max(cores, 8))
+    t = oracle_step_time(wl, attend, n_probe)
+    n_seq = int(min(wl.S, max(n_probe, n_probe * budget_s / max(t, 1e-6))))
+    n_seq = max(cores, n_seq // cores * cores) if n_seq >= cores else n_seq
+    n_seq = min(n_seq, wl.S)
+    t = oracle_step_time(wl, attend, n_seq)
+    step_s = t * wl.S / n_seq
+    return {"value": 1.0 / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n_seq} of {wl.S} sequences of {wl.name} (whole path, f64 oracle, OpenMP over sequences), "
+                      f"{t:.2f} s measured, scaled to the full step"}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return None
+    wl = wlm.CONFIGS[args.workload].small(n_layers=1)
+    cores = os.cpu_count() or 1
+    n_seq = min(wl.S, max(8, cores))
+    for _ in range(min(args.warmup, 1)):
+        oracle_step_time(wl, args.attend, n_seq)
+    t0 = time.perf_counter()
+    ts = [oracle_step_time(wl, args.attend, n_seq) for _ in range(args.steps)]
+    wall = time.perf_counter() - t0
+    step_s = float(np.mean(ts)) * wl.S / n_seq
+    val = 1.0 / step_s
+    sample = f"each step = {n_seq} of {wl.S} sequences of {wl.name}, scaled to the full step (f64 oracle, OpenMP over sequences)"
+    return {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "d": 128, "n": wl.n, "C": wl.C, "W": wl.W,
+                       "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "wall_s": wall}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(wlm.CONFIGS))
+    ap.add_argument("--attend", default="summary", choices=["summary", "raw"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if args.steps > 20:
+            args.steps = 20          # a bounded sample per step; keep the whole run within minutes
+        res = run_reference(args, rank)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        if world > 1:
+            import torch
+            import torch.distributed as dist
+            torch.cuda.set_device(local_rank)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        res = run_ours(args, rank, world, local_rank)
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            dist.destroy_process_group()
+    if res is not None:
+        print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    main()

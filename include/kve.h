@@ -159,6 +159,15 @@ int kvE_poll_status(kvE_store* st, int* device_status);
 int kvE_layer_state(const kvE_store* st, int layer, int* n_tokens, int* n_summarised, int* n_gated,
                     int* n_compacted);
 
+/* Per-kernel timing.  While enabled, every kernel launch of this handle is bracketed by a pair of CUDA
+ * events on the launch stream (events are created on the first enable; no device memory).
+ * kvE_profile_read synchronises the device and writes, per kernel id, the duration in microseconds
+ * of that kernel's most recent launch, or -1 if it has not run since profiling was enabled. */
+enum { KVE_K_APPEND = 0, KVE_K_CHUNK_MEAN, KVE_K_CHUNK_MLP, KVE_K_GATE_PROJ, KVE_K_GATE_RNN, KVE_K_COMPACT,
+       KVE_K_ATTN, KVE_K_ATTN_DENSE, KVE_K_COUNT };
+int kvE_profile(kvE_store* st, int enable);
+int kvE_profile_read(kvE_store* st, float* us /* [KVE_K_COUNT] */);
+
 /* Text of the last CUDA runtime error seen by this handle's calls ("" if none). */
 const char* kvE_last_cuda_error(const kvE_store* st);
 

@@ -23,7 +23,9 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_decode_attn", "kvE_decode_attn_dense",
-           "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error"]
+           "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
+           "kvE_profile", "kvE_profile_read"]
+KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense"]
 
 
 class KveError(RuntimeError):
@@ -85,6 +87,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
                                          C.c_float, C.c_int, C.c_void_p]
     lib.kvE_poll_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.kvE_layer_state.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_int)] * 4
+    lib.kvE_profile.argtypes = [C.c_void_p, C.c_int]
+    lib.kvE_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
     lib.kvE_last_cuda_error.restype = C.c_char_p
     lib.kvE_last_cuda_error.argtypes = [C.c_void_p]
     for name in EXPORTS:
@@ -252,6 +256,12 @@ class Store:
     def layer_state(self, layer=0) -> dict:
         return kvE_layer_state(self, layer)
 
+    def profile(self, enable: bool):
+        kvE_profile(self, enable)
+
+    def profile_read(self) -> dict:
+        return kvE_profile_read(self)
+
 
 def kvE_append(st: Store, layer, k_new, v_new, stream=None) -> int:
     """k_new, v_new: bf16 [S, n_new, 128] device tensors.  Returns the number of chunks ready to gate."""
@@ -323,3 +333,14 @@ def kvE_layer_state(st: Store, layer=0) -> dict:
     v = [C.c_int(0) for _ in range(4)]
     _check("kvE_layer_state", st.lib.kvE_layer_state(st.handle, layer, *[C.byref(x) for x in v]))
     return dict(zip(("n_tokens", "n_summarised", "n_gated", "n_compacted"), (x.value for x in v)))
+
+
+def kvE_profile(st: Store, enable: bool):
+    _check("kvE_profile", st.lib.kvE_profile(st.handle, 1 if enable else 0), st.handle)
+
+
+def kvE_profile_read(st: Store) -> dict:
+    """microseconds of the most recent launch of each kernel (None if it has not run)"""
+    us = (C.c_float * len(KERNEL_IDS))()
+    _check("kvE_profile_read", st.lib.kvE_profile_read(st.handle, us), st.handle)
+    return {k: (float(us[i]) if us[i] >= 0 else None) for i, k in enumerate(KERNEL_IDS)}

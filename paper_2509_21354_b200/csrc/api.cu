@@ -26,6 +26,11 @@ struct kvE_store {
   int max_splits;
   std::vector<LayerState> layers;
   std::string cuda_error;
+  // optional per-kernel timing: one (start, stop) event pair per kernel id
+  bool profiling = false;
+  cudaEvent_t ev[2 * KVE_K_COUNT] = {};
+  bool ev_made = false;
+  bool ev_used[KVE_K_COUNT] = {};
 };
 
 namespace {
@@ -63,6 +68,22 @@ Carve carve(const kvE_config& c) {
   k.total = o;
   return k;
 }
+
+// brackets the launches issued during its lifetime with the kernel id's event pair
+struct Prof {
+  kvE_store* st;
+  int id;
+  cudaStream_t s;
+  Prof(kvE_store* st_, int id_, cudaStream_t s_) : st(st_), id(id_), s(s_) {
+    if (st->profiling) cudaEventRecord(st->ev[2 * id], s);
+  }
+  ~Prof() {
+    if (st->profiling) {
+      cudaEventRecord(st->ev[2 * id + 1], s);
+      st->ev_used[id] = true;
+    }
+  }
+};
 
 int cuda_fail(kvE_store* st, cudaError_t e) {
   st->cuda_error = cudaGetErrorString(e);
@@ -126,6 +147,7 @@ int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* 
   }
   AttnPlan plan = plan_attention(st, rows_upper);
   char* ws = static_cast<char*>(st->buf.workspace);
+  Prof prof(st, mode == ATTN_DENSE ? KVE_K_ATTN_DENSE : KVE_K_ATTN, stream);
   cudaError_t e = launch_attn(view(st, layer), mode, ls.n_compacted, ls.n_tokens, plan, q, out, lse, scale,
                               reinterpret_cast<float*>(ws + st->off_partials),
                               reinterpret_cast<int32_t*>(ws + st->off_counters), stream);
@@ -177,6 +199,8 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
 }
 
 int kvE_destroy(kvE_store* st) {
+  if (st && st->ev_made)
+    for (cudaEvent_t e : st->ev) cudaEventDestroy(e);
   delete st;
   return KVE_OK;
 }
@@ -186,6 +210,7 @@ int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, i
   LayerState& ls = st->layers[layer];
   if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   if (n_new > 0) {
+    Prof prof(st, KVE_K_APPEND, static_cast<cudaStream_t>(stream));
     cudaError_t e = launch_append(view(st, layer), k_new, v_new, n_new, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(st, e);
     ls.n_tokens += n_new;
@@ -219,8 +244,13 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
   if (chunk_end == chunk_begin) return KVE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const LayerView v = view(st, layer);
-  cudaError_t e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, s);
+  cudaError_t e;
+  {
+    Prof prof(st, KVE_K_CHUNK_MEAN, s);
+    e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, s);
+  }
   if (e == cudaSuccess && mlp) {
+    Prof prof(st, KVE_K_CHUNK_MLP, s);
     MlpWeights mw;
     mw.W1K = static_cast<const uint16_t*>(w->W1K); mw.W2K = static_cast<const uint16_t*>(w->W2K);
     mw.W1V = static_cast<const uint16_t*>(w->W1V); mw.W2V = static_cast<const uint16_t*>(w->W2V);
@@ -245,11 +275,17 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const LayerView v = view(st, layer);
   float* P = reinterpret_cast<float*>(static_cast<char*>(st->buf.workspace) + st->off_P);
-  cudaError_t e = launch_gate_proj(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_ih), w->b_ih, w->b_hh,
-                                   st->cfg.d_g, P, s);
-  if (e == cudaSuccess)
+  cudaError_t e;
+  {
+    Prof prof(st, KVE_K_GATE_PROJ, s);
+    e = launch_gate_proj(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_ih), w->b_ih, w->b_hh,
+                         st->cfg.d_g, P, s);
+  }
+  if (e == cudaSuccess) {
+    Prof prof(st, KVE_K_GATE_RNN, s);
     e = launch_gate_rnn(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_hh), w->w_s, w->b_s, st->cfg.d_g,
                         P, chunk_begin == 0, s);
+  }
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_gated = chunk_end;
   if (ls.n_compacted > chunk_begin) ls.n_compacted = chunk_begin;   // scores changed under the keep list
@@ -259,6 +295,7 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   if (bad_layer(st, layer)) return KVE_ERR_ARG;
   LayerState& ls = st->layers[layer];
+  Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_compact(view(st, layer), ls.n_gated, tau, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_compacted = ls.n_gated;
@@ -331,6 +368,34 @@ int kvE_layer_state(const kvE_store* st, int layer, int* n_tokens, int* n_summar
   if (n_summarised) *n_summarised = ls.n_summarised;
   if (n_gated) *n_gated = ls.n_gated;
   if (n_compacted) *n_compacted = ls.n_compacted;
+  return KVE_OK;
+}
+
+int kvE_profile(kvE_store* st, int enable) {
+  if (!st) return KVE_ERR_ARG;
+  if (enable && !st->ev_made) {
+    for (cudaEvent_t& e : st->ev) {
+      cudaError_t rc = cudaEventCreate(&e);
+      if (rc != cudaSuccess) return cuda_fail(st, rc);
+    }
+    st->ev_made = true;
+  }
+  st->profiling = enable != 0;
+  for (bool& u : st->ev_used) u = false;
+  return KVE_OK;
+}
+
+int kvE_profile_read(kvE_store* st, float* us) {
+  if (!st || !us) return KVE_ERR_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  for (int k = 0; k < KVE_K_COUNT; ++k) {
+    us[k] = -1.f;
+    if (st->ev_made && st->ev_used[k]) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, st->ev[2 * k], st->ev[2 * k + 1]) == cudaSuccess) us[k] = ms * 1000.f;
+    }
+  }
   return KVE_OK;
 }
 
