@@ -142,6 +142,31 @@ int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* l
 int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse,
                           float scale, void* stream);
 
+/* kvE_decode_attn without any scratch from the caller.  (The paper has no counterpart: this is a
+ * deployment aid.)  Some users of this library must not allocate device memory once they are
+ * running: a robot-control loop that handed the whole GPU to its framework's memory pool at
+ * start-up and may not stall on, or fail in, an allocation between two control ticks; a plug-in that
+ * is given device pointers by a host application and has no right to allocate on that device.  For
+ * them the split-K partial results and tickets of the attention kernel live in a device array that
+ * is part of the library image itself (KVE_STATIC_SCRATCH_BYTES, about 2.1 MiB, held by every GPU that
+ * loads the library until the process exits) instead of the handle's workspace, and this call
+ * performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - same arguments, result and errors as kvE_decode_attn (gated attention of `layer`, mode from
+ *     cfg.attend); q, out: DEVICE bf16 [S][d]; lse: DEVICE fp32 [S] or NULL.
+ *   - limits: S <= KVE_STATIC_MAX_SEQUENCES and S * splits <= KVE_STATIC_MAX_PARTIALS, where splits
+ *     (1..32) is what the library picks for the layer's current length; beyond that the call
+ *     returns KVE_ERR_CAPACITY without launching (text via kvE_last_cuda_error).
+ *   - the first call on each device looks up the array's device address (that device must be
+ *     current); make that first call outside any stream capture.
+ *   - one array per device, shared by every handle and stream: the call clears the tickets it
+ *     needs on `stream` before the kernel, but two calls that overlap on the GPU (different
+ *     streams, or different handles) race on it.  Serialise them, or use kvE_decode_attn. */
+#define KVE_STATIC_MAX_SEQUENCES 2048
+#define KVE_STATIC_MAX_PARTIALS 4096
+#define KVE_STATIC_SCRATCH_BYTES (KVE_STATIC_MAX_SEQUENCES * 4 + KVE_STATIC_MAX_PARTIALS * 132 * 4)
+int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale,
+                           void* stream);
+
 /* One whole decode step of `layer` from HOST memory: copies k_new, v_new, q (bf16 [S][d] each,
  * ideally pinned) to the device, appends the token, brings summaries, gate and keep list up to
  * date for every chunk that has left the window (from scratch if `from_scratch` != 0), runs

@@ -23,7 +23,7 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_decode_attn", "kvE_decode_attn_dense",
-           "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
+           "kvE_decode_attn_static", "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense"]
 
@@ -82,6 +82,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_compact.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_void_p]
     lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
     lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
+    lib.kvE_decode_attn_static.argtypes = lib.kvE_decode_attn.argtypes
     lib.kvE_decode_step_host.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float,
                                          C.c_float, C.c_int, C.c_void_p]
@@ -246,6 +247,9 @@ class Store:
     def decode_attn_dense(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)
 
+    def decode_attn_static(self, layer, q, out=None, lse=None, scale=None, stream=None):
+        return kvE_decode_attn_static(self, layer, q, out, lse, scale, stream)
+
     def decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale=None,
                          from_scratch=False, stream=None):
         kvE_decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale, from_scratch, stream)
@@ -307,6 +311,13 @@ def kvE_decode_attn(st: Store, layer, q, out=None, lse=None, scale=None, stream=
 
 def kvE_decode_attn_dense(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):
     return _attn("kvE_decode_attn_dense", st, layer, q, out, lse, scale, stream)
+
+
+def kvE_decode_attn_static(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):
+    """kvE_decode_attn with the split-K scratch inside the library image (no caller scratch, no
+    allocation inside the call).  `out` is allocated here with torch only when the caller passes none;
+    a caller that must not allocate passes its own."""
+    return _attn("kvE_decode_attn_static", st, layer, q, out, lse, scale, stream)
 
 
 def kvE_decode_step_host(st: Store, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale=None,

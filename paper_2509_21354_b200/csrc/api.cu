@@ -1,6 +1,7 @@
 // Host side of libkve: the C ABI of include/kve.h.  Validates arguments, tracks per-layer progress
 // (tokens stored, chunks summarised / gated / compacted) and enqueues the kernels.  Allocates no
 // device memory.
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -38,6 +39,7 @@ namespace {
 constexpr int MAX_SPLITS = 32;
 constexpr size_t ALIGN = 256;
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+constexpr size_t align_const(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 int check_config(const kvE_config* c) {
   if (!c) return KVE_ERR_ARG;
@@ -402,3 +404,68 @@ int kvE_profile_read(kvE_store* st, float* us) {
 const char* kvE_last_cuda_error(const kvE_store* st) { return st ? st->cuda_error.c_str() : ""; }
 
 }  // extern "C"
+
+// ---- kvE_decode_attn_static: gated attention whose split-K scratch lives inside the library ----------
+// The scratch is a file-scope device array: every GPU that loads the library carries it until the
+// process exits.  In host code `g_static_scratch` is only a stand-in for the symbol, not a device
+// address, so the address the kernel gets is looked up once per device with cudaGetSymbolAddress.
+namespace {
+
+constexpr int STATIC_MAX_SEQ = KVE_STATIC_MAX_SEQUENCES;
+constexpr int STATIC_MAX_REC = KVE_STATIC_MAX_PARTIALS;
+constexpr size_t STATIC_COUNTER_BYTES = align_const(STATIC_MAX_SEQ * sizeof(int32_t));
+constexpr size_t STATIC_BYTES = STATIC_COUNTER_BYTES + (size_t)STATIC_MAX_REC * ATTN_PARTIAL_FLOATS * sizeof(float);
+
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[MAX_DEVICES] = {};
+
+// device address of the scratch on the CURRENT device (looked up on the first call per device)
+cudaError_t static_scratch(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale,
+                                      void* stream) {
+  if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
+  const LayerState& ls = st->layers[layer];
+  const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;
+  const long long rows_upper = (long long)ls.n_compacted * per + (ls.n_tokens - (long long)ls.n_compacted * st->cfg.C);
+  const AttnPlan plan = plan_attention(st, rows_upper);
+  const long long records = (long long)st->S * plan.max_splits;
+  if (st->S > STATIC_MAX_SEQ || records > STATIC_MAX_REC) {
+    st->cuda_error = "kvE_decode_attn_static: " + std::to_string(st->S) + " sequences x " +
+                     std::to_string(plan.max_splits) + " splits exceed the built-in scratch (" +
+                     std::to_string(STATIC_MAX_SEQ) + " sequences, " + std::to_string(STATIC_MAX_REC) +
+                     " partial records); use kvE_decode_attn";
+    return KVE_ERR_CAPACITY;
+  }
+  unsigned char* scratch = nullptr;
+  cudaError_t e = static_scratch(&scratch);
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* counters = reinterpret_cast<int32_t*>(scratch);
+  float* partials = reinterpret_cast<float*>(scratch + STATIC_COUNTER_BYTES);
+  // the array keeps whatever the last call left: the tickets must start at zero
+  e = cudaMemsetAsync(counters, 0, sizeof(int32_t) * (size_t)st->S, s);
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  e = launch_attn(view(st, layer), mode, ls.n_compacted, ls.n_tokens, plan, q, out, lse, scale, partials, counters, s);
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+}
