@@ -6,6 +6,7 @@
 // rounding as a plain sequential loop), divided by C with an IEEE division.
 #include "common.cuh"
 #include "kernels.h"
+#include "umma.cuh"
 
 namespace kve {
 
@@ -176,10 +177,261 @@ __global__ void __launch_bounds__(MLP_THREADS) kve_chunk_mlp_kernel(LayerView v,
   }
 }
 
+// ---- the same MLP on the 5th-generation tensor cores (d_sum a multiple of 64, at most 256) ----------------
+// Both layers are GEMMs over a tile of 128 (sequence, chunk) units:
+//   H = M W1^T  (128 x d_sum, K = 128),   Y = gelu(H + b1) W2^T  (128 x 128, K = d_sum).
+// The left operands (the chunk means, the activations) are fp32.  Each is split exactly into three
+// bf16 planes (x = p0 + p1 + p2), the weights are bf16 by definition, so every product the tensor
+// core forms is exact and the result differs from a plain fp32 loop only in summation order.
+//  * A CTA serves one side (keys or values) and keeps that side's W1 and W2 (64 KB each, K-major,
+//    128-byte swizzle) in shared memory for all its tiles.
+//  * Layer 1: 24 tcgen05.mma (3 planes x K/16) of shape 128 x d_sum accumulate H in tensor memory.
+//  * Layer 2 runs in slices of 64 hidden units: the eight warps read a slice of H from tensor
+//    memory, add b1, apply the erf GELU, split into planes and store them as the next A operand
+//    (double-buffered, 48 KB per slice, in the space the layer-1 planes have left); one thread
+//    issues the slice's 12 MMAs into the second accumulator while the warps prepare the next slice.
+//  * Epilogue: Y + b2 -> fp32 summary and its bf16 rounding.
+// Every mbarrier wait is bounded; on give-up the status word gets KVE_ERR_TIMEOUT.
+constexpr int MT_M = 128;
+constexpr int MT_THREADS = 256;
+constexpr int MT_MAX_DSUM = 256;
+constexpr int MT_PLANE_KB_BYTES = MT_M * umma::KBLOCK_ROW_BYTES;          // 16 KB: one plane, one K-block of 64
+constexpr int MT_SMEM_A = 0;                                              // 96 KB: 3 planes x 2 K-blocks, later 2 x (3 planes x 1)
+constexpr int MT_SMEM_W1 = MT_SMEM_A + 6 * MT_PLANE_KB_BYTES;
+constexpr int MT_SMEM_W2 = MT_SMEM_W1 + MT_MAX_DSUM * D * 2;
+constexpr int MT_SMEM_B1 = MT_SMEM_W2 + D * MT_MAX_DSUM * 2;
+constexpr int MT_SMEM_B2 = MT_SMEM_B1 + MT_MAX_DSUM * 4;
+constexpr int MT_SMEM_BAR = MT_SMEM_B2 + D * 4;
+constexpr int MT_SMEM_BYTES = MT_SMEM_BAR + 64 + 1024;                    // + slack to reach a 1024-byte boundary
+constexpr int MT_TMEM_COLS = 512;                                         // H: columns [0, d_sum), Y: columns [256, 384)
+constexpr int MT_TMEM_Y = 256;
+
+// exact split of an fp32 value into three bf16 pieces: x = p[0] + p[1] + p[2]
+__device__ __forceinline__ void split3_bits(float x, uint32_t (&p)[3]) {
+  p[0] = f32_to_bf16_bits(x);
+  const float r1 = x - __uint_as_float(p[0] << 16);
+  p[1] = f32_to_bf16_bits(r1);
+  const float r2 = r1 - __uint_as_float(p[1] << 16);
+  p[2] = f32_to_bf16_bits(r2);
+}
+
+// splits 8 consecutive fp32 values and stores the three 16-byte pieces at dst + pl * plane_stride
+__device__ __forceinline__ void store_split8(const float (&x)[8], unsigned char* dst, int plane_stride) {
+  uint32_t w[3][4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    uint32_t a[3], b[3];
+    split3_bits(x[2 * e], a);
+    split3_bits(x[2 * e + 1], b);
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) w[pl][e] = a[pl] | (b[pl] << 16);
+  }
+#pragma unroll
+  for (int pl = 0; pl < 3; ++pl)
+    *reinterpret_cast<uint4*>(dst + pl * plane_stride) = make_uint4(w[pl][0], w[pl][1], w[pl][2], w[pl][3]);
+}
+
+__global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerView v, int t0, int n_range, long long n_units,
+                                                                         MlpWeights w, int d_sum) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* As = smem + MT_SMEM_A;
+  unsigned char* W1s = smem + MT_SMEM_W1;
+  unsigned char* W2s = smem + MT_SMEM_W2;
+  float* b1s = reinterpret_cast<float*>(smem + MT_SMEM_B1);
+  float* b2s = reinterpret_cast<float*>(smem + MT_SMEM_B2);
+  uint64_t* bar_h = reinterpret_cast<uint64_t*>(smem + MT_SMEM_BAR);       // layer-1 MMAs done
+  uint64_t* bar_buf = bar_h + 1;                                            // [2]: slice MMAs that read buffer b done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + MT_SMEM_BAR + 32);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int side = blockIdx.y;
+  const uint16_t* W1 = side ? w.W1V : w.W1K;
+  const uint16_t* W2 = side ? w.W2V : w.W2K;
+  const float* b1 = side ? w.b1V : w.b1K;
+  const float* b2 = side ? w.b2V : w.b2K;
+  float* sum_f32 = side ? v.vsum_f32 : v.ksum_f32;
+  uint16_t* sum_b16 = side ? v.vsum_bf16 : v.ksum_bf16;
+  const int n_slices = d_sum / 64;
+  const long long n_tiles = (n_units + MT_M - 1) / MT_M;
+
+  // ---- one-time set-up -----------------------------------------------------------------------------
+  for (int i = tid; i < d_sum * 16; i += MT_THREADS) {              // W1 [d_sum][128]: rows of 16 pieces, 2 K-blocks
+    const int r = i >> 4, p = i & 15;
+    const uint4 val = __ldg(reinterpret_cast<const uint4*>(W1 + (long long)r * D) + p);
+    *reinterpret_cast<uint4*>(W1s + (p >> 3) * (d_sum * umma::KBLOCK_ROW_BYTES) + umma::piece_offset(r, p & 7)) = val;
+  }
+  const int w2_pieces = d_sum / 8;
+  for (int i = tid; i < D * w2_pieces; i += MT_THREADS) {           // W2 [128][d_sum]: n_slices K-blocks of 16 KB
+    const int r = i / w2_pieces, p = i - r * w2_pieces;
+    const uint4 val = __ldg(reinterpret_cast<const uint4*>(W2 + (long long)r * d_sum) + p);
+    *reinterpret_cast<uint4*>(W2s + (p >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, p & 7)) = val;
+  }
+  for (int i = tid; i < d_sum; i += MT_THREADS) b1s[i] = b1[i];
+  for (int i = tid; i < D; i += MT_THREADS) b2s[i] = b2[i];
+  if (warp == 0) umma::tmem_alloc(tmem_slot, MT_TMEM_COLS);
+  if (tid == 0) {
+    mbar_init(bar_h, 1);
+    mbar_init(&bar_buf[0], 1);
+    mbar_init(&bar_buf[1], 1);
+    mbar_fence_init();
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+  const uint32_t tmem_h = *tmem_slot, tmem_y = tmem_h + MT_TMEM_Y;
+  const uint32_t idesc1 = umma::instr_desc_bf16(MT_M, d_sum), idesc2 = umma::instr_desc_bf16(MT_M, D);
+  const uint32_t a_base = smem_u32(As), w1_base = smem_u32(W1s), w2_base = smem_u32(W2s);
+  const int lg = warp & 3, half = warp >> 2;
+  const int row_in_tile = lg * 32 + lane;
+  const uint32_t tmem_lane = (uint32_t)(lg * 32) << 16;
+
+  uint32_t ph_h = 0, ph_buf[2] = {0, 0};
+  bool failed = false;
+  for (long long tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
+    const long long unit0 = tile * MT_M;
+    // ---- chunk means -> three bf16 planes (layer-1 A operand) ------------------------------------------
+#pragma unroll 2
+    for (int i = tid; i < MT_M * 16; i += MT_THREADS) {
+      const int r = i >> 4, pc = i & 15;
+      const long long unit = unit0 + r;
+      float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (unit < n_units) {
+        const int s = (int)(unit / n_range);
+        const int t = t0 + (int)(unit - (long long)s * n_range);
+        const float4* src = reinterpret_cast<const float4*>(sum_f32 + ((long long)s * v.max_chunks + t) * D + pc * 8);
+        const float4 a = src[0], b = src[1];
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+      }
+      // plane pl, K-block kb at (pl * 2 + kb) * 16 KB
+      store_split8(x, As + (pc >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, pc & 7), 2 * MT_PLANE_KB_BYTES);
+    }
+    umma::fence_smem_to_async();
+    __syncthreads();
+    if (tid == 0) {
+      umma::fence_after_sync();
+      bool acc = false;
+#pragma unroll 1
+      for (int pl = 2; pl >= 0; --pl)                 // smallest plane first
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            umma::mma_bf16(tmem_h, umma::smem_desc(a_base + (pl * 2 + kb) * MT_PLANE_KB_BYTES + k * 32),
+                           umma::smem_desc(w1_base + kb * (d_sum * umma::KBLOCK_ROW_BYTES) + k * 32), idesc1, acc);
+            acc = true;
+          }
+      umma::commit(bar_h);
+    }
+    {
+      const bool ok = mbar_wait_bounded(bar_h, ph_h);
+      ph_h ^= 1;
+      if (__syncthreads_or(!ok)) { failed = true; break; }
+    }
+    umma::fence_after_sync();
+
+    // ---- layer 2 in slices of 64 hidden units ------------------------------------------------------------
+    for (int j = 0; j < n_slices; ++j) {
+      const int buf = j & 1;
+      if (j >= 2) {        // the MMAs of slice j - 2 still read this buffer
+        const bool ok = mbar_wait_bounded(&bar_buf[buf], ph_buf[buf]);
+        ph_buf[buf] ^= 1;
+        if (__syncthreads_or(!ok)) { failed = true; break; }
+      }
+      float h[32];
+      umma::tmem_ld32(tmem_h + tmem_lane + (uint32_t)(j * 64 + half * 32), h);
+      unsigned char* abuf = As + buf * 3 * MT_PLANE_KB_BYTES;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float g[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) g[e] = gelu_erf(h[q * 8 + e] + b1s[j * 64 + half * 32 + q * 8 + e]);
+        store_split8(g, abuf + umma::piece_offset(row_in_tile, half * 4 + q), MT_PLANE_KB_BYTES);
+      }
+      umma::fence_smem_to_async();
+      umma::fence_before_sync();
+      __syncthreads();
+      if (tid == 0) {
+        umma::fence_after_sync();
+        const uint32_t ab = a_base + buf * 3 * MT_PLANE_KB_BYTES;
+#pragma unroll 1
+        for (int pl = 2; pl >= 0; --pl)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma::mma_bf16(tmem_y, umma::smem_desc(ab + pl * MT_PLANE_KB_BYTES + k * 32),
+                           umma::smem_desc(w2_base + j * MT_PLANE_KB_BYTES + k * 32), idesc2, !(j == 0 && pl == 2 && k == 0));
+        umma::commit(&bar_buf[buf]);
+      }
+    }
+    if (failed) break;
+    // drain: one outstanding commit per buffer that was used (the later one covers every MMA before it)
+    {
+      bool ok = true;
+      const int first = (n_slices >= 2) ? (n_slices & 1) : 0;     // older buffer first
+      for (int u = 0; u < (n_slices >= 2 ? 2 : 1); ++u) {
+        const int b = (first + u) & 1;
+        ok = mbar_wait_bounded(&bar_buf[b], ph_buf[b]) && ok;
+        ph_buf[b] ^= 1;
+      }
+      if (__syncthreads_or(!ok)) { failed = true; break; }
+    }
+    umma::fence_after_sync();
+
+    // ---- epilogue: Y + b2 -> fp32 summary and its bf16 rounding ----------------------------------------------
+    {
+      const long long unit = unit0 + row_in_tile;
+      long long o = 0;
+      if (unit < n_units) {
+        const int s = (int)(unit / n_range);
+        const int t = t0 + (int)(unit - (long long)s * n_range);
+        o = ((long long)s * v.max_chunks + t) * D;
+      }
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {
+        const int c = half * 64 + cc * 32;
+        float y[32];
+        umma::tmem_ld32(tmem_y + tmem_lane + (uint32_t)c, y);
+        if (unit < n_units) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) y[e] += b2s[c + e];
+          float4* df = reinterpret_cast<float4*>(sum_f32 + o + c);
+          uint4* db = reinterpret_cast<uint4*>(sum_b16 + o + c);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) df[e] = make_float4(y[4 * e], y[4 * e + 1], y[4 * e + 2], y[4 * e + 3]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            db[e] = make_uint4(pack_bf16x2(y[8 * e], y[8 * e + 1]), pack_bf16x2(y[8 * e + 2], y[8 * e + 3]),
+                               pack_bf16x2(y[8 * e + 4], y[8 * e + 5]), pack_bf16x2(y[8 * e + 6], y[8 * e + 7]));
+        }
+      }
+    }
+    umma::fence_before_sync();
+    __syncthreads();     // accumulators and operand space are free for the next tile
+  }
+  if (failed && tid == 0) set_status(v.status, ERR_TIMEOUT);
+
+  umma::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) umma::tmem_dealloc(tmem_h, MT_TMEM_COLS);
+}
+
 cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st) {
   const int n_range = t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
+  if (d_sum % 64 == 0 && d_sum <= MT_MAX_DSUM) {
+    static bool attr_tc = false;
+    if (!attr_tc) {
+      cudaError_t e = cudaFuncSetAttribute(kve_chunk_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MT_SMEM_BYTES);
+      if (e != cudaSuccess) return e;
+      attr_tc = true;
+    }
+    const long long n_tiles = (n_units + MT_M - 1) / MT_M;
+    const long long per_side = n_tiles < 74 ? n_tiles : 74;      // one CTA per SM: half of the 148 SMs per side
+    dim3 grid((unsigned)per_side, 2);
+    kve_chunk_mlp_tc_kernel<<<grid, MT_THREADS, MT_SMEM_BYTES, st>>>(v, t0, n_range, n_units, w, d_sum);
+    return cudaGetLastError();
+  }
   const size_t smem = sizeof(float) * (size_t)MLP_ROWS * (D + d_sum);
   static bool attr_set = false;
   if (!attr_set) {
