@@ -10,13 +10,22 @@
 //  * Per step the CTA computes its rows of W_hh h for all its sequences with warp-level tensor-core
 //    MMAs (m16n8k16, bf16 x bf16 -> fp32).  W_hh is bf16 by definition; the fp32 state h is split
 //    exactly into three bf16 planes (h = hi + mid + lo), so the products are exact and only the
-//    accumulation order differs from a plain fp32 loop.
+//    accumulation order differs from a plain fp32 loop.  Each plane has its own accumulators
+//    (three times as many independent MMA chains), added smallest plane first at the end.
 //  * MMA rows are ordered so that one thread ends up holding the i, f, g, o pre-activations of the
 //    same (hidden unit, sequence): the cell update is thread-local, c lives in registers.
-//  * New h values are split into planes and stored into the shared memory of every CTA of the
-//    cluster (distributed shared memory, double-buffered), one cluster barrier per step.
-//  * Per-warp partial dot products of the score head go to CTA 0 of the cluster, which adds them in a
-//    fixed order (deterministic) and writes s_t.
+//  * Exchange of h_t: a warp gathers the planes of its 8 hidden units in a small staging area of
+//    its own, then 16-byte st.async stores (one per plane, sequence and destination CTA) put them
+//    into the double-buffered h planes of every CTA of the cluster.  Each store counts its bytes
+//    on an mbarrier of the receiving CTA, so a step costs one one-way transfer and no
+//    cluster-wide barrier.  A CTA can only be sent step t+1 data after it has itself sent step t
+//    data, i.e. after all its warps have finished reading the buffer that is being overwritten.
+//  * Per-warp partial dot products of the score head travel the same way to CTA 0 of the cluster,
+//    whose warps add them in a fixed order (deterministic) one step later, in the shadow of the
+//    next step's MMAs, and write s_t.
+//  * P_{t+1} is fetched into registers while step t computes.
+// Every mbarrier wait is bounded (one second); on give-up the status word gets KVE_ERR_TIMEOUT and
+// the CTA stops sending, which lets its peers run into their own limits and leave as well.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -34,6 +43,7 @@ struct RnnArgs {
   float* scores;           // [S][max_chunks]
   float* lstm_h;           // [S][d_g]
   float* lstm_c;
+  int32_t* status;
   int S, max_chunks, t0, n_range, reset;
 };
 
@@ -47,11 +57,41 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t ran
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t val) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(val) : "memory");
+// stores into the shared memory of a CTA of the cluster (address from mapa) that count their bytes
+// on an mbarrier of the same CTA when they land
+__device__ __forceinline__ void st_async_u32(uint32_t addr, uint32_t val, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];" ::"r"(addr), "r"(val),
+               "r"(bar)
+               : "memory");
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float val) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(val) : "memory");
+__device__ __forceinline__ void st_async_v4(uint32_t addr, const uint4& v, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.u32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+               "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded: gives up one second after the quick polls ran out, then false
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_t parity) {
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+  unsigned long long t_start, t_now;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_start));
+  do {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    __nanosleep(128);
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_now));
+  } while (t_now - t_start < 1000000000ull);
+  return false;
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -77,19 +117,37 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   constexpr int KT = DG / 16;            // k tiles
   constexpr int NS = 8 * NT;             // sequences per cluster
   constexpr int LDH = DG + 8;            // padded plane row (bf16 elements): conflict-free B fragments
+  constexpr int HS_BUF = RNN_PLANES * NS * LDH;                 // bf16 elements per h buffer
+  constexpr int STG_WARP = RNN_PLANES * NS * UW;                // bf16 elements of one warp's staging area
+  constexpr int N_PIECES = RNN_PLANES * NS * MP;                // 16-byte pieces a warp sends to each CTA per step
+  constexpr uint32_t H_BYTES = RNN_PLANES * NS * DG * 2;        // bytes of h planes a CTA receives per step
+  constexpr uint32_t SP_BYTES = CL * RNN_WARPS * NS * 4;        // bytes of score partials CTA 0 receives per step
+  constexpr int OFF_SPART = 2 * HS_BUF * 2;
+  constexpr int OFF_STAGE = OFF_SPART + 2 * NS * 32 * 4;
+  constexpr int OFF_BARS = OFF_STAGE + RNN_WARPS * STG_WARP * 2;
   static_assert(UW % 8 == 0 && MP >= 1, "8 warps x 8k hidden units per CTA");
   static_assert(CL * RNN_WARPS <= 32, "score partials fit one warp");
+  static_assert(OFF_SPART % 16 == 0 && OFF_STAGE % 16 == 0 && OFF_BARS % 16 == 0 && (LDH * 2) % 16 == 0, "16-byte pieces");
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                                   // [2][PLANES][NS][LDH]
-  float* spart = reinterpret_cast<float*>(smem_raw + 2 * RNN_PLANES * NS * LDH * 2);      // [2][NS][32]
-  constexpr int HS_BUF = RNN_PLANES * NS * LDH;   // elements per buffer
+  uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                          // [2][PLANES][NS][LDH]
+  float* spart = reinterpret_cast<float*>(smem_raw + OFF_SPART);                 // [2][NS][32]
+  uint16_t* stage = reinterpret_cast<uint16_t*>(smem_raw + OFF_STAGE);           // [warps][PLANES][NS][UW]
+  uint64_t* hbar = reinterpret_cast<uint64_t*>(smem_raw + OFF_BARS);             // [2] h planes landed
+  uint64_t* sbar = hbar + 2;                                                     // [2] score partials landed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tig = lane & 3;
   const uint32_t rank = cluster_rank();
   const int cid = blockIdx.x / CL;
   const int seq0 = cid * NS;
+  uint16_t* my_stage = stage + warp * STG_WARP;
+
+  if (tid == 0) {
+    mbar_init(&hbar[0], 1); mbar_init(&hbar[1], 1);
+    mbar_init(&sbar[0], 1); mbar_init(&sbar[1], 1);
+    mbar_fence_init();
+  }
 
   // ---- W_hh rows of this CTA as A fragments, resident in registers --------------------------------
   uint32_t A[2 * MP][KT][4];
@@ -108,8 +166,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
 #pragma unroll
   for (int p = 0; p < MP; ++p) wsu[p] = a.w_s[(int)rank * HU + warp * UW + p * 8 + g];
 
-  // ---- initial state ---------------------------------------------------------------------------
-  // every CTA needs the full h of its sequences (all d_g units) as planes in buffer 0
+  // ---- initial state: every CTA needs the full h of its sequences as planes in buffer 0 -------------
   for (int i = tid; i < NS * (DG / 2); i += RNN_THREADS) {
     const int j = i / (DG / 2), k2 = i % (DG / 2);
     const int s = seq0 + j;
@@ -138,14 +195,79 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         c[p][nt][e] = live ? a.lstm_c[(long long)s * DG + ug] : 0.f;
         hlast[p][nt][e] = live ? a.lstm_h[(long long)s * DG + ug] : 0.f;
       }
-  // all CTAs of the cluster are running and have filled buffer 0 before anyone writes remotely
-  cluster_sync_all();
+
+  // addresses in the other CTAs that do not change from step to step
+  uint32_t hbar_remote[CL], hs_remote[CL];
+#pragma unroll
+  for (int r = 0; r < CL; ++r) {
+    hbar_remote[r] = map_to_rank(smem_u32(&hbar[0]), r);
+    hs_remote[r] = map_to_rank(smem_u32(hs), r);
+  }
+  const uint32_t sbar_remote0 = map_to_rank(smem_u32(&sbar[0]), 0);
+  const uint32_t spart_remote0 = map_to_rank(smem_u32(spart), 0);
 
   const int n_cols = 4 * DG;
+  float pin[MP][NT][4][2];     // P of the current step
+#pragma unroll
+  for (int p = 0; p < MP; ++p)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int s = seq0 + nt * 8 + tig * 2 + e;
+        const int ug = (int)rank * HU + warp * UW + p * 8 + g;
+        const float* prow = a.P + ((long long)s * a.n_range) * n_cols + ug;
+#pragma unroll
+        for (int gate = 0; gate < 4; ++gate) pin[p][nt][gate][e] = (s < a.S) ? __ldcs(prow + gate * DG) : 0.f;
+      }
+
+  // barriers initialised and buffer 0 filled in every CTA before anyone sends
+  cluster_sync_all();
+
+  bool alive = true;
   for (int step = 0; step < a.n_range; ++step) {
     const int buf = step & 1;
-    // ---- P_t for this thread's (unit, gate, sequence) entries; prefetch P_{t+1} into L2 ----------
-    float pin[MP][NT][4][2];
+    const bool send_h = step + 1 < a.n_range;
+    // this step's sends of the cluster land in buffer buf^1: announce the bytes
+    if (tid == 0 && send_h) mbar_arrive_expect_tx(&hbar[buf ^ 1], H_BYTES);
+    if (tid == 0 && rank == 0) mbar_arrive_expect_tx(&sbar[buf], SP_BYTES);
+    if (step > 0) {
+      // h_{t-1} from every CTA of the cluster (each buffer completes once per two steps)
+      if (!mbar_wait_cluster_bounded(&hbar[buf], ((step - 1) >> 1) & 1)) {
+        if (lane == 0) set_status(a.status, ERR_TIMEOUT);
+        alive = false;
+      }
+      if (!__all_sync(0xffffffffu, alive)) alive = false;
+      if (!alive) break;
+    }
+
+    // ---- W_hh h_{t-1} on the tensor cores: one accumulator set per plane ---------------------------
+    float acc[RNN_PLANES][2 * MP][NT][4];
+#pragma unroll
+    for (int pl = 0; pl < RNN_PLANES; ++pl)
+#pragma unroll
+      for (int mt = 0; mt < 2 * MP; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[pl][mt][nt][e] = 0.f;
+    const uint16_t* hb = hs + buf * HS_BUF;
+#pragma unroll
+    for (int kt = 0; kt < KT; ++kt) {
+#pragma unroll
+      for (int pl = 0; pl < RNN_PLANES; ++pl) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const uint32_t* brow = reinterpret_cast<const uint32_t*>(hb + (pl * NS + nt * 8 + g) * LDH + kt * 16);
+          const uint32_t b0 = brow[tig], b1 = brow[4 + tig];
+#pragma unroll
+          for (int mt = 0; mt < 2 * MP; ++mt) mma_bf16_16816(acc[pl][mt][nt], A[mt][kt], b0, b1);
+        }
+      }
+    }
+
+    // ---- P_{t+1} into registers while the MMAs drain ----------------------------------------------------
+    float pnext[MP][NT][4][2];
 #pragma unroll
     for (int p = 0; p < MP; ++p)
 #pragma unroll
@@ -154,81 +276,77 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         for (int e = 0; e < 2; ++e) {
           const int s = seq0 + nt * 8 + tig * 2 + e;
           const int ug = (int)rank * HU + warp * UW + p * 8 + g;
-          const float* prow = a.P + ((long long)s * a.n_range + step) * n_cols + ug;
+          const bool live = s < a.S && send_h;
+          const float* prow = a.P + ((long long)s * a.n_range + step + 1) * n_cols + ug;
 #pragma unroll
-          for (int gate = 0; gate < 4; ++gate) pin[p][nt][gate][e] = (s < a.S) ? __ldcs(prow + gate * DG) : 0.f;
-          if (s < a.S && step + 1 < a.n_range) {
-#pragma unroll
-            for (int gate = 0; gate < 4; ++gate)
-              asm volatile("prefetch.global.L2 [%0];" ::"l"(prow + n_cols + gate * DG));
-          }
+          for (int gate = 0; gate < 4; ++gate) pnext[p][nt][gate][e] = live ? __ldcs(prow + gate * DG) : 0.f;
         }
 
-    // ---- W_hh h_{t-1} on the tensor cores ---------------------------------------------------------
-    float acc[2 * MP][NT][4];
-#pragma unroll
-    for (int mt = 0; mt < 2 * MP; ++mt)
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
-    const uint16_t* hb = hs + buf * HS_BUF;
-#pragma unroll
-    for (int kt = 0; kt < KT; ++kt) {
-#pragma unroll
-      for (int pl = RNN_PLANES - 1; pl >= 0; --pl) {     // smallest plane first
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          const uint32_t* brow = reinterpret_cast<const uint32_t*>(hb + (pl * NS + nt * 8 + g) * LDH + kt * 16);
-          const uint32_t b0 = brow[tig], b1 = brow[4 + tig];
-#pragma unroll
-          for (int mt = 0; mt < 2 * MP; ++mt) mma_bf16_16816(acc[mt][nt], A[mt][kt], b0, b1);
+    // ---- CTA 0: score of the previous step (its partials landed while this step's MMAs ran) ---------------
+    if (rank == 0 && step > 0) {
+      const int pb = buf ^ 1;
+      if (!mbar_wait_cluster_bounded(&sbar[pb], ((step - 1) >> 1) & 1)) {
+        if (lane == 0) set_status(a.status, ERR_TIMEOUT);
+      }
+      for (int j = warp; j < NS; j += RNN_WARPS) {
+        float vsum = (lane < CL * RNN_WARPS) ? spart[(pb * NS + j) * 32 + lane] : 0.f;
+        vsum = warp_sum(vsum);
+        const int s = seq0 + j;
+        if (lane == 0 && s < a.S) {
+          const float z = vsum + a.b_s;
+          a.scores[(long long)s * a.max_chunks + a.t0 + step - 1] = 1.f / (1.f + expf(-z));
         }
       }
     }
 
-    // ---- cell update (thread-local), h exchange, score partials ----------------------------------
+    // ---- cell update (thread-local), planes of h_t into the warp's staging area ---------------------
     float spv[NT][2];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) spv[nt][0] = spv[nt][1] = 0.f;
-    uint16_t* hn = hs + (buf ^ 1) * HS_BUF;
+    __syncwarp();      // the previous step's pieces have been read out of the staging area
 #pragma unroll
     for (int p = 0; p < MP; ++p) {
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        float hv[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const float ig = fast_sigmoid(acc[2 * p][nt][e] + pin[p][nt][0][e]);
-          const float fg = fast_sigmoid(acc[2 * p][nt][2 + e] + pin[p][nt][1][e]);
-          const float gg = fast_tanh(acc[2 * p + 1][nt][e] + pin[p][nt][2][e]);
-          const float og = fast_sigmoid(acc[2 * p + 1][nt][2 + e] + pin[p][nt][3][e]);
+          float pre[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {   // q: 0 = i, 1 = f (tile 2p, rows g / g+8), 2 = g, 3 = o (tile 2p+1)
+            const int mt = 2 * p + (q >> 1), ai = (q & 1) * 2 + e;
+            pre[q] = ((acc[2][mt][nt][ai] + acc[1][mt][nt][ai]) + acc[0][mt][nt][ai]) + pin[p][nt][q][e];
+          }
+          const float ig = fast_sigmoid(pre[0]);
+          const float fg = fast_sigmoid(pre[1]);
+          const float gg = fast_tanh(pre[2]);
+          const float og = fast_sigmoid(pre[3]);
           const float cn = fmaf(fg, c[p][nt][e], ig * gg);
           c[p][nt][e] = cn;
-          hv[e] = og * fast_tanh(cn);
-          hlast[p][nt][e] = hv[e];
-          spv[nt][e] = fmaf(wsu[p], hv[e], spv[nt][e]);
-        }
-        // pair up neighbouring units (g even / odd) so each thread stores 2 units of one sequence
-        const bool odd = g & 1;
-        const float other = __shfl_xor_sync(0xffffffffu, odd ? hv[0] : hv[1], 4);
-        const float lo_unit = odd ? other : hv[0];
-        const float hi_unit = odd ? hv[1] : other;
-        const int j = nt * 8 + tig * 2 + (odd ? 1 : 0);
-        const int k = (int)rank * HU + warp * UW + p * 8 + (g & ~1);
-        uint32_t pl0[3], pl1[3];
-        split3(lo_unit, pl0);
-        split3(hi_unit, pl1);
+          const float hv = og * fast_tanh(cn);
+          hlast[p][nt][e] = hv;
+          spv[nt][e] = fmaf(wsu[p], hv, spv[nt][e]);
+          if (send_h) {
+            uint32_t pl3[3];
+            split3(hv, pl3);
+            const int j = nt * 8 + tig * 2 + e;
 #pragma unroll
-        for (int pl = 0; pl < RNN_PLANES; ++pl) {
-          const uint32_t word = pl0[pl] | (pl1[pl] << 16);
-          const uint32_t local = smem_u32(hn + (pl * NS + j) * LDH + k);
-#pragma unroll
-          for (int r = 0; r < CL; ++r) st_cluster_u32(map_to_rank(local, r), word);
+            for (int pl = 0; pl < RNN_PLANES; ++pl) my_stage[(pl * NS + j) * UW + p * 8 + g] = (uint16_t)pl3[pl];
+          }
         }
       }
     }
-    // reduce score partials over the 8 units of the warp's lane groups (lanes differ in g)
+    // ---- 16-byte pieces (plane, sequence, 8 units) to every CTA of the cluster -----------------------------
+    if (send_h) {
+      __syncwarp();
+      for (int idx = lane; idx < N_PIECES; idx += 32) {
+        const int row = idx / MP, p = idx - row * MP;          // row = pl * NS + j
+        const uint4 val = *reinterpret_cast<const uint4*>(my_stage + row * UW + p * 8);
+        const uint32_t off = (uint32_t)(((buf ^ 1) * HS_BUF + row * LDH + (int)rank * HU + warp * UW + p * 8) * 2);
+#pragma unroll
+        for (int r = 0; r < CL; ++r) st_async_v4(hs_remote[r] + off, val, hbar_remote[r] + (buf ^ 1) * 8);
+      }
+    }
+    // score partials over the 8 units of the warp's lane groups (lanes differ in g) -> CTA 0
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -239,21 +357,34 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         vsum += __shfl_xor_sync(0xffffffffu, vsum, 16);
         if (g == 0) {
           const int j = nt * 8 + tig * 2 + e;
-          const uint32_t local = smem_u32(spart + (buf * NS + j) * 32 + (int)rank * RNN_WARPS + warp);
-          st_cluster_f32(map_to_rank(local, 0), vsum);
+          const uint32_t off = (uint32_t)(((buf * NS + j) * 32 + (int)rank * RNN_WARPS + warp) * 4);
+          st_async_u32(spart_remote0 + off, __float_as_uint(vsum), sbar_remote0 + buf * 8);
         }
       }
 
-    cluster_sync_all();   // h_t planes and score partials are visible everywhere
+#pragma unroll
+    for (int p = 0; p < MP; ++p)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) pin[p][nt][q][e] = pnext[p][nt][q][e];
+  }
 
-    if (rank == 0) {
+  // ---- CTA 0: score of the last step ------------------------------------------------------------------
+  if (rank == 0 && alive && a.n_range > 0) {
+    const int pb = (a.n_range - 1) & 1;
+    if (!mbar_wait_cluster_bounded(&sbar[pb], ((a.n_range - 1) >> 1) & 1)) {
+      if (lane == 0) set_status(a.status, ERR_TIMEOUT);
+    } else {
       for (int j = warp; j < NS; j += RNN_WARPS) {
-        float vsum = (lane < CL * RNN_WARPS) ? spart[(buf * NS + j) * 32 + lane] : 0.f;
+        float vsum = (lane < CL * RNN_WARPS) ? spart[(pb * NS + j) * 32 + lane] : 0.f;
         vsum = warp_sum(vsum);
         const int s = seq0 + j;
         if (lane == 0 && s < a.S) {
           const float z = vsum + a.b_s;
-          a.scores[(long long)s * a.max_chunks + a.t0 + step] = 1.f / (1.f + expf(-z));
+          a.scores[(long long)s * a.max_chunks + a.t0 + a.n_range - 1] = 1.f / (1.f + expf(-z));
         }
       }
     }
@@ -268,17 +399,19 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       for (int e = 0; e < 2; ++e) {
         const int s = seq0 + nt * 8 + tig * 2 + e;
         const int ug = (int)rank * HU + warp * UW + p * 8 + g;
-        if (s < a.S) {
+        if (s < a.S && alive) {
           a.lstm_c[(long long)s * DG + ug] = c[p][nt][e];
           a.lstm_h[(long long)s * DG + ug] = hlast[p][nt][e];
         }
       }
+  // nobody leaves while a peer may still be sending into its shared memory
+  cluster_sync_all();
 }
 
 template <int DG, int CL, int NT>
 static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
   constexpr int NS = 8 * NT;
-  constexpr int smem = 2 * RNN_PLANES * NS * (DG + 8) * 2 + 2 * NS * 32 * 4;
+  constexpr int smem = 2 * RNN_PLANES * NS * (DG + 8) * 2 + 2 * NS * 32 * 4 + RNN_PLANES * NS * (DG / CL) * 2 + 4 * 8;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kve_gate_rnn_kernel<DG, CL, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -295,7 +428,7 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
   if (t1 <= t0 || v.S <= 0) return cudaSuccess;
   RnnArgs a;
   a.P = P; a.W_hh = W_hh; a.w_s = w_s; a.b_s = b_s;
-  a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c;
+  a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c; a.status = v.status;
   a.S = v.S; a.max_chunks = v.max_chunks; a.t0 = t0; a.n_range = t1 - t0; a.reset = reset_state ? 1 : 0;
   // 16 sequences per cluster once 8 per cluster would need more than one wave of clusters
   switch (d_g) {
