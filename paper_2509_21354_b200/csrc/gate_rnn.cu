@@ -16,13 +16,14 @@
 //    same (hidden unit, sequence): the cell update is thread-local, c lives in registers.
 //  * Exchange of h_t: a warp gathers the planes of its 8 hidden units in a small staging area of
 //    its own, then 16-byte st.async stores (one per plane, sequence and destination CTA) put them
-//    into the double-buffered h planes of every CTA of the cluster.  Each store counts its bytes
-//    on an mbarrier of the receiving CTA, so a step costs one one-way transfer and no
+//    into the double-buffered h planes of every other CTA of the cluster (the own copy is a plain
+//    store followed by a local arrive).  Each remote store counts its bytes on an mbarrier of the
+//    receiving CTA, so a step costs one one-way transfer and no
 //    cluster-wide barrier.  A CTA can only be sent step t+1 data after it has itself sent step t
 //    data, i.e. after all its warps have finished reading the buffer that is being overwritten.
-//  * Per-warp partial dot products of the score head travel the same way to CTA 0 of the cluster,
-//    whose warps add them in a fixed order (deterministic) one step later, in the shadow of the
-//    next step's MMAs, and write s_t.
+//  * The score head is not part of the chain: h_t is stored into the (already consumed) gate-0
+//    slot of row (s, t) of P, and a second, fully parallel kernel computes
+//    s_t = sigmoid(w_s . h_t + b_s) for all (s, t) afterwards, with a fixed summation order.
 //  * P_{t+1} is fetched into registers while step t computes.
 // Every mbarrier wait is bounded (one second); on give-up the status word gets KVE_ERR_TIMEOUT and
 // the CTA stops sending, which lets its peers run into their own limits and leave as well.
@@ -36,9 +37,9 @@ constexpr int RNN_THREADS = RNN_WARPS * 32;
 constexpr int RNN_PLANES = 3;
 
 struct RnnArgs {
-  const float* P;          // [S * n_range][4 d_g]
+  float* P;                // [S * n_range][4 d_g]; columns [0, d_g) of row (s, t) receive h_t once P_t is consumed
   const uint16_t* W_hh;    // bf16 [4 d_g][d_g]
-  const float* w_s;        // [d_g]
+  const float* w_s;        // [d_g] (score kernel)
   float b_s;
   float* scores;           // [S][max_chunks]
   float* lstm_h;           // [S][d_g]
@@ -99,6 +100,13 @@ __device__ __forceinline__ void cluster_sync_all() {
 
 __device__ __forceinline__ float fast_sigmoid(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
 __device__ __forceinline__ float fast_tanh(float x) { return 2.f * fast_sigmoid(2.f * x) - 1.f; }
+// four 8 x 8 b16 blocks of shared memory as mma fragments (lane l gives the address of row l & 7 of block l >> 3)
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
 
 // exact 3-way split of an fp32 value into bf16 pieces: x = p0 + p1 + p2
 __device__ __forceinline__ void split3(float x, uint32_t (&p)[3]) {
@@ -120,21 +128,16 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   constexpr int HS_BUF = RNN_PLANES * NS * LDH;                 // bf16 elements per h buffer
   constexpr int STG_WARP = RNN_PLANES * NS * UW;                // bf16 elements of one warp's staging area
   constexpr int N_PIECES = RNN_PLANES * NS * MP;                // 16-byte pieces a warp sends to each CTA per step
-  constexpr uint32_t H_BYTES = RNN_PLANES * NS * DG * 2;        // bytes of h planes a CTA receives per step
-  constexpr uint32_t SP_BYTES = CL * RNN_WARPS * NS * 4;        // bytes of score partials CTA 0 receives per step
-  constexpr int OFF_SPART = 2 * HS_BUF * 2;
-  constexpr int OFF_STAGE = OFF_SPART + 2 * NS * 32 * 4;
+  constexpr uint32_t H_BYTES = RNN_PLANES * NS * (DG - HU) * 2; // bytes of h planes a CTA receives from its peers per step
+  constexpr int OFF_STAGE = 2 * HS_BUF * 2;
   constexpr int OFF_BARS = OFF_STAGE + RNN_WARPS * STG_WARP * 2;
   static_assert(UW % 8 == 0 && MP >= 1, "8 warps x 8k hidden units per CTA");
-  static_assert(CL * RNN_WARPS <= 32, "score partials fit one warp");
-  static_assert(OFF_SPART % 16 == 0 && OFF_STAGE % 16 == 0 && OFF_BARS % 16 == 0 && (LDH * 2) % 16 == 0, "16-byte pieces");
+  static_assert(OFF_STAGE % 16 == 0 && OFF_BARS % 16 == 0 && (LDH * 2) % 16 == 0, "16-byte pieces");
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                          // [2][PLANES][NS][LDH]
-  float* spart = reinterpret_cast<float*>(smem_raw + OFF_SPART);                 // [2][NS][32]
   uint16_t* stage = reinterpret_cast<uint16_t*>(smem_raw + OFF_STAGE);           // [warps][PLANES][NS][UW]
   uint64_t* hbar = reinterpret_cast<uint64_t*>(smem_raw + OFF_BARS);             // [2] h planes landed
-  uint64_t* sbar = hbar + 2;                                                     // [2] score partials landed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tig = lane & 3;
@@ -144,8 +147,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   uint16_t* my_stage = stage + warp * STG_WARP;
 
   if (tid == 0) {
-    mbar_init(&hbar[0], 1); mbar_init(&hbar[1], 1);
-    mbar_init(&sbar[0], 1); mbar_init(&sbar[1], 1);
+    mbar_init(&hbar[0], 1 + RNN_WARPS); mbar_init(&hbar[1], 1 + RNN_WARPS);
     mbar_fence_init();
   }
 
@@ -162,9 +164,6 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       for (int kt = 0; kt < KT; ++kt) A[mt][kt][j] = __ldg(wrow + kt * 8 + (j >> 1) * 4 + tig);
     }
   }
-  float wsu[MP];
-#pragma unroll
-  for (int p = 0; p < MP; ++p) wsu[p] = a.w_s[(int)rank * HU + warp * UW + p * 8 + g];
 
   // ---- initial state: every CTA needs the full h of its sequences as planes in buffer 0 -------------
   for (int i = tid; i < NS * (DG / 2); i += RNN_THREADS) {
@@ -203,8 +202,6 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     hbar_remote[r] = map_to_rank(smem_u32(&hbar[0]), r);
     hs_remote[r] = map_to_rank(smem_u32(hs), r);
   }
-  const uint32_t sbar_remote0 = map_to_rank(smem_u32(&sbar[0]), 0);
-  const uint32_t spart_remote0 = map_to_rank(smem_u32(spart), 0);
 
   const int n_cols = 4 * DG;
   float pin[MP][NT][4][2];     // P of the current step
@@ -230,7 +227,6 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     const bool send_h = step + 1 < a.n_range;
     // this step's sends of the cluster land in buffer buf^1: announce the bytes
     if (tid == 0 && send_h) mbar_arrive_expect_tx(&hbar[buf ^ 1], H_BYTES);
-    if (tid == 0 && rank == 0) mbar_arrive_expect_tx(&sbar[buf], SP_BYTES);
     if (step > 0) {
       // h_{t-1} from every CTA of the cluster (each buffer completes once per two steps)
       if (!mbar_wait_cluster_bounded(&hbar[buf], ((step - 1) >> 1) & 1)) {
@@ -251,19 +247,33 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[pl][mt][nt][e] = 0.f;
-    const uint16_t* hb = hs + buf * HS_BUF;
+    // B fragments: one ldmatrix.x4 brings the 8 sequences x 32 k-values of a plane (two k tiles);
+    // lane l addresses row (l & 7) of the 8 x 8 block (l >> 3).  Loaded one k-tile pair ahead.
+    const uint32_t hb_lane = smem_u32(hs + buf * HS_BUF + (lane & 7) * LDH + (lane >> 3) * 8);
+    uint32_t bf[2][RNN_PLANES][NT][4];
 #pragma unroll
-    for (int kt = 0; kt < KT; ++kt) {
+    for (int pl = 0; pl < RNN_PLANES; ++pl)
 #pragma unroll
-      for (int pl = 0; pl < RNN_PLANES; ++pl) {
+      for (int nt = 0; nt < NT; ++nt) ldmatrix_x4(bf[0][pl][nt], hb_lane + (uint32_t)(((pl * NS + nt * 8) * LDH) * 2));
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          const uint32_t* brow = reinterpret_cast<const uint32_t*>(hb + (pl * NS + nt * 8 + g) * LDH + kt * 16);
-          const uint32_t b0 = brow[tig], b1 = brow[4 + tig];
+    for (int kp = 0; kp < KT / 2; ++kp) {
+      const int cur = kp & 1;
+      if (kp + 1 < KT / 2) {
 #pragma unroll
-          for (int mt = 0; mt < 2 * MP; ++mt) mma_bf16_16816(acc[pl][mt][nt], A[mt][kt], b0, b1);
-        }
+        for (int pl = 0; pl < RNN_PLANES; ++pl)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            ldmatrix_x4(bf[cur ^ 1][pl][nt], hb_lane + (uint32_t)(((pl * NS + nt * 8) * LDH + (kp + 1) * 32) * 2));
       }
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+#pragma unroll
+        for (int pl = 0; pl < RNN_PLANES; ++pl)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int mt = 0; mt < 2 * MP; ++mt)
+              mma_bf16_16816(acc[pl][mt][nt], A[mt][2 * kp + half], bf[cur][pl][nt][2 * half], bf[cur][pl][nt][2 * half + 1]);
     }
 
     // ---- P_{t+1} into registers while the MMAs drain ----------------------------------------------------
@@ -280,29 +290,13 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           const float* prow = a.P + ((long long)s * a.n_range + step + 1) * n_cols + ug;
 #pragma unroll
           for (int gate = 0; gate < 4; ++gate) pnext[p][nt][gate][e] = live ? __ldcs(prow + gate * DG) : 0.f;
+          if (s < a.S && step + 2 < a.n_range) {
+#pragma unroll
+            for (int gate = 0; gate < 4; ++gate) asm volatile("prefetch.global.L2 [%0];" ::"l"(prow + n_cols + gate * DG));
+          }
         }
-
-    // ---- CTA 0: score of the previous step (its partials landed while this step's MMAs ran) ---------------
-    if (rank == 0 && step > 0) {
-      const int pb = buf ^ 1;
-      if (!mbar_wait_cluster_bounded(&sbar[pb], ((step - 1) >> 1) & 1)) {
-        if (lane == 0) set_status(a.status, ERR_TIMEOUT);
-      }
-      for (int j = warp; j < NS; j += RNN_WARPS) {
-        float vsum = (lane < CL * RNN_WARPS) ? spart[(pb * NS + j) * 32 + lane] : 0.f;
-        vsum = warp_sum(vsum);
-        const int s = seq0 + j;
-        if (lane == 0 && s < a.S) {
-          const float z = vsum + a.b_s;
-          a.scores[(long long)s * a.max_chunks + a.t0 + step - 1] = 1.f / (1.f + expf(-z));
-        }
-      }
-    }
 
     // ---- cell update (thread-local), planes of h_t into the warp's staging area ---------------------
-    float spv[NT][2];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) spv[nt][0] = spv[nt][1] = 0.f;
     __syncwarp();      // the previous step's pieces have been read out of the staging area
 #pragma unroll
     for (int p = 0; p < MP; ++p) {
@@ -324,7 +318,11 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           c[p][nt][e] = cn;
           const float hv = og * fast_tanh(cn);
           hlast[p][nt][e] = hv;
-          spv[nt][e] = fmaf(wsu[p], hv, spv[nt][e]);
+          {
+            // P_t of this (unit, sequence) is consumed: its gate-0 slot carries h_t to the score kernel
+            const int sq = seq0 + nt * 8 + tig * 2 + e;
+            if (sq < a.S) a.P[((long long)sq * a.n_range + step) * n_cols + (int)rank * HU + warp * UW + p * 8 + g] = hv;
+          }
           if (send_h) {
             uint32_t pl3[3];
             split3(hv, pl3);
@@ -342,26 +340,15 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         const int row = idx / MP, p = idx - row * MP;          // row = pl * NS + j
         const uint4 val = *reinterpret_cast<const uint4*>(my_stage + row * UW + p * 8);
         const uint32_t off = (uint32_t)(((buf ^ 1) * HS_BUF + row * LDH + (int)rank * HU + warp * UW + p * 8) * 2);
+        // own CTA: plain store (ordered by this warp's arrive below); peers: counted remote stores
+        *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(hs) + off) = val;
 #pragma unroll
-        for (int r = 0; r < CL; ++r) st_async_v4(hs_remote[r] + off, val, hbar_remote[r] + (buf ^ 1) * 8);
+        for (int r = 0; r < CL; ++r)
+          if (r != (int)rank) st_async_v4(hs_remote[r] + off, val, hbar_remote[r] + (buf ^ 1) * 8);
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&hbar[buf ^ 1]);     // release: this warp's local pieces are in place
     }
-    // score partials over the 8 units of the warp's lane groups (lanes differ in g) -> CTA 0
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        float vsum = spv[nt][e];
-        vsum += __shfl_xor_sync(0xffffffffu, vsum, 4);
-        vsum += __shfl_xor_sync(0xffffffffu, vsum, 8);
-        vsum += __shfl_xor_sync(0xffffffffu, vsum, 16);
-        if (g == 0) {
-          const int j = nt * 8 + tig * 2 + e;
-          const uint32_t off = (uint32_t)(((buf * NS + j) * 32 + (int)rank * RNN_WARPS + warp) * 4);
-          st_async_u32(spart_remote0 + off, __float_as_uint(vsum), sbar_remote0 + buf * 8);
-        }
-      }
-
 #pragma unroll
     for (int p = 0; p < MP; ++p)
 #pragma unroll
@@ -370,24 +357,6 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         for (int q = 0; q < 4; ++q)
 #pragma unroll
           for (int e = 0; e < 2; ++e) pin[p][nt][q][e] = pnext[p][nt][q][e];
-  }
-
-  // ---- CTA 0: score of the last step ------------------------------------------------------------------
-  if (rank == 0 && alive && a.n_range > 0) {
-    const int pb = (a.n_range - 1) & 1;
-    if (!mbar_wait_cluster_bounded(&sbar[pb], ((a.n_range - 1) >> 1) & 1)) {
-      if (lane == 0) set_status(a.status, ERR_TIMEOUT);
-    } else {
-      for (int j = warp; j < NS; j += RNN_WARPS) {
-        float vsum = (lane < CL * RNN_WARPS) ? spart[(pb * NS + j) * 32 + lane] : 0.f;
-        vsum = warp_sum(vsum);
-        const int s = seq0 + j;
-        if (lane == 0 && s < a.S) {
-          const float z = vsum + a.b_s;
-          a.scores[(long long)s * a.max_chunks + a.t0 + a.n_range - 1] = 1.f / (1.f + expf(-z));
-        }
-      }
-    }
   }
 
   // ---- carried state out ---------------------------------------------------------------------------
@@ -408,10 +377,35 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   cluster_sync_all();
 }
 
+// ---- score head: s_t = sigmoid(w_s . h_t + b_s), one warp per (sequence, chunk) --------------------------
+// h_t sits in columns [0, d_g) of row (s, t) of P.  Lane l sums elements l*4 .. l*4+3 (+128 per round) in
+// order, then a butterfly over the lanes: the same order for every launch.
+__global__ void __launch_bounds__(256) kve_gate_score_kernel(const float* __restrict__ P, const float* __restrict__ w_s,
+                                                             float b_s, float* __restrict__ scores, long long n_rows,
+                                                             int n_range, int t0, int max_chunks, int d_g) {
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= n_rows) return;
+  const float4* h = reinterpret_cast<const float4*>(P + row * 4 * d_g);
+  const float4* w = reinterpret_cast<const float4*>(w_s);
+  float acc = 0.f;
+  for (int i = lane; i < d_g / 4; i += 32) {
+    const float4 hv = __ldcs(h + i), wv = __ldg(w + i);
+    acc = fmaf(hv.x, wv.x, acc); acc = fmaf(hv.y, wv.y, acc);
+    acc = fmaf(hv.z, wv.z, acc); acc = fmaf(hv.w, wv.w, acc);
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) {
+    const int s = (int)(row / n_range);
+    const int t = t0 + (int)(row - (long long)s * n_range);
+    scores[(long long)s * max_chunks + t] = 1.f / (1.f + expf(-(acc + b_s)));
+  }
+}
+
 template <int DG, int CL, int NT>
 static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
   constexpr int NS = 8 * NT;
-  constexpr int smem = 2 * RNN_PLANES * NS * (DG + 8) * 2 + 2 * NS * 32 * 4 + RNN_PLANES * NS * (DG / CL) * 2 + 4 * 8;
+  constexpr int smem = 2 * RNN_PLANES * NS * (DG + 8) * 2 + RNN_PLANES * NS * (DG / CL) * 2 + 2 * 8;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kve_gate_rnn_kernel<DG, CL, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -424,19 +418,25 @@ static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
 }
 
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
-                            int d_g, const float* P, bool reset_state, cudaStream_t st) {
+                            int d_g, float* P, bool reset_state, cudaStream_t st) {
   if (t1 <= t0 || v.S <= 0) return cudaSuccess;
   RnnArgs a;
   a.P = P; a.W_hh = W_hh; a.w_s = w_s; a.b_s = b_s;
   a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c; a.status = v.status;
   a.S = v.S; a.max_chunks = v.max_chunks; a.t0 = t0; a.n_range = t1 - t0; a.reset = reset_state ? 1 : 0;
   // 16 sequences per cluster once 8 per cluster would need more than one wave of clusters
+  cudaError_t e;
   switch (d_g) {
-    case 256: return (v.S > 8 * (148 / 4)) ? launch_rnn_t<256, 4, 2>(a, st) : launch_rnn_t<256, 4, 1>(a, st);
-    case 128: return launch_rnn_t<128, 1, 1>(a, st);
-    case 64:  return (v.S > 8 * 148) ? launch_rnn_t<64, 1, 2>(a, st) : launch_rnn_t<64, 1, 1>(a, st);
+    case 256: e = (v.S > 8 * (148 / 4)) ? launch_rnn_t<256, 4, 2>(a, st) : launch_rnn_t<256, 4, 1>(a, st); break;
+    case 128: e = launch_rnn_t<128, 1, 1>(a, st); break;
+    case 64:  e = (v.S > 8 * 148) ? launch_rnn_t<64, 1, 2>(a, st) : launch_rnn_t<64, 1, 1>(a, st); break;
     default:  return cudaErrorInvalidValue;
   }
+  if (e != cudaSuccess) return e;
+  const long long n_rows = (long long)v.S * a.n_range;
+  kve_gate_score_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(P, w_s, b_s, v.scores, n_rows, a.n_range, t0,
+                                                                      v.max_chunks, d_g);
+  return cudaGetLastError();
 }
 
 }  // namespace kve
