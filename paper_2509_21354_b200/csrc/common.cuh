@@ -28,8 +28,20 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
   u += 0x7fffu + ((u >> 16) & 1u);
   return u >> 16;
 }
+// two fp32 -> packed bf16 pair (lo in bits 0..15), round to nearest even, one conversion instruction
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+// exact split of two fp32 values into three bf16 pieces each (x = p0 + p1 + p2), packed pairwise:
+// w[pl] holds piece pl of `a` in bits 0..15 and of `b` in bits 16..31
+__device__ __forceinline__ void split3_pair(float a, float b, uint32_t (&w)[3]) {
+  w[0] = pack_bf16x2(a, b);
+  const float ra = a - bf16lo(w[0]), rb = b - bf16hi(w[0]);
+  w[1] = pack_bf16x2(ra, rb);
+  const float sa = ra - bf16lo(w[1]), sb = rb - bf16hi(w[1]);
+  w[2] = pack_bf16x2(sa, sb);
 }
 
 // ---- shared-memory addresses, mbarriers, bulk copies --------------------------------------------

@@ -206,30 +206,29 @@ constexpr int MT_SMEM_BYTES = MT_SMEM_BAR + 64 + 1024;                    // + s
 constexpr int MT_TMEM_COLS = 512;                                         // H: columns [0, d_sum), Y: columns [256, 384)
 constexpr int MT_TMEM_Y = 256;
 
-// exact split of an fp32 value into three bf16 pieces: x = p[0] + p[1] + p[2]
-__device__ __forceinline__ void split3_bits(float x, uint32_t (&p)[3]) {
-  p[0] = f32_to_bf16_bits(x);
-  const float r1 = x - __uint_as_float(p[0] << 16);
-  p[1] = f32_to_bf16_bits(r1);
-  const float r2 = r1 - __uint_as_float(p[1] << 16);
-  p[2] = f32_to_bf16_bits(r2);
-}
-
 // splits 8 consecutive fp32 values and stores the three 16-byte pieces at dst + pl * plane_stride
 __device__ __forceinline__ void store_split8(const float (&x)[8], unsigned char* dst, int plane_stride) {
-  uint32_t w[3][4];
+  uint32_t w[4][3];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    uint32_t a[3], b[3];
-    split3_bits(x[2 * e], a);
-    split3_bits(x[2 * e + 1], b);
-#pragma unroll
-    for (int pl = 0; pl < 3; ++pl) w[pl][e] = a[pl] | (b[pl] << 16);
-  }
+  for (int e = 0; e < 4; ++e) split3_pair(x[2 * e], x[2 * e + 1], w[e]);
 #pragma unroll
   for (int pl = 0; pl < 3; ++pl)
-    *reinterpret_cast<uint4*>(dst + pl * plane_stride) = make_uint4(w[pl][0], w[pl][1], w[pl][2], w[pl][3]);
+    *reinterpret_cast<uint4*>(dst + pl * plane_stride) = make_uint4(w[0][pl], w[1][pl], w[2][pl], w[3][pl]);
 }
+
+// erf by the rational-times-exponential formula 7.1.26 of Abramowitz & Stegun (absolute error below
+// 1.5e-7, i.e. at the level of fp32 rounding of the activations), odd extension for x < 0
+__device__ __forceinline__ float erf_as(float x) {
+  const float ax = fabsf(x);
+  const float t = __fdividef(1.f, fmaf(0.3275911f, ax, 1.f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float y = 1.f - poly * t * __expf(-ax * ax);
+  return copysignf(y, x);
+}
+__device__ __forceinline__ float gelu_tc(float x) { return 0.5f * x * (1.f + erf_as(x * 0.70710678118654752440f)); }
 
 __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerView v, int t0, int n_range, long long n_units,
                                                                          MlpWeights w, int d_sum) {
@@ -258,14 +257,14 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
   // ---- one-time set-up -----------------------------------------------------------------------------
   for (int i = tid; i < d_sum * 16; i += MT_THREADS) {              // W1 [d_sum][128]: rows of 16 pieces, 2 K-blocks
     const int r = i >> 4, p = i & 15;
-    const uint4 val = __ldg(reinterpret_cast<const uint4*>(W1 + (long long)r * D) + p);
-    *reinterpret_cast<uint4*>(W1s + (p >> 3) * (d_sum * umma::KBLOCK_ROW_BYTES) + umma::piece_offset(r, p & 7)) = val;
+    cp_async16(W1s + (p >> 3) * (d_sum * umma::KBLOCK_ROW_BYTES) + umma::piece_offset(r, p & 7),
+               reinterpret_cast<const uint4*>(W1 + (long long)r * D) + p, true);
   }
   const int w2_pieces = d_sum / 8;
   for (int i = tid; i < D * w2_pieces; i += MT_THREADS) {           // W2 [128][d_sum]: n_slices K-blocks of 16 KB
     const int r = i / w2_pieces, p = i - r * w2_pieces;
-    const uint4 val = __ldg(reinterpret_cast<const uint4*>(W2 + (long long)r * d_sum) + p);
-    *reinterpret_cast<uint4*>(W2s + (p >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, p & 7)) = val;
+    cp_async16(W2s + (p >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, p & 7),
+               reinterpret_cast<const uint4*>(W2 + (long long)r * d_sum) + p, true);
   }
   for (int i = tid; i < d_sum; i += MT_THREADS) b1s[i] = b1[i];
   for (int i = tid; i < D; i += MT_THREADS) b2s[i] = b2[i];
@@ -276,6 +275,8 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
     mbar_init(&bar_buf[1], 1);
     mbar_fence_init();
   }
+  cp_async_wait_all();
+  umma::fence_smem_to_async();
   umma::fence_before_sync();
   __syncthreads();
   umma::fence_after_sync();
@@ -291,20 +292,31 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
   for (long long tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
     const long long unit0 = tile * MT_M;
     // ---- chunk means -> three bf16 planes (layer-1 A operand) ------------------------------------------
-#pragma unroll 2
-    for (int i = tid; i < MT_M * 16; i += MT_THREADS) {
-      const int r = i >> 4, pc = i & 15;
-      const long long unit = unit0 + r;
-      float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      if (unit < n_units) {
-        const int s = (int)(unit / n_range);
-        const int t = t0 + (int)(unit - (long long)s * n_range);
-        const float4* src = reinterpret_cast<const float4*>(sum_f32 + ((long long)s * v.max_chunks + t) * D + pc * 8);
-        const float4 a = src[0], b = src[1];
-        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+    {
+      // a thread keeps its 32-byte column pc and walks down 8 rows: all 16 loads first, then the splits
+      // (32-bit index arithmetic, one division per row; the host checks the ranges)
+      const int pc = tid & 15;
+      const uint32_t u0 = (uint32_t)unit0, nr = (uint32_t)n_range, total = (uint32_t)n_units;
+      float4 lo[8], hi[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t unit = u0 + (tid >> 4) + 16 * i;
+        lo[i] = hi[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (unit < total) {
+          const uint32_t s = unit / nr;
+          const uint32_t t = (uint32_t)t0 + (unit - s * nr);
+          const float4* src = reinterpret_cast<const float4*>(sum_f32 + (size_t)(s * (uint32_t)v.max_chunks + t) * D + pc * 8);
+          lo[i] = src[0];
+          hi[i] = src[1];
+        }
       }
-      // plane pl, K-block kb at (pl * 2 + kb) * 16 KB
-      store_split8(x, As + (pc >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, pc & 7), 2 * MT_PLANE_KB_BYTES);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int r = (tid >> 4) + 16 * i;
+        const float x[8] = {lo[i].x, lo[i].y, lo[i].z, lo[i].w, hi[i].x, hi[i].y, hi[i].z, hi[i].w};
+        // plane pl, K-block kb at (pl * 2 + kb) * 16 KB
+        store_split8(x, As + (pc >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, pc & 7), 2 * MT_PLANE_KB_BYTES);
+      }
     }
     umma::fence_smem_to_async();
     __syncthreads();
@@ -345,7 +357,7 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
       for (int q = 0; q < 4; ++q) {
         float g[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) g[e] = gelu_erf(h[q * 8 + e] + b1s[j * 64 + half * 32 + q * 8 + e]);
+        for (int e = 0; e < 8; ++e) g[e] = gelu_tc(h[q * 8 + e] + b1s[j * 64 + half * 32 + q * 8 + e]);
         store_split8(g, abuf + umma::piece_offset(row_in_tile, half * 4 + q), MT_PLANE_KB_BYTES);
       }
       umma::fence_smem_to_async();
@@ -378,31 +390,47 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
     umma::fence_after_sync();
 
     // ---- epilogue: Y + b2 -> fp32 summary and its bf16 rounding ----------------------------------------------
+    // The operand space is idle now: it holds the output row table and, per warp, a 32 x 32 block on
+    // its way out.  tcgen05.ld hands a thread one row; the block is turned through shared memory
+    // (16-byte groups, group q of row r at position q ^ (r & 7)) so that every store instruction
+    // writes whole 128-byte (fp32) / 64-byte (bf16) row segments.
     {
-      const long long unit = unit0 + row_in_tile;
-      long long o = 0;
-      if (unit < n_units) {
-        const int s = (int)(unit / n_range);
-        const int t = t0 + (int)(unit - (long long)s * n_range);
-        o = ((long long)s * v.max_chunks + t) * D;
+      int* row_tab = reinterpret_cast<int*>(As + (MT_THREADS / 32) * 4096);       // [128] summary row, -1 beyond the end
+      float* stg = reinterpret_cast<float*>(As) + warp * 1024;
+      if (tid < MT_M) {
+        const long long unit = unit0 + tid;
+        int o = -1;
+        if (unit < n_units) {
+          const uint32_t s = (uint32_t)unit / (uint32_t)n_range;
+          o = (int)(s * (uint32_t)v.max_chunks + (uint32_t)t0 + ((uint32_t)unit - s * (uint32_t)n_range));
+        }
+        row_tab[tid] = o;
       }
+      __syncthreads();
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {
         const int c = half * 64 + cc * 32;
         float y[32];
         umma::tmem_ld32(tmem_y + tmem_lane + (uint32_t)c, y);
-        if (unit < n_units) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) y[e] += b2s[c + e];
-          float4* df = reinterpret_cast<float4*>(sum_f32 + o + c);
-          uint4* db = reinterpret_cast<uint4*>(sum_b16 + o + c);
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<float4*>(stg + lane * 32 + ((q ^ (lane & 7)) << 2)) =
+              make_float4(y[4 * q] + b2s[c + 4 * q], y[4 * q + 1] + b2s[c + 4 * q + 1], y[4 * q + 2] + b2s[c + 4 * q + 2],
+                          y[4 * q + 3] + b2s[c + 4 * q + 3]);
+        __syncwarp();
+        const int q = lane & 7;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) df[e] = make_float4(y[4 * e], y[4 * e + 1], y[4 * e + 2], y[4 * e + 3]);
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            db[e] = make_uint4(pack_bf16x2(y[8 * e], y[8 * e + 1]), pack_bf16x2(y[8 * e + 2], y[8 * e + 3]),
-                               pack_bf16x2(y[8 * e + 4], y[8 * e + 5]), pack_bf16x2(y[8 * e + 6], y[8 * e + 7]));
+        for (int i = 0; i < 8; ++i) {
+          const int rr = i * 4 + (lane >> 3);
+          const float4 val = *reinterpret_cast<const float4*>(stg + rr * 32 + ((q ^ (rr & 7)) << 2));
+          const int orow = row_tab[lg * 32 + rr];
+          if (orow >= 0) {
+            const size_t o = (size_t)orow * D + c + q * 4;
+            *reinterpret_cast<float4*>(sum_f32 + o) = val;
+            *reinterpret_cast<uint2*>(sum_b16 + o) = make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
+          }
         }
+        __syncwarp();
       }
     }
     umma::fence_before_sync();
@@ -419,7 +447,8 @@ cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeight
   const int n_range = t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
-  if (d_sum % 64 == 0 && d_sum <= MT_MAX_DSUM) {
+  if (d_sum % 64 == 0 && d_sum <= MT_MAX_DSUM && n_units + MT_M < (1LL << 31) &&
+      (long long)v.S * v.max_chunks < (1LL << 31)) {
     static bool attr_tc = false;
     if (!attr_tc) {
       cudaError_t e = cudaFuncSetAttribute(kve_chunk_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MT_SMEM_BYTES);
