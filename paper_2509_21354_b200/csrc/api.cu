@@ -122,8 +122,8 @@ bool bad_layer(const kvE_store* st, int layer) { return !st || layer < 0 || laye
 
 // rows per split and grid width for `n_rows_upper` logical rows per sequence
 AttnPlan plan_attention(const kvE_store* st, long long n_rows_upper) {
-  const long long target_ctas = 148LL * 2 * 2;     // about two waves at two CTAs per SM
-  long long splits = (target_ctas + st->S - 1) / st->S;
+  const long long one_wave = 148LL * 2;            // two CTAs per SM: everything resident at once, fewest merges
+  long long splits = one_wave / st->S;
   const long long max_useful = (n_rows_upper + 2 * ATTN_TILE_ROWS - 1) / (2 * ATTN_TILE_ROWS);   // >= 128 rows per split
   if (splits > max_useful) splits = max_useful;
   if (splits > MAX_SPLITS) splits = MAX_SPLITS;
