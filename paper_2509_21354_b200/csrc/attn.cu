@@ -3,7 +3,8 @@
 // and, with mode = DENSE, Eq. 1 over every stored token (the full-cache baseline).
 //
 // HBM-bound: every retained K and V row (256 bytes each) is read exactly once.
-//  * grid = (splits, sequences); a CTA owns a contiguous range of a sequence's logical rows.
+//  * grid = (splits, sequences); a CTA owns a contiguous range of a sequence's logical rows
+//    (raw tail first, kept chunks after it).
 //  * one producer warp turns logical rows into addresses (summary store / page table), merges
 //    rows that are contiguous in memory into runs with a ballot, and issues one bulk copy
 //    (TMA engine, global -> shared, mbarrier byte counting) per run into a 3-stage ring of
@@ -43,27 +44,29 @@ struct AttnArgs {
 
 // address of logical row L of sequence s (K and V); falls back to a safe row and flags the status
 // word when an index is out of range
-__device__ __forceinline__ void row_address(const AttnArgs& a, int s, int L, int n_lead, int raw0,
+// The CTA walks a sequence's rows in the order [raw tail ; kept chunks]: the raw tail's addresses need
+// only the page table, so the first tiles can be requested while the keep list is still on its way
+// (softmax does not care about the order of its rows).
+__device__ __forceinline__ void row_address(const AttnArgs& a, int s, int L, int n_tail, int raw0,
                                             const uint16_t*& kp, const uint16_t*& vp) {
   const LayerView& v = a.v;
   const long long sb = (long long)s * v.max_chunks;
-  if (L < n_lead && a.mode == ATTN_SUMMARY) {
-    int t = v.keep_idx[sb + L];
+  int chunk, r;
+  if (L < n_tail) {
+    const int p = raw0 + L;
+    chunk = p / v.C;
+    r = p - chunk * v.C;
+  } else if (a.mode == ATTN_SUMMARY) {
+    int t = v.keep_idx[sb + (L - n_tail)];
     if (t < 0 || t >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); t = 0; }
     kp = v.ksum_bf16 + (sb + t) * D;
     vp = v.vsum_bf16 + (sb + t) * D;
     return;
-  }
-  int chunk, r;
-  if (L < n_lead) {   // RAW: row r of the (L / C)-th kept chunk
-    const int ci = L / v.C;
-    r = L - ci * v.C;
+  } else {            // RAW: row r of the ((L - n_tail) / C)-th kept chunk
+    const int ci = (L - n_tail) / v.C;
+    r = (L - n_tail) - ci * v.C;
     chunk = v.keep_idx[sb + ci];
     if (chunk < 0 || chunk >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); chunk = 0; }
-  } else {
-    const int p = raw0 + (L - n_lead);
-    chunk = p / v.C;
-    r = p - chunk * v.C;
   }
   long long page = v.page_table[sb + chunk];
   if (page < 0 || page >= v.n_pages) { set_status(v.status, ERR_CAPACITY); page = 0; }
@@ -99,7 +102,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   const int M = (a.mode == ATTN_DENSE) ? 0 : min(max(v.keep_cnt[s], 0), a.n_chunks);
   const int raw0 = (a.mode == ATTN_DENSE) ? 0 : a.n_chunks * v.C;
   const int n_lead = (a.mode == ATTN_RAW) ? M * v.C : M;
-  const int n_rows = n_lead + max(0, n - raw0);
+  const int n_tail = max(0, n - raw0);
+  const int n_rows = n_tail + n_lead;
   const int n_splits = max(1, (n_rows + a.rows_per_split - 1) / a.rows_per_split);
   if (split >= n_splits) return;
   const int r_begin = split * a.rows_per_split;
@@ -117,11 +121,26 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
 
   if (warp == AT_CWARPS) {
     // ================= producer warp =================
-    for (int i = 0; i < n_tiles; ++i) {
+    // Row addresses need up to two dependent global loads (keep list, page table).  They are resolved
+    // AT_STAGES tiles ahead of the copies, each tile in a slot of its own, so the look-ups of several
+    // tiles are in flight together and never sit between a freed stage and its refill.
+    struct TileAddr { const uint16_t *k[AT_TILE / 32], *v[AT_TILE / 32]; };
+    auto resolve = [&](int i, TileAddr& t) {
+      const int row0 = r_begin + i * AT_TILE;
+      const int rows_in_tile = (i < n_tiles) ? min(AT_TILE, r_end - row0) : 0;
+#pragma unroll
+      for (int half = 0; half < AT_TILE / 32; ++half) {
+        const int rl = half * 32 + lane;
+        t.k[half] = t.v[half] = nullptr;
+        if (rl < rows_in_tile) row_address(a, s, row0 + rl, n_tail, raw0, t.k[half], t.v[half]);
+      }
+    };
+    // waits for the stage, issues the copies of tile i from its resolved addresses; false on a timed-out wait
+    auto issue = [&](int i, const TileAddr& t) -> bool {
       const int stage = i % AT_STAGES, round = i / AT_STAGES;
       if (round > 0 && !mbar_wait_bounded(&empty[stage], (round - 1) & 1)) {
         if (lane == 0) set_status(v.status, ERR_TIMEOUT);
-        break;
+        return false;
       }
       const int row0 = r_begin + i * AT_TILE;
       const int rows_in_tile = min(AT_TILE, r_end - row0);
@@ -131,8 +150,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       for (int half = 0; half < AT_TILE / 32; ++half) {
         const int rl = half * 32 + lane;
         const bool valid = rl < rows_in_tile;
-        const uint16_t *kp = nullptr, *vp = nullptr;
-        if (valid) row_address(a, s, row0 + rl, n_lead, raw0, kp, vp);
+        const uint16_t *kp = t.k[half], *vp = t.v[half];
         const unsigned long long ka = (unsigned long long)kp, va = (unsigned long long)vp;
         const unsigned long long kprev = __shfl_up_sync(0xffffffffu, ka, 1);
         const unsigned long long vprev = __shfl_up_sync(0xffffffffu, va, 1);
@@ -148,6 +166,18 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
           bulk_g2s(Vs + stage * AT_STAGE_ELEMS + rl * D, vp, bytes, &full[stage]);
         }
       }
+      return true;
+    };
+    static_assert(AT_STAGES == 3, "three slots of look-ahead");
+    TileAddr t0, t1, t2;
+    resolve(0, t0);
+    resolve(1, t1);
+    resolve(2, t2);
+    for (int i = 0; i < n_tiles; i += AT_STAGES) {
+      if (!issue(i, t0)) break;
+      resolve(i + 3, t0);
+      if (i + 1 < n_tiles) { if (!issue(i + 1, t1)) break; resolve(i + 4, t1); }
+      if (i + 2 < n_tiles) { if (!issue(i + 2, t2)) break; resolve(i + 5, t2); }
     }
   } else {
     // ================= consumer warps =================
