@@ -34,7 +34,7 @@ METRIC = "gated_decode_attention_steps_per_sec"
 UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 SCALE = 1.0 / math.sqrt(128.0)
-KERNELS_PER_STEP = 9   # set_len, append (copy + length), chunk mean, chunk MLP, gate projection, gate recurrence, compact, attention
+KERNELS_PER_STEP = 10  # set_len, append (copy + length), chunk mean, chunk MLP, gate projection, gate recurrence, score head, compact, attention
 
 
 def load_peaks():
@@ -52,6 +52,18 @@ def shard_batch(B_per_gpu: int, rank: int, world: int):
     the gated cache of one (layer, batch, head) never reads another's."""
     lo = rank * B_per_gpu
     return lo, lo + B_per_gpu
+
+
+def max_over_ranks(values, world: int, device="cuda"):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time of a
+    multi-GPU step).  The only collective of the benchmark; identity when world == 1."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
 
 
 # ---------------------------------------------------------------------------------------------- clocks
@@ -140,6 +152,17 @@ def algorithmic_bytes(wl, Nc, keep_mean, R):
     return by
 
 
+def algorithmic_flops(wl, Nc):
+    """Floating-point operations of the contraction-shaped kernels as the method defines them (one
+    multiply-add = 2; the exact-split planes the kernels use on top are not counted)."""
+    S, d_g, d = wl.S, wl.d_g, 128
+    fl = {"gate_proj": S * Nc * 2 * (2 * d) * (4 * d_g),
+          "gate_rnn": S * Nc * (2 * d_g * 4 * d_g + 2 * d_g)}
+    if wl.agg == "mlp":
+        fl["chunk_mlp"] = 2 * S * Nc * 2 * (d * wl.d_sum + wl.d_sum * d)
+    return fl
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -201,6 +224,24 @@ def run_ours(args, rank, world, local_rank):
     ms_total = ev0.elapsed_time(ev1)
     assert st.poll_status() == 0
 
+    # ---- steady-state decode step (between two gate triggers): append one token, gated attention ----
+    def step_steady():
+        st.set_len(0, n0 - 1)
+        st.append(0, k3, v3)
+        st.decode_attn(0, q, out)
+
+    for _ in range(3):
+        step_steady()
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step_steady()
+    ev1.record()
+    barrier()
+    ms_steady = max_over_ranks([ev0.elapsed_time(ev1)], world)[0]
+    steady = {"what": "append + gated attention only (summaries, gate and keep list reused: the state between two triggers)",
+              "value": world * args.steps / (ms_steady * 1e-3), "unit": UNIT, "ms_per_step": ms_steady / args.steps}
+
     # ---- end to end: the same step through kvE_decode_step_host, host buffers, copies timed ----
     hk, hv, hq = (t.cpu().pin_memory() for t in (k_new, v_new, q))
     hout = torch.zeros((S, 128), dtype=torch.bfloat16).pin_memory()
@@ -219,10 +260,7 @@ def run_ours(args, rank, world, local_rank):
     e2e_s = time.perf_counter() - t0
     same = bool(torch.equal(hout.cuda(), out))
 
-    if world > 1:
-        t = torch.tensor([ms_total, e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, e2e_s = t[0].item(), t[1].item()
+    ms_total, e2e_s = max_over_ranks([ms_total, e2e_s], world)
     if rank != 0:
         return None
 
@@ -251,10 +289,16 @@ def run_ours(args, rank, world, local_rank):
     by_kernel = {"append": S * 4 * 256, "chunk_mean": by["chunk_mean"], "chunk_mlp": by["chunk_mlp"],
                  "gate_proj": by["gate_proj"], "gate_rnn": by["gate_rnn"], "compact": by["compact"],
                  "attn": by["attn_gated"], "attn_dense": by["attn_dense"]}
+    fl = algorithmic_flops(wl, Nc)
+    tensor_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])     # kernels timed inside a long step
     kern = {}
     for k, t in us.items():
         kern[k] = {"us": t, "bytes": by_kernel[k], "GB/s": by_kernel[k] / (t * 1e-6) / 1e9}
         kern[k]["frac_of_hbm_peak"] = kern[k]["GB/s"] / hbm
+        if k in fl:
+            kern[k]["flops"] = fl[k]
+            kern[k]["TFLOP/s"] = fl[k] / (t * 1e-6) / 1e12
+            kern[k]["frac_of_bf16_peak"] = kern[k]["TFLOP/s"] / tensor_peak
     kern["attn"]["us_l2_flushed"] = us_attn_cold
     kern["attn"]["GB/s_l2_flushed"] = by_kernel["attn"] / (us_attn_cold * 1e-6) / 1e9
     dominant = max((k for k in kern if k != "attn_dense"), key=lambda k: kern[k]["us"])
@@ -263,16 +307,29 @@ def run_ours(args, rank, world, local_rank):
     if os.path.exists(tp):
         with open(tp) as f:
             traffic = json.load(f).get(dominant)
-    roofline = {"kernel": dominant, "bound": "hbm", "achieved": kern[dominant]["GB/s"], "peak": hbm, "unit": "GB/s",
-                "frac": kern[dominant]["GB/s"] / hbm, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                "algorithmic_bytes": kern[dominant]["bytes"], "us_per_launch": kern[dominant]["us"]}
+    if dominant in fl:
+        roofline = {"kernel": dominant, "bound": "tensor", "achieved": kern[dominant]["TFLOP/s"], "peak": tensor_peak,
+                    "unit": "TFLOP/s", "frac": kern[dominant]["frac_of_bf16_peak"], "traffic": traffic,
+                    "peak_kind": f"of {peak_kind} (sustained bf16)", "algorithmic_flops": fl[dominant],
+                    "us_per_launch": kern[dominant]["us"]}
+        if dominant == "gate_rnn":
+            roofline["note"] = (f"{Nc} strictly sequential LSTM steps per sequence: bounded by per-step latency "
+                                f"({kern[dominant]['us'] / Nc:.2f} us per step), not by tensor throughput")
+    else:
+        roofline = {"kernel": dominant, "bound": "hbm", "achieved": kern[dominant]["GB/s"], "peak": hbm, "unit": "GB/s",
+                    "frac": kern[dominant]["GB/s"] / hbm, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                    "algorithmic_bytes": kern[dominant]["bytes"], "us_per_launch": kern[dominant]["us"]}
+    hbm_kernel = max((k for k in ("chunk_mean", "attn")), key=lambda k: kern[k]["us"])
+    roofline_hbm = {"kernel": hbm_kernel, "bound": "hbm", "achieved": kern[hbm_kernel]["GB/s"], "peak": hbm, "unit": "GB/s",
+                    "frac": kern[hbm_kernel]["GB/s"] / hbm, "algorithmic_bytes": kern[hbm_kernel]["bytes"],
+                    "us_per_launch": kern[hbm_kernel]["us"], "peak_kind": f"of {peak_kind}"}
     us["attn_gated"] = us_attn_cold
 
     ms_step = ms_total / args.steps
     res = {
         "metric": METRIC, "value": world * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "d": 128, "n": wl.n, "C": wl.C, "W": wl.W,
                    "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend, "n_layers_timed": 1,
                    "stale_chunks": Nc, "kept_chunks_mean": keep_mean, "n_eff": R + keep_mean,
@@ -283,6 +340,8 @@ def run_ours(args, rank, world, local_rank):
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "clocks": clk.summary(),
         "roofline": roofline,
+        "roofline_largest_hbm_kernel": roofline_hbm,
+        "steady_state": steady,
         "kernels": kern,
         "attention_vs_dense": {"note": "attention kernels alone, L2 flushed before every launch",
                                "gated_us": us["attn_gated"], "dense_us": us["attn_dense"],
