@@ -172,7 +172,7 @@ def run_ours(args, rank, world, local_rank):
     wl = wlm.CONFIGS[args.workload].small(n_layers=1)
     lo, _ = shard_batch(wl.B, rank, world)
     seed = 1000 + lo
-    st = b.Store(B=wl.B, H=wl.H, C_=wl.C, W=wl.W, max_tokens=wl.n, d_g=wl.d_g, agg=wl.agg, d_sum=wl.d_sum,
+    st = b.Store(B=wl.B, H=wl.H, C_=wl.C, W=wl.W, max_tokens=wl.n + wl.C, d_g=wl.d_g, agg=wl.agg, d_sum=wl.d_sum,
                  attend=args.attend, page_perm="random", seed=seed)
     g = fill_cache(st, wl, seed)
     mlp = wlm.gen_mlp_weights(wl)
@@ -225,8 +225,9 @@ def run_ours(args, rank, world, local_rank):
     assert st.poll_status() == 0
 
     # ---- steady-state decode step (between two gate triggers): append one token, gated attention ----
+    # (token n0 + 1: no chunk leaves the window, so the keep list of the last full step stands)
     def step_steady():
-        st.set_len(0, n0 - 1)
+        st.set_len(0, n0)
         st.append(0, k3, v3)
         st.decode_attn(0, q, out)
 
@@ -239,6 +240,9 @@ def run_ours(args, rank, world, local_rank):
     ev1.record()
     barrier()
     ms_steady = max_over_ranks([ev0.elapsed_time(ev1)], world)[0]
+    assert st.poll_status() == 0
+    step()                      # back to the state and output of a full step
+    torch.cuda.synchronize()
     steady = {"what": "append + gated attention only (summaries, gate and keep list reused: the state between two triggers)",
               "value": world * args.steps / (ms_steady * 1e-3), "unit": UNIT, "ms_per_step": ms_steady / args.steps}
 
@@ -303,10 +307,11 @@ def run_ours(args, rank, world, local_rank):
     kern["attn"]["GB/s_l2_flushed"] = by_kernel["attn"] / (us_attn_cold * 1e-6) / 1e9
     dominant = max((k for k in kern if k != "attn_dense"), key=lambda k: kern[k]["us"])
     traffic = None
-    tp = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tp):
+    tp = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.txt")
+    if os.path.exists(tp) and args.attend == "summary":
         with open(tp) as f:
-            traffic = json.load(f).get(dominant)
+            tab = dict(line.split() for line in f if line.strip() and not line.startswith("#"))
+        traffic = int(tab[dominant]) if dominant in tab else None
     if dominant in fl:
         roofline = {"kernel": dominant, "bound": "tensor", "achieved": kern[dominant]["TFLOP/s"], "peak": tensor_peak,
                     "unit": "TFLOP/s", "frac": kern[dominant]["frac_of_bf16_peak"], "traffic": traffic,
