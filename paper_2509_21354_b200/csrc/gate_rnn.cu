@@ -70,6 +70,12 @@ __device__ __forceinline__ void st_async_v4(uint32_t addr, const uint4& v, uint3
                "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(bar)
                : "memory");
 }
+// bulk copy from this CTA's shared memory into a peer's (addresses from mapa), bytes counted on the peer's barrier
+__device__ __forceinline__ void bulk_s2cluster(uint32_t dst, uint32_t src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "r"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -124,18 +130,18 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   constexpr int MP = UW / 8;             // pairs of m16 tiles per warp (a pair = 8 units x 4 gates)
   constexpr int KT = DG / 16;            // k tiles
   constexpr int NS = 8 * NT;             // sequences per cluster
-  constexpr int LDH = DG + 8;            // padded plane row (bf16 elements): conflict-free B fragments
-  constexpr int HS_BUF = RNN_PLANES * NS * LDH;                 // bf16 elements per h buffer
+  constexpr int KBLK = RNN_PLANES * NS * 8;                     // bf16 elements of one k-block: [plane][sequence][8 units]
+  constexpr int HS_BUF = (DG / 8) * KBLK;                       // bf16 elements per h buffer: [k-block][plane][sequence][8]
   constexpr int STG_WARP = RNN_PLANES * NS * UW;                // bf16 elements of one warp's staging area
   constexpr int N_PIECES = RNN_PLANES * NS * MP;                // 16-byte pieces a warp sends to each CTA per step
   constexpr uint32_t H_BYTES = RNN_PLANES * NS * (DG - HU) * 2; // bytes of h planes a CTA receives from its peers per step
   constexpr int OFF_STAGE = 2 * HS_BUF * 2;
   constexpr int OFF_BARS = OFF_STAGE + RNN_WARPS * STG_WARP * 2;
   static_assert(UW % 8 == 0 && MP >= 1, "8 warps x 8k hidden units per CTA");
-  static_assert(OFF_STAGE % 16 == 0 && OFF_BARS % 16 == 0 && (LDH * 2) % 16 == 0, "16-byte pieces");
+  static_assert(OFF_STAGE % 16 == 0 && OFF_BARS % 16 == 0, "16-byte pieces");
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                          // [2][PLANES][NS][LDH]
+  uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                          // [2][DG / 8][PLANES][NS][8]
   uint16_t* stage = reinterpret_cast<uint16_t*>(smem_raw + OFF_STAGE);           // [warps][PLANES][NS][UW]
   uint64_t* hbar = reinterpret_cast<uint64_t*>(smem_raw + OFF_BARS);             // [2] h planes landed
 
@@ -179,7 +185,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     split3(h1, p1);
 #pragma unroll
     for (int pl = 0; pl < RNN_PLANES; ++pl)
-      *reinterpret_cast<uint32_t*>(hs + (pl * NS + j) * LDH + k2 * 2) = p0[pl] | (p1[pl] << 16);
+      *reinterpret_cast<uint32_t*>(hs + (k2 >> 2) * KBLK + (pl * NS + j) * 8 + (k2 & 3) * 2) = p0[pl] | (p1[pl] << 16);
   }
   float c[MP][NT][2], hlast[MP][NT][2];
 #pragma unroll
@@ -196,12 +202,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       }
 
   // addresses in the other CTAs that do not change from step to step
-  uint32_t hbar_remote[CL], hs_remote[CL];
-#pragma unroll
-  for (int r = 0; r < CL; ++r) {
-    hbar_remote[r] = map_to_rank(smem_u32(&hbar[0]), r);
-    hs_remote[r] = map_to_rank(smem_u32(hs), r);
-  }
+  // lane r < CL feeds peer r: that CTA's h buffers and barriers, as addresses in the cluster window
+  const uint32_t peer_hs = map_to_rank(smem_u32(hs), lane < CL ? lane : 0);
+  const uint32_t peer_bar = map_to_rank(smem_u32(&hbar[0]), lane < CL ? lane : 0);
 
   const int n_cols = 4 * DG;
   float pin[MP][NT][4][2];     // P of the current step
@@ -249,12 +252,12 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           for (int e = 0; e < 4; ++e) acc[pl][mt][nt][e] = 0.f;
     // B fragments: one ldmatrix.x4 brings the 8 sequences x 32 k-values of a plane (two k tiles);
     // lane l addresses row (l & 7) of the 8 x 8 block (l >> 3).  Loaded one k-tile pair ahead.
-    const uint32_t hb_lane = smem_u32(hs + buf * HS_BUF + (lane & 7) * LDH + (lane >> 3) * 8);
+    const uint32_t hb_lane = smem_u32(hs + buf * HS_BUF + (lane >> 3) * KBLK + (lane & 7) * 8);
     uint32_t bf[2][RNN_PLANES][NT][4];
 #pragma unroll
     for (int pl = 0; pl < RNN_PLANES; ++pl)
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) ldmatrix_x4(bf[0][pl][nt], hb_lane + (uint32_t)(((pl * NS + nt * 8) * LDH) * 2));
+      for (int nt = 0; nt < NT; ++nt) ldmatrix_x4(bf[0][pl][nt], hb_lane + (uint32_t)(((pl * NS + nt * 8) * 8) * 2));
 #pragma unroll
     for (int kp = 0; kp < KT / 2; ++kp) {
       const int cur = kp & 1;
@@ -263,7 +266,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         for (int pl = 0; pl < RNN_PLANES; ++pl)
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt)
-            ldmatrix_x4(bf[cur ^ 1][pl][nt], hb_lane + (uint32_t)(((pl * NS + nt * 8) * LDH + (kp + 1) * 32) * 2));
+            ldmatrix_x4(bf[cur ^ 1][pl][nt], hb_lane + (uint32_t)(((kp + 1) * 4 * KBLK + (pl * NS + nt * 8) * 8) * 2));
       }
 #pragma unroll
       for (int half = 0; half < 2; ++half)
@@ -297,7 +300,8 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         }
 
     // ---- cell update (thread-local), planes of h_t into the warp's staging area ---------------------
-    __syncwarp();      // the previous step's pieces have been read out of the staging area
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    __syncwarp();      // the previous step's copies have read the staging area
 #pragma unroll
     for (int p = 0; p < MP; ++p) {
 #pragma unroll
@@ -328,27 +332,31 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
             split3(hv, pl3);
             const int j = nt * 8 + tig * 2 + e;
 #pragma unroll
-            for (int pl = 0; pl < RNN_PLANES; ++pl) my_stage[(pl * NS + j) * UW + p * 8 + g] = (uint16_t)pl3[pl];
+            for (int pl = 0; pl < RNN_PLANES; ++pl) my_stage[p * KBLK + (pl * NS + j) * 8 + g] = (uint16_t)pl3[pl];
           }
         }
       }
     }
-    // ---- 16-byte pieces (plane, sequence, 8 units) to every CTA of the cluster -----------------------------
+    // ---- the warp's k-blocks (8 units each: [plane][sequence][8], contiguous) to every CTA of the cluster ----
     if (send_h) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // staging writes -> visible to the bulk copies
       __syncwarp();
-      for (int idx = lane; idx < N_PIECES; idx += 32) {
-        const int row = idx / MP, p = idx - row * MP;          // row = pl * NS + j
-        const uint4 val = *reinterpret_cast<const uint4*>(my_stage + row * UW + p * 8);
-        const uint32_t off = (uint32_t)(((buf ^ 1) * HS_BUF + row * LDH + (int)rank * HU + warp * UW + p * 8) * 2);
-        // own CTA: plain store (ordered by this warp's arrive below); peers: counted remote stores
-        *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(hs) + off) = val;
 #pragma unroll
-        for (int r = 0; r < CL; ++r)
-          if (r != (int)rank) st_async_v4(hs_remote[r] + off, val, hbar_remote[r] + (buf ^ 1) * 8);
+      for (int p = 0; p < MP; ++p) {
+        const uint32_t off = (uint32_t)(((buf ^ 1) * HS_BUF + ((int)rank * (HU / 8) + warp * MP + p) * KBLK) * 2);
+        // peers: one bulk copy per k-block and peer, its bytes counted on the receiver's barrier
+        if (lane < CL && lane != (int)rank)
+          bulk_s2cluster(peer_hs + off, smem_u32(my_stage + p * KBLK), KBLK * 2, peer_bar + (buf ^ 1) * 8);
+        // own CTA: plain 16-byte stores (ordered by this warp's arrive below)
+        for (int idx = lane; idx < KBLK / 8; idx += 32)
+          *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(hs) + off + idx * 16) =
+              *reinterpret_cast<const uint4*>(my_stage + p * KBLK + idx * 8);
       }
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&hbar[buf ^ 1]);     // release: this warp's local pieces are in place
     }
+
 #pragma unroll
     for (int p = 0; p < MP; ++p)
 #pragma unroll
@@ -405,7 +413,7 @@ __global__ void __launch_bounds__(256) kve_gate_score_kernel(const float* __rest
 template <int DG, int CL, int NT>
 static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
   constexpr int NS = 8 * NT;
-  constexpr int smem = 2 * RNN_PLANES * NS * (DG + 8) * 2 + RNN_PLANES * NS * (DG / CL) * 2 + 2 * 8;
+  constexpr int smem = 2 * RNN_PLANES * NS * DG * 2 + RNN_PLANES * NS * (DG / CL) * 2 + 2 * 8;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kve_gate_rnn_kernel<DG, CL, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
