@@ -23,15 +23,15 @@ __device__ __forceinline__ void add_row(float (&acc)[8], const uint4& w) {
 __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerView v, int t0, int n_range,
                                                                         long long n_units, int final_output) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long unit = (long long)blockIdx.x * MEAN_WARPS + warp;
-  if (unit >= n_units) return;
+  // persistent warps: unit = global warp id, then strides of the whole grid
+  for (long long unit = (long long)blockIdx.x * MEAN_WARPS + warp; unit < n_units; unit += (long long)gridDim.x * MEAN_WARPS) {
   const int s = (int)(unit / n_range);
   const int t = t0 + (int)(unit - (long long)s * n_range);
   const int is_v = lane >> 4, l16 = lane & 15;
   const long long page = v.page_table[(long long)s * v.max_chunks + t];
   if (page < 0 || page >= v.n_pages) {
     if (lane == 0) set_status(v.status, ERR_CAPACITY);
-    return;
+    continue;
   }
   const uint4* src = reinterpret_cast<const uint4*>((is_v ? v.v_pages : v.k_pages) + page * v.C * D) + l16;
   float acc[8];
@@ -62,13 +62,15 @@ __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerVi
     b.w = pack_bf16x2(acc[6], acc[7]);
     *reinterpret_cast<uint4*>((is_v ? v.vsum_bf16 : v.ksum_bf16) + o) = b;
   }
+  }
 }
 
 cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, cudaStream_t st) {
   const int n_range = t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
-  const long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
+  long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
+  if (blocks > 148LL * 8) blocks = 148LL * 8;      // 64 resident warps per SM, every CTA resident from the start
   kve_chunk_mean_kernel<<<(unsigned)blocks, MEAN_WARPS * 32, 0, st>>>(v, t0, n_range, n_units, final_output ? 1 : 0);
   return cudaGetLastError();
 }
