@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(MLP_THREADS) kve_chunk_mlp_kernel(LayerView v,
 //  * Epilogue: Y + b2 -> fp32 summary and its bf16 rounding.
 // Every mbarrier wait is bounded; on give-up the status word gets KVE_ERR_TIMEOUT.
 constexpr int MT_M = 128;
-constexpr int MT_THREADS = 256;
+constexpr int MT_THREADS = 512;   // 16 warps: four per scheduler, to hide the latency of the GELU / split phases
 constexpr int MT_MAX_DSUM = 256;
 constexpr int MT_PLANE_KB_BYTES = MT_M * umma::KBLOCK_ROW_BYTES;          // 16 KB: one plane, one K-block of 64
 constexpr int MT_SMEM_A = 0;                                              // 96 KB: 3 planes x 2 K-blocks, later 2 x (3 planes x 1)
@@ -285,7 +285,7 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
   const uint32_t tmem_h = *tmem_slot, tmem_y = tmem_h + MT_TMEM_Y;
   const uint32_t idesc1 = umma::instr_desc_bf16(MT_M, d_sum), idesc2 = umma::instr_desc_bf16(MT_M, D);
   const uint32_t a_base = smem_u32(As), w1_base = smem_u32(W1s), w2_base = smem_u32(W2s);
-  const int lg = warp & 3, half = warp >> 2;
+  const int lg = warp & 3, part = warp >> 2;      // tensor-memory lanes 32 lg .., column part (0..3) of whatever is read
   const int row_in_tile = lg * 32 + lane;
   const uint32_t tmem_lane = (uint32_t)(lg * 32) << 16;
 
@@ -295,14 +295,14 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
     const long long unit0 = tile * MT_M;
     // ---- chunk means -> three bf16 planes (layer-1 A operand) ------------------------------------------
     {
-      // a thread keeps its 32-byte column pc and walks down 8 rows: all 16 loads first, then the splits
+      // a thread keeps its 32-byte column pc and walks down 4 rows: all 8 loads first, then the splits
       // (32-bit index arithmetic, one division per row; the host checks the ranges)
       const int pc = tid & 15;
       const uint32_t u0 = (uint32_t)unit0, nr = (uint32_t)n_range, total = (uint32_t)n_units;
-      float4 lo[8], hi[8];
+      float4 lo[4], hi[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const uint32_t unit = u0 + (tid >> 4) + 16 * i;
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t unit = u0 + (tid >> 4) + 32 * i;
         lo[i] = hi[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (unit < total) {
           const uint32_t s = unit / nr;
@@ -313,8 +313,8 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
         }
       }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int r = (tid >> 4) + 16 * i;
+      for (int i = 0; i < 4; ++i) {
+        const int r = (tid >> 4) + 32 * i;
         const float x[8] = {lo[i].x, lo[i].y, lo[i].z, lo[i].w, hi[i].x, hi[i].y, hi[i].z, hi[i].w};
         // plane pl, K-block kb at (pl * 2 + kb) * 16 KB
         store_split8(x, As + (pc >> 3) * MT_PLANE_KB_BYTES + umma::piece_offset(r, pc & 7), 2 * MT_PLANE_KB_BYTES);
@@ -352,15 +352,15 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
         ph_buf[buf] ^= 1;
         if (__syncthreads_or(!ok)) { failed = true; break; }
       }
-      float h[32];
-      umma::tmem_ld32(tmem_h + tmem_lane + (uint32_t)(j * 64 + half * 32), h);
+      float h[16];
+      umma::tmem_ld16(tmem_h + tmem_lane + (uint32_t)(j * 64 + part * 16), h);
       unsigned char* abuf = As + buf * 3 * MT_PLANE_KB_BYTES;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < 2; ++q) {
         float g[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) g[e] = gelu_tc(h[q * 8 + e] + b1s[j * 64 + half * 32 + q * 8 + e]);
-        store_split8(g, abuf + umma::piece_offset(row_in_tile, half * 4 + q), MT_PLANE_KB_BYTES);
+        for (int e = 0; e < 8; ++e) g[e] = gelu_tc(h[q * 8 + e] + b1s[j * 64 + part * 16 + q * 8 + e]);
+        store_split8(g, abuf + umma::piece_offset(row_in_tile, part * 2 + q), MT_PLANE_KB_BYTES);
       }
       umma::fence_smem_to_async();
       umma::fence_before_sync();
@@ -409,9 +409,8 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
         row_tab[tid] = o;
       }
       __syncthreads();
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        const int c = half * 64 + cc * 32;
+      {
+        const int c = part * 32;
         float y[32];
         umma::tmem_ld32(tmem_y + tmem_lane + (uint32_t)c, y);
 #pragma unroll
