@@ -8,6 +8,8 @@ namespace kve {
 // One thread moves 16 bytes.  idx -> (row of k_new/v_new, K-or-V, 16-byte lane within the 256-byte row).
 __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint4* __restrict__ k_new,
                                                          const uint4* __restrict__ v_new, int n_new) {
+  pdl_launch_dependents();
+  pdl_wait();
   const long long total = (long long)v.S * n_new * 32;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
@@ -30,11 +32,15 @@ __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint
 }
 
 __global__ void kve_advance_len_kernel(int32_t* seq_len, int B, int n_new) {
+  pdl_launch_dependents();
+  pdl_wait();
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) seq_len[b] += n_new;
 }
 
 __global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
+  pdl_launch_dependents();
+  pdl_wait();
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) seq_len[b] = n;
 }
@@ -44,15 +50,14 @@ cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_n
   long long blocks = (total + 255) / 256;
   if (blocks > 148LL * 32) blocks = 148LL * 32;   // grid-stride beyond 32 CTAs per SM
   if (blocks < 1) blocks = 1;
-  kve_append_kernel<<<(unsigned)blocks, 256, 0, st>>>(v, static_cast<const uint4*>(k_new),
-                                                      static_cast<const uint4*>(v_new), n_new);
-  kve_advance_len_kernel<<<(v.B + 127) / 128, 128, 0, st>>>(v.seq_len, v.B, n_new);
-  return cudaGetLastError();
+  cudaError_t e = launch_pdl(kve_append_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v, static_cast<const uint4*>(k_new),
+                             static_cast<const uint4*>(v_new), n_new);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(kve_advance_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n_new);
 }
 
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st) {
-  kve_set_len_kernel<<<(v.B + 127) / 128, 128, 0, st>>>(v.seq_len, v.B, n);
-  return cudaGetLastError();
+  return launch_pdl(kve_set_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n);
 }
 
 }  // namespace kve

@@ -93,9 +93,11 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   uint64_t* full = reinterpret_cast<uint64_t*>(comb + AT_CWARPS * ATTN_PARTIAL_FLOATS);   // 16-byte aligned
   uint64_t* empty = full + AT_STAGES;
 
+  pdl_launch_dependents();
   const LayerView& v = a.v;
   const int s = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_wait();      // lengths, keep lists and summaries come from earlier kernels
 
   int n = v.seq_len[s / v.H];
   n = min(max(n, 0), v.max_tokens);
@@ -311,8 +313,7 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_t
   a.q = static_cast<const uint16_t*>(q); a.out = static_cast<uint16_t*>(out); a.lse = lse; a.scale = scale;
   a.partials = partials; a.counters = counters;
   dim3 grid((unsigned)plan.max_splits, (unsigned)v.S);
-  kve_decode_attn_kernel<<<grid, AT_THREADS, AT_SMEM_BYTES, st>>>(a);
-  return cudaGetLastError();
+  return launch_pdl(kve_decode_attn_kernel, grid, dim3(AT_THREADS), AT_SMEM_BYTES, st, a);
 }
 
 }  // namespace kve

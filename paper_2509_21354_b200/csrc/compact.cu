@@ -9,6 +9,8 @@ namespace kve {
 constexpr int COMPACT_WARPS = 4;
 
 __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_kernel(LayerView v, int n_chunks, float tau) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int s = blockIdx.x * COMPACT_WARPS + warp;
   if (s >= v.S) return;
@@ -27,8 +29,7 @@ __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_kernel(LayerVi
 }
 
 cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStream_t st) {
-  kve_compact_kernel<<<(v.S + COMPACT_WARPS - 1) / COMPACT_WARPS, COMPACT_WARPS * 32, 0, st>>>(v, n_chunks, tau);
-  return cudaGetLastError();
+  return launch_pdl(kve_compact_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), 0, st, v, n_chunks, tau);
 }
 
 }  // namespace kve

@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(PJ_THREADS, 1) kve_gate_proj_kernel(LayerView 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + PJ_SMEM_BAR + 8);
   float* stg = reinterpret_cast<float*>(smem + PJ_SMEM_STG) + (threadIdx.x >> 5) * 1024;
 
+  pdl_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int col0 = blockIdx.x * PJ_N;
   const long long n_tiles = (n_rows + PJ_M - 1) / PJ_M;
@@ -125,6 +126,7 @@ __global__ void __launch_bounds__(PJ_THREADS, 1) kve_gate_proj_kernel(LayerView 
     }
   };
 
+  pdl_wait();      // the weight slice is on its way; the summaries come from the previous kernel
   long long tile = blockIdx.y;
   if (tile < n_tiles) gather_a(tile);
   cp_async_wait_all();
@@ -183,8 +185,7 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
   if (row_ctas > n_tiles) row_ctas = n_tiles;
   if (row_ctas < 1) row_ctas = 1;
   dim3 grid((unsigned)col_slices, (unsigned)row_ctas);
-  kve_gate_proj_kernel<<<grid, PJ_THREADS, PJ_SMEM_BYTES, st>>>(v, t0, n_range, n_rows, W_ih, b_ih, b_hh, n_cols, P);
-  return cudaGetLastError();
+  return launch_pdl(kve_gate_proj_kernel, grid, dim3(PJ_THREADS), PJ_SMEM_BYTES, st, v, t0, n_range, n_rows, W_ih, b_ih, b_hh, n_cols, P);
 }
 
 }  // namespace kve

@@ -152,6 +152,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   const int seq0 = cid * NS;
   uint16_t* my_stage = stage + warp * STG_WARP;
 
+  pdl_launch_dependents();
   if (tid == 0) {
     mbar_init(&hbar[0], 1 + RNN_WARPS); mbar_init(&hbar[1], 1 + RNN_WARPS);
     mbar_fence_init();
@@ -171,6 +172,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     }
   }
 
+  pdl_wait();      // W_hh is in registers; the carried state and P come from earlier kernels
   // ---- initial state: every CTA needs the full h of its sequences as planes in buffer 0 -------------
   for (int i = tid; i < NS * (DG / 2); i += RNN_THREADS) {
     const int j = i / (DG / 2), k2 = i % (DG / 2);
@@ -391,6 +393,8 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
 __global__ void __launch_bounds__(256) kve_gate_score_kernel(const float* __restrict__ P, const float* __restrict__ w_s,
                                                              float b_s, float* __restrict__ scores, long long n_rows,
                                                              int n_range, int t0, int max_chunks, int d_g) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= n_rows) return;
@@ -421,8 +425,7 @@ static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
     attr_set = true;
   }
   const int clusters = (a.S + NS - 1) / NS;
-  kve_gate_rnn_kernel<DG, CL, NT><<<clusters * CL, RNN_THREADS, smem, st>>>(a);
-  return cudaGetLastError();
+  return launch_pdl(kve_gate_rnn_kernel<DG, CL, NT>, dim3(clusters * CL), dim3(RNN_THREADS), smem, st, a);
 }
 
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
@@ -442,9 +445,8 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
   }
   if (e != cudaSuccess) return e;
   const long long n_rows = (long long)v.S * a.n_range;
-  kve_gate_score_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(P, w_s, b_s, v.scores, n_rows, a.n_range, t0,
-                                                                      v.max_chunks, d_g);
-  return cudaGetLastError();
+  return launch_pdl(kve_gate_score_kernel, dim3((unsigned)((n_rows + 7) / 8)), dim3(256), 0, st, (const float*)P, w_s, b_s, v.scores, n_rows,
+                    a.n_range, t0, v.max_chunks, d_g);
 }
 
 }  // namespace kve

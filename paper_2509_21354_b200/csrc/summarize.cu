@@ -22,6 +22,8 @@ __device__ __forceinline__ void add_row(float (&acc)[8], const uint4& w) {
 
 __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerView v, int t0, int n_range,
                                                                         long long n_units, int final_output) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // persistent warps: unit = global warp id, then strides of the whole grid
   for (long long unit = (long long)blockIdx.x * MEAN_WARPS + warp; unit < n_units; unit += (long long)gridDim.x * MEAN_WARPS) {
@@ -71,8 +73,7 @@ cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_out
   if (n_units <= 0) return cudaSuccess;
   long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
   if (blocks > 148LL * 8) blocks = 148LL * 8;      // 64 resident warps per SM, every CTA resident from the start
-  kve_chunk_mean_kernel<<<(unsigned)blocks, MEAN_WARPS * 32, 0, st>>>(v, t0, n_range, n_units, final_output ? 1 : 0);
-  return cudaGetLastError();
+  return launch_pdl(kve_chunk_mean_kernel, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units, final_output ? 1 : 0);
 }
 
 // ---- aggregator MLP (Eq. 2 read as mean -> d_sum -> d, exact-erf GELU), fp32 FMA ------------------
@@ -91,6 +92,8 @@ __device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8]) {
 
 __global__ void __launch_bounds__(MLP_THREADS) kve_chunk_mlp_kernel(LayerView v, int t0, int n_range, long long n_units,
                                                                    MlpWeights w, int d_sum) {
+  pdl_launch_dependents();
+  pdl_wait();
   extern __shared__ __align__(16) float smem[];
   float* Xs = smem;                    // [MLP_ROWS][128]
   float* Hs = smem + MLP_ROWS * D;     // [MLP_ROWS][d_sum]
@@ -245,6 +248,7 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
   uint64_t* bar_buf = bar_h + 1;                                            // [2]: slice MMAs that read buffer b done
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + MT_SMEM_BAR + 32);
 
+  pdl_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int side = blockIdx.y;
   const uint16_t* W1 = side ? w.W1V : w.W1K;
@@ -289,6 +293,7 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
   const int row_in_tile = lg * 32 + lane;
   const uint32_t tmem_lane = (uint32_t)(lg * 32) << 16;
 
+  pdl_wait();      // weights, barriers and tensor memory are set up; the chunk means come from the previous kernel
   uint32_t ph_h = 0, ph_buf[2] = {0, 0};
   bool failed = false;
   for (long long tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
@@ -459,8 +464,7 @@ cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeight
     const long long n_tiles = (n_units + MT_M - 1) / MT_M;
     const long long per_side = n_tiles < 74 ? n_tiles : 74;      // one CTA per SM: half of the 148 SMs per side
     dim3 grid((unsigned)per_side, 2);
-    kve_chunk_mlp_tc_kernel<<<grid, MT_THREADS, MT_SMEM_BYTES, st>>>(v, t0, n_range, n_units, w, d_sum);
-    return cudaGetLastError();
+    return launch_pdl(kve_chunk_mlp_tc_kernel, grid, dim3(MT_THREADS), MT_SMEM_BYTES, st, v, t0, n_range, n_units, w, d_sum);
   }
   const size_t smem = sizeof(float) * (size_t)MLP_ROWS * (D + d_sum);
   static bool attr_set = false;
@@ -471,8 +475,7 @@ cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeight
     attr_set = true;
   }
   dim3 grid((unsigned)((n_units + MLP_ROWS - 1) / MLP_ROWS), 2);
-  kve_chunk_mlp_kernel<<<grid, MLP_THREADS, smem, st>>>(v, t0, n_range, n_units, w, d_sum);
-  return cudaGetLastError();
+  return launch_pdl(kve_chunk_mlp_kernel, grid, dim3(MLP_THREADS), smem, st, v, t0, n_range, n_units, w, d_sum);
 }
 
 }  // namespace kve
