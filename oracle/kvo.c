@@ -18,6 +18,7 @@
  *   kvo_summarize   Sec. 3.2, Eq. 2 (aggregator; mean / mean->2-layer MLP / identity)
  *   kvo_gate        Sec. 3.2, Eq. 3 (LSTM over chunk summaries, score s_t in [0,1])
  *   kvo_compact     Sec. 3.2 retention rule "s_t >= tau"
+ *   kvo_reclaim     Sec. 3.3 memory reduction: pages of gated chunks handed back
  *   kvo_attn        Sec. 3.3 attention over window + retained chunks, with Eq. 1 as the softmax
  *   kvo_attn_dense  Eq. 1 over the full cache (the baseline of Sec. 3.3)
  *
@@ -223,6 +224,38 @@ int kvo_compact(const real* scores, int S, int stride, int n_chunks, double tau,
     for (int t = m; t < stride; ++t) keep_idx[(size_t)s * stride + t] = -1;
   }
   return 0;
+}
+
+/* ---- Sec. 3.3 / Sec. 4.2: the memory side of the method --------------------------------------- */
+/*
+ * Once a chunk has been summarised and gated, its raw tokens are no longer needed: a discarded
+ * chunk is never attended to again, and a retained chunk is attended to through its one summary
+ * row (n' = W + M rows instead of n, the memory ratio n / (W + M) of Sec. 3.3).  This returns the
+ * pages of such chunks to the caller.
+ *
+ * page_table  [S][stride] page id of chunk t of sequence s; entries handed back become -1
+ * scores      [S][stride]; chunk t is discarded iff scores < tau (the complement of kvo_compact)
+ * chunks      t in [t0, t1)
+ * mode        0: only discarded chunks give their page back (valid whatever attention reads)
+ *             1: every chunk in the range does (valid when retained chunks are read as summaries)
+ * free_list   receives the page ids, sequences in order, chunks ascending within a sequence;
+ *             entries already -1 are skipped.  Returns the number written, or -1 on a bad argument.
+ */
+long kvo_reclaim(int32_t* page_table, const real* scores, int S, int stride, int t0, int t1,
+                 double tau, int mode, int32_t* free_list) {
+  if (S < 0 || t0 < 0 || t1 < t0 || t1 > stride || (mode != 0 && mode != 1)) return -1;
+  const real tr = (real)tau;
+  long m = 0;
+  for (int s = 0; s < S; ++s)
+    for (int t = t0; t < t1; ++t) {
+      const size_t i = (size_t)s * stride + t;
+      const int discarded = !(scores[i] >= tr);
+      if ((mode == 1 || discarded) && page_table[i] >= 0) {
+        free_list[m++] = page_table[i];
+        page_table[i] = -1;
+      }
+    }
+  return m;
 }
 
 /* ---- Eq. 1 over an explicit row list ------------------------------------------------------ */

@@ -116,6 +116,20 @@ class Oracle:
             raise ValueError(f"kvo_compact rc={rc}")
         return keep_idx, keep_cnt
 
+    # -- Sec. 3.3 memory reduction: pages of gated chunks handed back --
+    def reclaim(self, page_table, scores, t0, t1, tau, mode):
+        """page_table [S, stride] int32 is edited in place (-1 where a page was handed back);
+        returns the free list (int32 array) in sequence-major, chunk-ascending order."""
+        S, stride = scores.shape
+        assert page_table.shape == (S, stride) and page_table.dtype == np.int32 and page_table.flags.c_contiguous
+        free = np.empty((S * max(t1 - t0, 0) + 1,), np.int32)
+        self.lib.kvo_reclaim.restype = C.c_long
+        m = self.lib.kvo_reclaim(_ptr(page_table, _i32p), _ptr(scores, self._realp), C.c_int(S), C.c_int(stride),
+                                 C.c_int(t0), C.c_int(t1), C.c_double(float(tau)), C.c_int(mode), _ptr(free, _i32p))
+        if m < 0:
+            raise ValueError(f"kvo_reclaim rc={m}")
+        return free[:m].copy()
+
     # -- Sec. 3.3 attention over window + retained chunks --
     def attn(self, q, K, V, Cs, n_chunks, keep_idx, keep_cnt, ksum_b16, vsum_b16, attend, scale):
         S, n, d = K.shape

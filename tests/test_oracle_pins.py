@@ -458,3 +458,44 @@ def test_pipeline_config1_shapes_and_counts(o32, o64):
         res[o.kind] = (sc, out)
     assert np.abs(res["f32"][0] - res["f64"][0]).max() < 1e-5
     assert np.abs(res["f32"][1] - res["f64"][1]).max() < 1e-5
+
+
+# ---- Sec. 3.3 memory reduction: pages of gated chunks handed back ---------------------------------
+def test_reclaim_is_the_complement_of_the_retention_rule_and_conserves_pages(o64, o32):
+    rng = np.random.default_rng(3)
+    S, stride, Nc, tau = 5, 12, 9, 0.5
+    for o in (o64, o32):
+        scores = rng.random((S, stride)).astype(o.real)
+        scores[0, 0] = tau                      # equality is retained (Sec. 3.2), hence NOT handed back in mode 0
+        pages = rng.permutation(S * stride).astype(np.int32).reshape(S, stride)
+        idx, cnt = o.compact(scores, Nc, tau)
+        pt = pages.copy()
+        free = o.reclaim(pt, scores, 0, Nc, tau, 0)
+        # brute force: every gated chunk not in the keep list, sequence-major, ascending
+        want = [pages[s, t] for s in range(S) for t in range(Nc) if t not in set(idx[s, :cnt[s]].tolist())]
+        assert free.tolist() == want and pages[0, 0] not in free
+        assert len(free) == S * Nc - int(cnt.sum())
+        for s in range(S):
+            for t in range(stride):
+                kept_or_ungated = t >= Nc or t in idx[s, :cnt[s]]
+                assert pt[s, t] == (pages[s, t] if kept_or_ungated else -1)
+        # nothing is lost or duplicated; a second call finds nothing left
+        assert sorted(free.tolist() + pt[pt >= 0].tolist()) == sorted(pages.ravel().tolist())
+        assert len(o.reclaim(pt, scores, 0, Nc, tau, 0)) == 0
+        # mode 1 (retained chunks live on as summaries): the rest of the gated range follows, window chunks never
+        rest = o.reclaim(pt, scores, 0, Nc, tau, 1)
+        assert sorted(rest.tolist()) == sorted(pages[s, t] for s in range(S) for t in range(Nc) if pt[s, t] == -1 and pages[s, t] not in free)
+        assert (pt[:, :Nc] == -1).all() and np.array_equal(pt[:, Nc:], pages[:, Nc:])
+        # the memory ratio of Sec. 3.3: n / (W + M) rows remain addressable per sequence
+        assert len(free) + len(rest) == S * Nc
+
+
+def test_reclaim_ranges_and_bad_arguments(o64):
+    scores = np.zeros((2, 6), np.float64)          # everything discarded at tau = 0.5
+    pt = np.arange(12, dtype=np.int32).reshape(2, 6)
+    assert o64.reclaim(pt, scores, 2, 4, 0.5, 0).tolist() == [2, 3, 8, 9]
+    assert o64.reclaim(pt, scores, 0, 6, 0.5, 0).tolist() == [0, 1, 4, 5, 6, 7, 10, 11]
+    with pytest.raises(ValueError):
+        o64.reclaim(pt, scores, 0, 7, 0.5, 0)
+    with pytest.raises(ValueError):
+        o64.reclaim(pt, scores, 0, 6, 0.5, 2)
