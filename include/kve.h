@@ -65,7 +65,7 @@ typedef struct {
   void* k_pages;        /* bf16 [n_pages][C][d]: one page = one chunk of one (layer, b, h) */
   void* v_pages;        /* bf16 [n_pages][C][d] */
   int64_t n_pages;
-  int32_t* page_table;  /* [n_layers][S][max_chunks] page ids, filled by the caller */
+  int32_t* page_table;  /* [n_layers][S][max_chunks] page ids, filled by the caller; kvE_reclaim_pages writes -1 */
   int32_t* seq_len;     /* [n_layers][B] tokens stored; written by kvE_append / kvE_set_len */
   float* ksum_f32;      /* [n_layers][S][max_chunks][d] chunk summaries, fp32 */
   float* vsum_f32;
@@ -132,6 +132,22 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
 /* Sec. 3.2 retention rule: keep chunk t iff scores[t] >= tau, over all gated chunks of `layer`;
  * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw. */
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream);
+
+/* Sec. 3.3 (n' = W + M, memory ratio n / (W + M)) and the KV-memory reduction of Sec. 4.2: hand the pages
+ * of gated chunks back to the caller.  Chunks [chunk_begin, chunk_end) of every sequence of `layer` must
+ * be covered by the keep list (kvE_compact; its tau decides "discarded").
+ *   mode KVE_RECLAIM_DISCARDED: pages of chunks with s_t < tau (never attended to again);
+ *   mode KVE_RECLAIM_GATED:     pages of all chunks in the range; needs cfg.attend == KVE_ATTEND_SUMMARY,
+ *                               where a retained chunk is read through its one summary row.
+ * free_list: DEVICE int32 [capacity], receives the page ids, sequences in order, chunks ascending;
+ * free_count: DEVICE int32, receives how many.  The page_table entries handed back become -1 (the
+ * library writes the caller's page table here); entries that are already -1 are skipped.  If the
+ * list would not fit, nothing is handed back, *free_count is 0 and the status word gets
+ * KVE_ERR_CAPACITY.  Afterwards the raw rows of those chunks are gone: summarising them again or
+ * kvE_decode_attn_dense flags KVE_ERR_CAPACITY in the status word instead of reading them. */
+enum { KVE_RECLAIM_DISCARDED = 0, KVE_RECLAIM_GATED = 1 };
+int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, int mode, int32_t* free_list,
+                      int64_t capacity, int32_t* free_count, void* stream);
 
 /* Sec. 3.3 + Eq. 1: out = softmax(q K'^T * scale) V' over [kept chunks ; raw tail] of `layer`.
  * q, out: DEVICE bf16 [S][d]; lse: DEVICE fp32 [S] or NULL (log-sum-exp of the scaled logits). */

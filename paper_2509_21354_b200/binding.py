@@ -23,7 +23,7 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_decode_attn", "kvE_decode_attn_dense",
-           "kvE_decode_attn_static", "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
+           "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense"]
 
@@ -83,6 +83,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
     lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
     lib.kvE_decode_attn_static.argtypes = lib.kvE_decode_attn.argtypes
+    lib.kvE_reclaim_pages.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
     lib.kvE_decode_step_host.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float,
                                          C.c_float, C.c_int, C.c_void_p]
@@ -247,6 +248,9 @@ class Store:
     def decode_attn_dense(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)
 
+    def reclaim_pages(self, layer, chunk_begin, chunk_end, mode="discarded", free_list=None, free_count=None, stream=None):
+        return kvE_reclaim_pages(self, layer, chunk_begin, chunk_end, mode, free_list, free_count, stream)
+
     def decode_attn_static(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_static(self, layer, q, out, lse, scale, stream)
 
@@ -311,6 +315,24 @@ def kvE_decode_attn(st: Store, layer, q, out=None, lse=None, scale=None, stream=
 
 def kvE_decode_attn_dense(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):
     return _attn("kvE_decode_attn_dense", st, layer, q, out, lse, scale, stream)
+
+
+RECLAIM = {"discarded": 0, "gated": 1}
+
+
+def kvE_reclaim_pages(st: Store, layer, chunk_begin, chunk_end, mode="discarded", free_list=None, free_count=None, stream=None):
+    """Hands pages of gated chunks back (Sec. 3.3).  free_list: int32 device tensor (its length is the
+    capacity; allocated here for the whole range if omitted), free_count: int32 device tensor [1].
+    Returns (free_list, free_count); the first free_count entries are valid once the stream has run."""
+    if free_list is None:
+        free_list = torch.empty((max(1, st.S * max(chunk_end - chunk_begin, 0)),), dtype=torch.int32, device=st.device)
+    if free_count is None:
+        free_count = torch.zeros((1,), dtype=torch.int32, device=st.device)
+    assert free_list.dtype == torch.int32 and free_count.dtype == torch.int32
+    _check("kvE_reclaim_pages", st.lib.kvE_reclaim_pages(st.handle, layer, int(chunk_begin), int(chunk_end), RECLAIM[mode],
+                                                        _p(free_list), C.c_int64(free_list.numel()), _p(free_count),
+                                                        _stream(stream)), st.handle)
+    return free_list, free_count
 
 
 def kvE_decode_attn_static(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):

@@ -16,6 +16,7 @@ struct LayerState {
   int n_summarised = 0;  // chunks [0, n_summarised) have summaries
   int n_gated = 0;       // chunks [0, n_gated) have scores; LSTM state stands after chunk n_gated-1
   int n_compacted = 0;   // keep list covers chunks [0, n_compacted); attention reads raw rows from there on
+  float tau = 0.f;       // threshold of the last kvE_compact
 };
 
 struct kvE_store {
@@ -23,7 +24,7 @@ struct kvE_store {
   kvE_buffers buf;
   int S, max_chunks;
   // workspace carve-up (byte offsets)
-  size_t off_P, off_partials, off_counters, off_stage, ws_needed;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, ws_needed;
   int max_splits;
   std::vector<LayerState> layers;
   std::string cuda_error;
@@ -56,7 +57,7 @@ int check_config(const kvE_config* c) {
 }
 
 struct Carve {
-  size_t off_P, off_partials, off_counters, off_stage, total;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, total;
 };
 Carve carve(const kvE_config& c) {
   const size_t S = (size_t)c.B * c.Hkv;
@@ -67,6 +68,7 @@ Carve carve(const kvE_config& c) {
   k.off_partials = o; o = align_up(o + S * MAX_SPLITS * ATTN_PARTIAL_FLOATS * sizeof(float));
   k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
   k.off_stage = o;    o = align_up(o + 4 * S * 128 * 2);   // k_new, v_new, q, out of kvE_decode_step_host
+  k.off_reclaim = o;  o = align_up(o + (2 * S + 1) * sizeof(int32_t));   // per-sequence counts and offsets of kvE_reclaim_pages
   k.total = o;
   return k;
 }
@@ -184,7 +186,7 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   st->S = cfg->B * cfg->Hkv;
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
   st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
-  st->off_stage = k.off_stage; st->ws_needed = k.total;
+  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->ws_needed = k.total;
   st->max_splits = MAX_SPLITS;
   st->layers.assign(cfg->n_layers, LayerState());
   cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.total - k.off_partials);
@@ -301,7 +303,26 @@ int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   cudaError_t e = launch_compact(view(st, layer), ls.n_gated, tau, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_compacted = ls.n_gated;
+  ls.tau = tau;
   return KVE_OK;
+}
+
+int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, int mode, int32_t* free_list,
+                      int64_t capacity, int32_t* free_count, void* stream) {
+  if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin || !free_list || !free_count || capacity < 0)
+    return KVE_ERR_ARG;
+  if (mode != KVE_RECLAIM_DISCARDED && mode != KVE_RECLAIM_GATED) return KVE_ERR_ARG;
+  const LayerState& ls = st->layers[layer];
+  if (chunk_end > ls.n_compacted) return KVE_ERR_STATE;                        // only chunks the retention rule has judged
+  if (mode == KVE_RECLAIM_GATED && st->cfg.attend != KVE_ATTEND_SUMMARY) return KVE_ERR_STATE;   // RAW attention still reads kept pages
+  if (chunk_end == chunk_begin) {
+    cudaError_t e = cudaMemsetAsync(free_count, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+  }
+  int32_t* scratch = reinterpret_cast<int32_t*>(static_cast<char*>(st->buf.workspace) + st->off_reclaim);
+  cudaError_t e = launch_reclaim(view(st, layer), chunk_begin, chunk_end, ls.tau, mode, scratch, free_list, capacity, free_count,
+                                 static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
 }
 
 int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {

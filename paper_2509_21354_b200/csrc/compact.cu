@@ -32,4 +32,105 @@ cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStre
   return launch_pdl(kve_compact_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), 0, st, v, n_chunks, tau);
 }
 
+// ---- kvE_reclaim_pages kernels (Sec. 3.3, memory ratio n / (W + M)): pages of gated chunks go back to the caller ----
+// A chunk gives its page back if it was discarded (score < tau) or, with mode 1, in any case (retained
+// chunks live on as their summary row).  Free-list order: sequences in order, chunks ascending, so the
+// result is unique.  count -> scan -> scatter; the scatter does nothing if the list would overflow.
+__device__ __forceinline__ bool reclaimable(const LayerView& v, int s, int t, float tau, int mode) {
+  const long long i = (long long)s * v.max_chunks + t;
+  return (mode == 1 || !(v.scores[i] >= tau)) && v.page_table[i] >= 0;
+}
+
+__global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_reclaim_count_kernel(LayerView v, int t0, int t1, float tau, int mode,
+                                                                              int32_t* counts) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s = blockIdx.x * COMPACT_WARPS + warp;
+  if (s >= v.S) return;
+  int n = 0;
+  for (int tb = t0; tb < t1; tb += 32) {
+    const int t = tb + lane;
+    n += __popc(__ballot_sync(0xffffffffu, t < t1 && reclaimable(v, s, t, tau, mode)));
+  }
+  if (lane == 0) counts[s] = n;
+}
+
+// one CTA: exclusive prefix sum of counts[0..S) -> offsets[0..S); offsets[S] = 1 if the total fits, else 0
+__global__ void __launch_bounds__(1024) kve_reclaim_scan_kernel(const int32_t* counts, int S, int32_t* offsets, long long capacity,
+                                                                int32_t* free_count, int32_t* status) {
+  pdl_launch_dependents();
+  pdl_wait();
+  __shared__ int warp_tot[32];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int per = (S + 1023) / 1024;
+  const int lo = min(S, tid * per), hi = min(S, lo + per);
+  int mine = 0;
+  for (int i = lo; i < hi; ++i) mine += counts[i];
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += x;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_tot[lane], wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += x;
+    }
+    warp_tot[lane] = wi - w;      // exclusive
+  }
+  __syncthreads();
+  int run = warp_tot[warp] + incl - mine;
+  for (int i = lo; i < hi; ++i) {
+    offsets[i] = run;
+    run += counts[i];
+  }
+  if (tid == 1023) {
+    const bool fits = (long long)run <= capacity;
+    offsets[S] = fits ? 1 : 0;
+    *free_count = fits ? run : 0;
+    if (!fits) set_status(status, ERR_CAPACITY);
+  }
+}
+
+__global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_reclaim_scatter_kernel(LayerView v, int t0, int t1, float tau, int mode,
+                                                                                const int32_t* offsets, int32_t* free_list) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s = blockIdx.x * COMPACT_WARPS + warp;
+  if (s >= v.S || offsets[v.S] == 0) return;
+  int32_t* table = const_cast<int32_t*>(v.page_table) + (long long)s * v.max_chunks;
+  int base = offsets[s];
+  for (int tb = t0; tb < t1; tb += 32) {
+    const int t = tb + lane;
+    const bool give = t < t1 && reclaimable(v, s, t, tau, mode);
+    const unsigned mask = __ballot_sync(0xffffffffu, give);
+    if (give) {
+      free_list[base + __popc(mask & ((1u << lane) - 1u))] = table[t];
+      table[t] = -1;
+    }
+    base += __popc(mask);
+  }
+}
+
+cudaError_t launch_reclaim(const LayerView& v, int t0, int t1, float tau, int mode, int32_t* scratch, int32_t* free_list,
+                           long long capacity, int32_t* free_count, cudaStream_t st) {
+  int32_t* counts = scratch;
+  int32_t* offsets = scratch + v.S;
+  const dim3 grid((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), block(COMPACT_WARPS * 32);
+  cudaError_t e = launch_pdl(kve_reclaim_count_kernel, grid, block, 0, st, v, t0, t1, tau, mode, counts);
+  if (e == cudaSuccess)
+    e = launch_pdl(kve_reclaim_scan_kernel, dim3(1), dim3(1024), 0, st, (const int32_t*)counts, v.S, offsets, capacity, free_count,
+                   v.status);
+  if (e == cudaSuccess)
+    e = launch_pdl(kve_reclaim_scatter_kernel, grid, block, 0, st, v, t0, t1, tau, mode, (const int32_t*)offsets, free_list);
+  return e;
+}
+
 }  // namespace kve

@@ -432,3 +432,63 @@ def test_sweep_points_sampled(B, n, C, keep):
         hz.check_output(b.bf16_to_bits(out[sel]), want, f"sweep {attend}")
         del st
         torch.cuda.empty_cache()
+
+
+# ---- Sec. 3.3 memory reduction: pages of gated chunks handed back ---------------------------------
+@pytest.mark.parametrize("attend,mode", [("summary", "discarded"), ("summary", "gated"), ("raw", "discarded")])
+def test_reclaim_pages_matches_oracle_and_leaves_attention_unchanged(attend, mode):
+    b = _binding()
+    wl = wlm.CFG2.small(B=2, H=8, n=2048 + 37, W=256, seed=21)       # ragged tail, MLP aggregator, 16 sequences
+    st, pb, agg_w, lstm_w = full_check(wl, attend)
+    q = b.bits_to_bf16(wlm.gen_q(wl, 0, 7))
+    before = b.bf16_to_bits(st.decode_attn(0, q))
+    table0 = st.page_table[0].cpu().numpy().copy()
+    want_table = table0.copy()
+    want_free = pb.o32.reclaim(want_table, pb.sc32.astype(np.float32), 0, pb.Nc, pb.tau, 0 if mode == "discarded" else 1)
+    # the f64 oracle takes the same decisions (scores keep their margin from tau)
+    t64 = table0.copy()
+    assert np.array_equal(pb.o64.reclaim(t64, pb.sc64, 0, pb.Nc, pb.tau, 0 if mode == "discarded" else 1), want_free)
+    free, cnt = st.reclaim_pages(0, 0, pb.Nc, mode)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    n_free = int(cnt.item())
+    assert n_free == len(want_free)
+    assert np.array_equal(free[:n_free].cpu().numpy(), want_free)                  # bit-exact, same order
+    assert np.array_equal(st.page_table[0].cpu().numpy(), want_table)
+    if mode == "gated":
+        assert n_free == st.S * pb.Nc                                               # n / (W + M): only summaries and the window remain
+    # attention never needed those pages
+    after = b.bf16_to_bits(st.decode_attn(0, q))
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0 and np.array_equal(before, after)
+    # a second call finds nothing; the dense baseline now runs into the holes and says so without faulting
+    _, cnt2 = st.reclaim_pages(0, 0, pb.Nc, mode)
+    torch.cuda.synchronize()
+    assert int(cnt2.item()) == 0
+    if n_free:
+        st.decode_attn_dense(0, q)
+        torch.cuda.synchronize()
+        assert st.poll_status() == -3
+
+
+def test_reclaim_pages_host_errors_and_overflow():
+    b = _binding()
+    wl = wlm.CFG1.small(B=1, H=4, n=1024, seed=3)
+    st, pb, _, lstm_w = full_check(wl, "raw")
+    with pytest.raises(b.KveError) as e:
+        st.reclaim_pages(0, 0, pb.Nc, "gated")                  # RAW attention still reads kept pages
+    assert e.value.rc == -4
+    with pytest.raises(b.KveError) as e:
+        st.reclaim_pages(0, 0, pb.Nc + 1, "discarded")          # beyond the keep list
+    assert e.value.rc == -4
+    table0 = st.page_table[0].clone()
+    n_disc = int(st.S * pb.Nc - st.keep_cnt[0].sum().item())
+    assert n_disc > 1
+    small = torch.empty((n_disc - 1,), dtype=torch.int32, device="cuda")
+    _, cnt = st.reclaim_pages(0, 0, pb.Nc, "discarded", free_list=small)
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == 0 and torch.equal(st.page_table[0], table0)          # nothing handed back
+    assert st.poll_status() == -3
+    _, cnt = st.reclaim_pages(0, 0, 0, "discarded")             # empty range
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == 0 and st.poll_status() == 0
