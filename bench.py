@@ -138,7 +138,7 @@ def fill_cache(st, wl, seed):
     return g
 
 
-def algorithmic_bytes(wl, Nc, keep_mean, R):
+def algorithmic_bytes(wl, Nc, keep_mean, R, attend="summary"):
     """Bytes each kernel must move per launch (per-unit figures x units; bf16 rows are 256 bytes)."""
     S, d_g = wl.S, wl.d_g
     by = {}
@@ -147,7 +147,8 @@ def algorithmic_bytes(wl, Nc, keep_mean, R):
     by["gate_proj"] = S * Nc * (2 * 256 + 4 * d_g * 4)                    # bf16 summaries in, fp32 P out
     by["gate_rnn"] = S * Nc * (4 * d_g * 4 + 4)                           # P in, scores out
     by["compact"] = S * (Nc * 4 + Nc * 4 + 4)
-    by["attn_gated"] = S * (2 * (R + keep_mean) * 256 + 2 * 256)          # retained rows of K and V once (+ q, out)
+    rows_per_kept = wl.C if attend == "raw" else 1                          # a kept chunk: its C raw rows, or its one summary row
+    by["attn_gated"] = S * (2 * (R + keep_mean * rows_per_kept) * 256 + 2 * 256)   # retained rows of K and V once (+ q, out)
     by["attn_dense"] = S * (2 * wl.n * 256 + 2 * 256)
     return by
 
@@ -289,7 +290,7 @@ def run_ours(args, rank, world, local_rank):
     us = {k: float(np.mean(v)) for k, v in in_step.items() if v}
     us["attn_dense"] = float(np.mean(cold["attn_dense"]))
     us_attn_cold = float(np.mean(cold["attn"]))
-    by = algorithmic_bytes(wl, Nc, keep_mean, R)
+    by = algorithmic_bytes(wl, Nc, keep_mean, R, args.attend)
     by_kernel = {"append": S * 4 * 256, "chunk_mean": by["chunk_mean"], "chunk_mlp": by["chunk_mlp"],
                  "gate_proj": by["gate_proj"], "gate_rnn": by["gate_rnn"], "compact": by["compact"],
                  "attn": by["attn_gated"], "attn_dense": by["attn_dense"]}
@@ -337,8 +338,8 @@ def run_ours(args, rank, world, local_rank):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "d": 128, "n": wl.n, "C": wl.C, "W": wl.W,
                    "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend, "n_layers_timed": 1,
-                   "stale_chunks": Nc, "kept_chunks_mean": keep_mean, "n_eff": R + keep_mean,
-                   "memory_ratio_n_over_n_eff": n0 / (R + keep_mean),
+                   "stale_chunks": Nc, "kept_chunks_mean": keep_mean, "n_eff": R + keep_mean * (wl.C if args.attend == "raw" else 1),
+                   "memory_ratio_n_over_n_eff": n0 / (R + keep_mean * (wl.C if args.attend == "raw" else 1)),
                    "l2": "inputs larger than L2 (each step streams 0.45 GB of stale KV + 0.06 GB window); per-kernel timings flush L2 before every launch"},
         "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * S * 256,
                 "d2h_bytes_per_step": S * 256, "matches_device_path": same},
