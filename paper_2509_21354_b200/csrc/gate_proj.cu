@@ -5,13 +5,15 @@
 // epilogue.
 //
 //  * A CTA owns one 256-column slice of W_ih^T for its whole life: the slice (128 KB, K-major,
-//    128-byte swizzle) is written to shared memory once.
-//  * It then walks over 128-row tiles of X (operand loads are cp.async copies, all in flight at
-//    once; two accumulators in tensor memory, so the MMAs of the next tile run during the epilogue).  The rows are gathered straight from the summary store
+//    128-byte swizzle) goes to shared memory once, by cp.async.
+//  * It then walks over 128-row tiles of X.  The rows are gathered straight from the summary store
 //    (columns 0..127 of a row from ksum_bf16, 128..255 from vsum_bf16) into the swizzled A tile
-//    (64 KB), one thread issues the 16 MMAs of the tile (K = 256 in steps of 16) and commits them
-//    to an mbarrier; all eight warps then read the 128 x 256 fp32 accumulator out of tensor
-//    memory (warp w: lanes 32 (w % 4) .., column half w / 4), add the bias and store P.
+//    (64 KB) by cp.async copies that are all in flight at once; one thread issues the 16 MMAs of
+//    the tile (K = 256 in steps of 16) and commits them to an mbarrier.
+//  * Two accumulators in tensor memory: while the eight warps read tile i out of one (warp w: lanes
+//    32 (w % 4) .., column half w / 4), add the bias and store P, the A tile of tile i+1 is gathered
+//    and its MMAs run into the other.  The epilogue turns each 32 x 32 block through shared memory
+//    so that a store instruction writes whole 128-byte row segments.
 //  * The only wait (on the MMA commit) is bounded; on give-up the status word gets KVE_ERR_TIMEOUT.
 #include "common.cuh"
 #include "kernels.h"
