@@ -193,6 +193,15 @@ int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const
                          const kvE_lstm_weights* lw, float tau, float scale, int from_scratch,
                          void* stream);
 
+/* The same step without the final wait: everything (copies included) is only enqueued on `stream`.
+ * The host buffers must be pinned and must stay untouched until the stream has passed this step
+ * (out_host is valid from then on); the next step may be enqueued right away, its copies and kernels
+ * queue up behind this one's. */
+int kvE_decode_step_host_async(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host,
+                               const void* q_host, void* out_host, const kvE_agg_weights* aw,
+                               const kvE_lstm_weights* lw, float tau, float scale, int from_scratch,
+                               void* stream);
+
 /* Reads *status_word (synchronises the device) into *device_status and clears it. */
 int kvE_poll_status(kvE_store* st, int* device_status);
 

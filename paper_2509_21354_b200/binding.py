@@ -23,7 +23,7 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_decode_attn", "kvE_decode_attn_dense",
-           "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
+           "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense"]
 
@@ -87,6 +87,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_decode_step_host.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float,
                                          C.c_float, C.c_int, C.c_void_p]
+    lib.kvE_decode_step_host_async.argtypes = lib.kvE_decode_step_host.argtypes
     lib.kvE_poll_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.kvE_layer_state.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_int)] * 4
     lib.kvE_profile.argtypes = [C.c_void_p, C.c_int]
@@ -255,8 +256,8 @@ class Store:
         return kvE_decode_attn_static(self, layer, q, out, lse, scale, stream)
 
     def decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale=None,
-                         from_scratch=False, stream=None):
-        kvE_decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale, from_scratch, stream)
+                         from_scratch=False, stream=None, wait=True):
+        kvE_decode_step_host(self, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale, from_scratch, stream, wait)
 
     def poll_status(self) -> int:
         return kvE_poll_status(self)
@@ -343,14 +344,18 @@ def kvE_decode_attn_static(st: Store, layer, q, out=None, lse=None, scale=None, 
 
 
 def kvE_decode_step_host(st: Store, layer, k_new, v_new, q, out, agg_weights, lstm_weights, tau, scale=None,
-                         from_scratch=False, stream=None):
-    """k_new, v_new, q, out: HOST bf16 [S, 128] tensors (pinned for asynchronous copies)."""
+                         from_scratch=False, stream=None, wait=True):
+    """k_new, v_new, q, out: HOST bf16 [S, 128] tensors (pinned for asynchronous copies).
+    wait=False calls kvE_decode_step_host_async: the step is only enqueued (pinned buffers required)."""
     for t in (k_new, v_new, q, out):
         assert not t.is_cuda and t.dtype == torch.bfloat16 and tuple(t.shape) == (st.S, 128) and t.is_contiguous()
     scale = 1.0 / np.sqrt(128.0) if scale is None else scale
     aw = C.byref(agg_weights.c) if agg_weights is not None else None
+    if not wait:
+        assert all(t.is_pinned() for t in (k_new, v_new, q, out))
+    fn = st.lib.kvE_decode_step_host if wait else st.lib.kvE_decode_step_host_async
     _check("kvE_decode_step_host",
-           st.lib.kvE_decode_step_host(st.handle, layer, C.c_void_p(k_new.data_ptr()), C.c_void_p(v_new.data_ptr()),
+           fn(st.handle, layer, C.c_void_p(k_new.data_ptr()), C.c_void_p(v_new.data_ptr()),
                                        C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), aw,
                                        C.byref(lstm_weights.c), C.c_float(tau), C.c_float(scale),
                                        1 if from_scratch else 0, _stream(stream)), st.handle)

@@ -336,9 +336,9 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
   return run_attention(st, layer, ATTN_DENSE, q, out, lse, scale, static_cast<cudaStream_t>(stream));
 }
 
-int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host, const void* q_host,
-                         void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
-                         int from_scratch, void* stream) {
+static int decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host, const void* q_host,
+                            void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
+                            int from_scratch, void* stream, bool wait) {
   if (bad_layer(st, layer) || !k_new_host || !v_new_host || !q_host || !out_host || !lw) return KVE_ERR_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t row_bytes = (size_t)st->S * 128 * 2;
@@ -369,8 +369,20 @@ int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const
   rc = kvE_decode_attn(st, layer, dq, dout, nullptr, scale, stream);
   if (rc != KVE_OK) return rc;
   e = cudaMemcpyAsync(out_host, dout, row_bytes, cudaMemcpyDeviceToHost, s);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess && wait) e = cudaStreamSynchronize(s);
   return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+}
+
+int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host, const void* q_host,
+                         void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
+                         int from_scratch, void* stream) {
+  return decode_step_host(st, layer, k_new_host, v_new_host, q_host, out_host, aw, lw, tau, scale, from_scratch, stream, true);
+}
+
+int kvE_decode_step_host_async(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host, const void* q_host,
+                               void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
+                               int from_scratch, void* stream) {
+  return decode_step_host(st, layer, k_new_host, v_new_host, q_host, out_host, aw, lw, tau, scale, from_scratch, stream, false);
 }
 
 int kvE_poll_status(kvE_store* st, int* device_status) {

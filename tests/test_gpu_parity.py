@@ -278,6 +278,16 @@ def test_decode_step_host_matches_stepwise_calls():
     want, _, _, _ = pb0.oracle_attn(q, "summary")
     hz.check_output(b.bf16_to_bits(out), want, "step_host")
     check_gate_and_keep(st, pb0)
+    # the asynchronous form: two steps enqueued back to back (the second rolls the first one's token back and
+    # redoes it), nothing waited for until the stream is synchronised; same result
+    out2 = torch.zeros(wl.S, 128, dtype=torch.bfloat16).pin_memory()
+    hk, hv, hq = pin(pb0.K[:, -1]), pin(pb0.V[:, -1]), pin(q)
+    for _ in range(2):
+        st.set_len(0, 1024 - 1)
+        st.decode_step_host(0, hk, hv, hq, out2, None, lw, pb0.tau, from_scratch=True, wait=False)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    assert torch.equal(out2, out)
 
 
 def test_host_side_errors():
