@@ -4,7 +4,9 @@
 // P_t (= W_ih x_t + b_ih + b_hh) comes from the projection GEMM.
 //
 // The chain over t is strictly sequential, so the kernel is built for latency per step:
-//  * A thread-block cluster of CL CTAs owns NS = 8*NT sequences for all steps.  Each CTA owns
+//  * A thread-block cluster of CL CTAs owns NG groups of 8 sequences for all steps (NG = 2 when one
+//    group per cluster would not fit the GPU in one wave: the groups are independent pipelines, and a
+//    warp handles them one after the other, so one group's exchange overlaps the other's arithmetic).  Each CTA owns
 //    HU = d_g / CL hidden units, i.e. 4*HU rows of W_hh, and keeps them in REGISTERS as mma A
 //    fragments for the whole kernel (128 registers per thread at d_g = 256, CL = 4).
 //  * Per step the CTA computes its rows of W_hh h for all its sequences with warp-level tensor-core
@@ -123,38 +125,39 @@ __device__ __forceinline__ void split3(float x, uint32_t (&p)[3]) {
   p[2] = f32_to_bf16_bits(r2);
 }
 
-template <int DG, int CL, int NT>
+// NG independent groups of 8 sequences per cluster.  A group is one pipeline (own h buffers, barriers,
+// staging and cell state); a warp works through the groups one after the other within a step, so
+// while group A's new h is on its way between the CTAs the warp is busy with group B.
+template <int DG, int CL, int NG>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve_gate_rnn_kernel(RnnArgs a) {
   constexpr int HU = DG / CL;            // hidden units owned by this CTA
   constexpr int UW = HU / RNN_WARPS;     // hidden units per warp
   constexpr int MP = UW / 8;             // pairs of m16 tiles per warp (a pair = 8 units x 4 gates)
   constexpr int KT = DG / 16;            // k tiles
-  constexpr int NS = 8 * NT;             // sequences per cluster
+  constexpr int NS = 8;                  // sequences per group: the n of the m16n8k16 MMA
   constexpr int KBLK = RNN_PLANES * NS * 8;                     // bf16 elements of one k-block: [plane][sequence][8 units]
   constexpr int HS_BUF = (DG / 8) * KBLK;                       // bf16 elements per h buffer: [k-block][plane][sequence][8]
-  constexpr int STG_WARP = RNN_PLANES * NS * UW;                // bf16 elements of one warp's staging area
-  constexpr int N_PIECES = RNN_PLANES * NS * MP;                // 16-byte pieces a warp sends to each CTA per step
-  constexpr uint32_t H_BYTES = RNN_PLANES * NS * (DG - HU) * 2; // bytes of h planes a CTA receives from its peers per step
-  constexpr int OFF_STAGE = 2 * HS_BUF * 2;
-  constexpr int OFF_BARS = OFF_STAGE + RNN_WARPS * STG_WARP * 2;
+  constexpr int STG_WARP = MP * KBLK;                           // bf16 elements of one warp's staging area (its k-blocks)
+  constexpr uint32_t H_BYTES = RNN_PLANES * NS * (DG - HU) * 2; // bytes of h planes a CTA receives from its peers per step and group
+  constexpr int OFF_STAGE = NG * 2 * HS_BUF * 2;
+  constexpr int OFF_BARS = OFF_STAGE + NG * RNN_WARPS * STG_WARP * 2;
   static_assert(UW % 8 == 0 && MP >= 1, "8 warps x 8k hidden units per CTA");
   static_assert(OFF_STAGE % 16 == 0 && OFF_BARS % 16 == 0, "16-byte pieces");
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                          // [2][DG / 8][PLANES][NS][8]
-  uint16_t* stage = reinterpret_cast<uint16_t*>(smem_raw + OFF_STAGE);           // [warps][PLANES][NS][UW]
-  uint64_t* hbar = reinterpret_cast<uint64_t*>(smem_raw + OFF_BARS);             // [2] h planes landed
+  uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);                          // [NG][2][DG / 8][PLANES][NS][8]
+  uint16_t* stage = reinterpret_cast<uint16_t*>(smem_raw + OFF_STAGE);           // [NG][warps][MP][PLANES][NS][8]
+  uint64_t* hbar = reinterpret_cast<uint64_t*>(smem_raw + OFF_BARS);             // [NG][2] h planes landed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tig = lane & 3;
   const uint32_t rank = cluster_rank();
   const int cid = blockIdx.x / CL;
-  const int seq0 = cid * NS;
-  uint16_t* my_stage = stage + warp * STG_WARP;
+  const int seq0 = cid * NS * NG;        // group gi owns sequences seq0 + 8 gi .. + 7
 
   pdl_launch_dependents();
   if (tid == 0) {
-    mbar_init(&hbar[0], 1 + RNN_WARPS); mbar_init(&hbar[1], 1 + RNN_WARPS);
+    for (int i = 0; i < 2 * NG; ++i) mbar_init(&hbar[i], 1 + RNN_WARPS);
     mbar_fence_init();
   }
 
@@ -173,10 +176,11 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   }
 
   pdl_wait();      // W_hh is in registers; the carried state and P come from earlier kernels
-  // ---- initial state: every CTA needs the full h of its sequences as planes in buffer 0 -------------
-  for (int i = tid; i < NS * (DG / 2); i += RNN_THREADS) {
-    const int j = i / (DG / 2), k2 = i % (DG / 2);
-    const int s = seq0 + j;
+  // ---- initial state: every CTA needs the full h of its sequences as planes in buffer 0 of each group -------------
+  for (int i = tid; i < NG * NS * (DG / 2); i += RNN_THREADS) {
+    const int js = i / (DG / 2), k2 = i % (DG / 2);      // js: sequence of the cluster, 0 .. 8 NG - 1
+    const int gi = js / NS, j = js % NS;
+    const int s = seq0 + js;
     float h0 = 0.f, h1 = 0.f;
     if (!a.reset && s < a.S) {
       const float2 hv = *reinterpret_cast<const float2*>(a.lstm_h + (long long)s * DG + k2 * 2);
@@ -187,200 +191,184 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     split3(h1, p1);
 #pragma unroll
     for (int pl = 0; pl < RNN_PLANES; ++pl)
-      *reinterpret_cast<uint32_t*>(hs + (k2 >> 2) * KBLK + (pl * NS + j) * 8 + (k2 & 3) * 2) = p0[pl] | (p1[pl] << 16);
+      *reinterpret_cast<uint32_t*>(hs + gi * 2 * HS_BUF + (k2 >> 2) * KBLK + (pl * NS + j) * 8 + (k2 & 3) * 2) = p0[pl] | (p1[pl] << 16);
   }
-  float c[MP][NT][2], hlast[MP][NT][2];
+  float c[NG][MP][2], hlast[NG][MP][2];
+  float pin[NG][MP][4][2];     // P of the current step
+  const int n_cols = 4 * DG;
 #pragma unroll
-  for (int p = 0; p < MP; ++p)
+  for (int gi = 0; gi < NG; ++gi)
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+    for (int p = 0; p < MP; ++p)
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const int s = seq0 + nt * 8 + tig * 2 + e;
+        const int s = seq0 + gi * NS + tig * 2 + e;
         const int ug = (int)rank * HU + warp * UW + p * 8 + g;
         const bool live = !a.reset && s < a.S;
-        c[p][nt][e] = live ? a.lstm_c[(long long)s * DG + ug] : 0.f;
-        hlast[p][nt][e] = live ? a.lstm_h[(long long)s * DG + ug] : 0.f;
+        c[gi][p][e] = live ? a.lstm_c[(long long)s * DG + ug] : 0.f;
+        hlast[gi][p][e] = live ? a.lstm_h[(long long)s * DG + ug] : 0.f;
+        const float* prow = a.P + ((long long)s * a.n_range) * n_cols + ug;
+#pragma unroll
+        for (int gate = 0; gate < 4; ++gate) pin[gi][p][gate][e] = (s < a.S) ? __ldcs(prow + gate * DG) : 0.f;
       }
 
-  // addresses in the other CTAs that do not change from step to step
   // lane r < CL feeds peer r: that CTA's h buffers and barriers, as addresses in the cluster window
   const uint32_t peer_hs = map_to_rank(smem_u32(hs), lane < CL ? lane : 0);
   const uint32_t peer_bar = map_to_rank(smem_u32(&hbar[0]), lane < CL ? lane : 0);
-
-  const int n_cols = 4 * DG;
-  float pin[MP][NT][4][2];     // P of the current step
-#pragma unroll
-  for (int p = 0; p < MP; ++p)
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int s = seq0 + nt * 8 + tig * 2 + e;
-        const int ug = (int)rank * HU + warp * UW + p * 8 + g;
-        const float* prow = a.P + ((long long)s * a.n_range) * n_cols + ug;
-#pragma unroll
-        for (int gate = 0; gate < 4; ++gate) pin[p][nt][gate][e] = (s < a.S) ? __ldcs(prow + gate * DG) : 0.f;
-      }
 
   // barriers initialised and buffer 0 filled in every CTA before anyone sends
   cluster_sync_all();
 
   bool alive = true;
-  for (int step = 0; step < a.n_range; ++step) {
+  for (int step = 0; step < a.n_range && alive; ++step) {
     const int buf = step & 1;
     const bool send_h = step + 1 < a.n_range;
-    // this step's sends of the cluster land in buffer buf^1: announce the bytes
-    if (tid == 0 && send_h) mbar_arrive_expect_tx(&hbar[buf ^ 1], H_BYTES);
-    if (step > 0) {
-      // h_{t-1} from every CTA of the cluster (each buffer completes once per two steps)
-      if (!mbar_wait_cluster_bounded(&hbar[buf], ((step - 1) >> 1) & 1)) {
-        if (lane == 0) set_status(a.status, ERR_TIMEOUT);
-        alive = false;
-      }
-      if (!__all_sync(0xffffffffu, alive)) alive = false;
-      if (!alive) break;
+    // this step's sends of the cluster land in buffer buf^1 of each group: announce the bytes
+    if (tid == 0 && send_h) {
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) mbar_arrive_expect_tx(&hbar[2 * gi + (buf ^ 1)], H_BYTES);
     }
-
-    // ---- W_hh h_{t-1} on the tensor cores: one accumulator set per plane ---------------------------
-    float acc[RNN_PLANES][2 * MP][NT][4];
 #pragma unroll
-    for (int pl = 0; pl < RNN_PLANES; ++pl)
-#pragma unroll
-      for (int mt = 0; mt < 2 * MP; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[pl][mt][nt][e] = 0.f;
-    // B fragments: one ldmatrix.x4 brings the 8 sequences x 32 k-values of a plane (two k tiles);
-    // lane l addresses row (l & 7) of the 8 x 8 block (l >> 3).  Loaded one k-tile pair ahead.
-    const uint32_t hb_lane = smem_u32(hs + buf * HS_BUF + (lane >> 3) * KBLK + (lane & 7) * 8);
-    uint32_t bf[2][RNN_PLANES][NT][4];
-#pragma unroll
-    for (int pl = 0; pl < RNN_PLANES; ++pl)
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) ldmatrix_x4(bf[0][pl][nt], hb_lane + (uint32_t)(((pl * NS + nt * 8) * 8) * 2));
-#pragma unroll
-    for (int kp = 0; kp < KT / 2; ++kp) {
-      const int cur = kp & 1;
-      if (kp + 1 < KT / 2) {
-#pragma unroll
-        for (int pl = 0; pl < RNN_PLANES; ++pl)
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt)
-            ldmatrix_x4(bf[cur ^ 1][pl][nt], hb_lane + (uint32_t)(((kp + 1) * 4 * KBLK + (pl * NS + nt * 8) * 8) * 2));
+    for (int gi = 0; gi < NG; ++gi) {
+      uint16_t* hs_g = hs + gi * 2 * HS_BUF;
+      uint16_t* my_stage = stage + (gi * RNN_WARPS + warp) * STG_WARP;
+      uint64_t* hbar_g = hbar + 2 * gi;
+      const int seq_g = seq0 + gi * NS;
+      if (step > 0) {
+        // h_{t-1} of this group from every CTA of the cluster (each buffer completes once per two steps)
+        if (!mbar_wait_cluster_bounded(&hbar_g[buf], ((step - 1) >> 1) & 1)) {
+          if (lane == 0) set_status(a.status, ERR_TIMEOUT);
+          alive = false;
+        }
+        if (!__all_sync(0xffffffffu, alive)) alive = false;
+        if (!alive) break;
       }
+
+      // ---- W_hh h_{t-1} on the tensor cores: one accumulator set per plane ---------------------------
+      float acc[RNN_PLANES][2 * MP][4];
 #pragma unroll
-      for (int half = 0; half < 2; ++half)
+      for (int pl = 0; pl < RNN_PLANES; ++pl)
 #pragma unroll
-        for (int pl = 0; pl < RNN_PLANES; ++pl)
+        for (int mt = 0; mt < 2 * MP; ++mt)
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt)
+          for (int e = 0; e < 4; ++e) acc[pl][mt][e] = 0.f;
+      // B fragments: one ldmatrix.x4 brings the 8 sequences x 32 k-values of a plane (two k tiles);
+      // lane l addresses row (l & 7) of the 8 x 8 block (l >> 3).  Loaded one k-tile pair ahead.
+      const uint32_t hb_lane = smem_u32(hs_g + buf * HS_BUF + (lane >> 3) * KBLK + (lane & 7) * 8);
+      uint32_t bf[2][RNN_PLANES][4];
+#pragma unroll
+      for (int pl = 0; pl < RNN_PLANES; ++pl) ldmatrix_x4(bf[0][pl], hb_lane + (uint32_t)(pl * NS * 8 * 2));
+#pragma unroll
+      for (int kp = 0; kp < KT / 2; ++kp) {
+        const int cur = kp & 1;
+        if (kp + 1 < KT / 2) {
+#pragma unroll
+          for (int pl = 0; pl < RNN_PLANES; ++pl)
+            ldmatrix_x4(bf[cur ^ 1][pl], hb_lane + (uint32_t)(((kp + 1) * 4 * KBLK + pl * NS * 8) * 2));
+        }
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+          for (int pl = 0; pl < RNN_PLANES; ++pl)
 #pragma unroll
             for (int mt = 0; mt < 2 * MP; ++mt)
-              mma_bf16_16816(acc[pl][mt][nt], A[mt][2 * kp + half], bf[cur][pl][nt][2 * half], bf[cur][pl][nt][2 * half + 1]);
-    }
+              mma_bf16_16816(acc[pl][mt], A[mt][2 * kp + half], bf[cur][pl][2 * half], bf[cur][pl][2 * half + 1]);
+      }
 
-    // ---- P_{t+1} into registers while the MMAs drain ----------------------------------------------------
-    float pnext[MP][NT][4][2];
+      // ---- P_{t+1} into registers while the MMAs drain ----------------------------------------------------
+      float pnext[MP][4][2];
 #pragma unroll
-    for (int p = 0; p < MP; ++p)
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
+      for (int p = 0; p < MP; ++p)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const int s = seq0 + nt * 8 + tig * 2 + e;
+          const int s = seq_g + tig * 2 + e;
           const int ug = (int)rank * HU + warp * UW + p * 8 + g;
           const bool live = s < a.S && send_h;
           const float* prow = a.P + ((long long)s * a.n_range + step + 1) * n_cols + ug;
 #pragma unroll
-          for (int gate = 0; gate < 4; ++gate) pnext[p][nt][gate][e] = live ? __ldcs(prow + gate * DG) : 0.f;
+          for (int gate = 0; gate < 4; ++gate) pnext[p][gate][e] = live ? __ldcs(prow + gate * DG) : 0.f;
           if (s < a.S && step + 2 < a.n_range) {
 #pragma unroll
             for (int gate = 0; gate < 4; ++gate) asm volatile("prefetch.global.L2 [%0];" ::"l"(prow + n_cols + gate * DG));
           }
         }
 
-    // ---- cell update (thread-local), planes of h_t into the warp's staging area ---------------------
-    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-    __syncwarp();      // the previous step's copies have read the staging area
+      // ---- cell update (thread-local), planes of h_t into the warp's staging area ---------------------
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();      // earlier copies have read the staging areas
 #pragma unroll
-    for (int p = 0; p < MP; ++p) {
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
+      for (int p = 0; p < MP; ++p) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           float pre[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {   // q: 0 = i, 1 = f (tile 2p, rows g / g+8), 2 = g, 3 = o (tile 2p+1)
             const int mt = 2 * p + (q >> 1), ai = (q & 1) * 2 + e;
-            pre[q] = ((acc[2][mt][nt][ai] + acc[1][mt][nt][ai]) + acc[0][mt][nt][ai]) + pin[p][nt][q][e];
+            pre[q] = ((acc[2][mt][ai] + acc[1][mt][ai]) + acc[0][mt][ai]) + pin[gi][p][q][e];
           }
           const float ig = fast_sigmoid(pre[0]);
           const float fg = fast_sigmoid(pre[1]);
           const float gg = fast_tanh(pre[2]);
           const float og = fast_sigmoid(pre[3]);
-          const float cn = fmaf(fg, c[p][nt][e], ig * gg);
-          c[p][nt][e] = cn;
+          const float cn = fmaf(fg, c[gi][p][e], ig * gg);
+          c[gi][p][e] = cn;
           const float hv = og * fast_tanh(cn);
-          hlast[p][nt][e] = hv;
+          hlast[gi][p][e] = hv;
           {
             // P_t of this (unit, sequence) is consumed: its gate-0 slot carries h_t to the score kernel
-            const int sq = seq0 + nt * 8 + tig * 2 + e;
+            const int sq = seq_g + tig * 2 + e;
             if (sq < a.S) a.P[((long long)sq * a.n_range + step) * n_cols + (int)rank * HU + warp * UW + p * 8 + g] = hv;
           }
           if (send_h) {
             uint32_t pl3[3];
             split3(hv, pl3);
-            const int j = nt * 8 + tig * 2 + e;
+            const int j = tig * 2 + e;
 #pragma unroll
             for (int pl = 0; pl < RNN_PLANES; ++pl) my_stage[p * KBLK + (pl * NS + j) * 8 + g] = (uint16_t)pl3[pl];
           }
         }
       }
-    }
-    // ---- the warp's k-blocks (8 units each: [plane][sequence][8], contiguous) to every CTA of the cluster ----
-    if (send_h) {
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // staging writes -> visible to the bulk copies
-      __syncwarp();
+      // ---- the warp's k-blocks (8 units each: [plane][sequence][8], contiguous) to every CTA of the cluster ----
+      if (send_h) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // staging writes -> visible to the bulk copies
+        __syncwarp();
 #pragma unroll
-      for (int p = 0; p < MP; ++p) {
-        const uint32_t off = (uint32_t)(((buf ^ 1) * HS_BUF + ((int)rank * (HU / 8) + warp * MP + p) * KBLK) * 2);
-        // peers: one bulk copy per k-block and peer, its bytes counted on the receiver's barrier
-        if (lane < CL && lane != (int)rank)
-          bulk_s2cluster(peer_hs + off, smem_u32(my_stage + p * KBLK), KBLK * 2, peer_bar + (buf ^ 1) * 8);
-        // own CTA: plain 16-byte stores (ordered by this warp's arrive below)
-        for (int idx = lane; idx < KBLK / 8; idx += 32)
-          *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(hs) + off + idx * 16) =
-              *reinterpret_cast<const uint4*>(my_stage + p * KBLK + idx * 8);
+        for (int p = 0; p < MP; ++p) {
+          const uint32_t off = (uint32_t)(((gi * 2 + (buf ^ 1)) * HS_BUF + ((int)rank * (HU / 8) + warp * MP + p) * KBLK) * 2);
+          // peers: one bulk copy per k-block and peer, its bytes counted on the receiver's barrier
+          if (lane < CL && lane != (int)rank)
+            bulk_s2cluster(peer_hs + off, smem_u32(my_stage + p * KBLK), KBLK * 2, peer_bar + (2 * gi + (buf ^ 1)) * 8);
+          // own CTA: plain 16-byte stores (ordered by this warp's arrive below)
+          for (int idx = lane; idx < KBLK / 8; idx += 32)
+            *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(hs) + off + idx * 16) =
+                *reinterpret_cast<const uint4*>(my_stage + p * KBLK + idx * 8);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&hbar_g[buf ^ 1]);     // release: this warp's local pieces are in place
       }
-      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&hbar[buf ^ 1]);     // release: this warp's local pieces are in place
-    }
 
 #pragma unroll
-    for (int p = 0; p < MP; ++p)
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
+      for (int p = 0; p < MP; ++p)
 #pragma unroll
         for (int q = 0; q < 4; ++q)
 #pragma unroll
-          for (int e = 0; e < 2; ++e) pin[p][nt][q][e] = pnext[p][nt][q][e];
+          for (int e = 0; e < 2; ++e) pin[gi][p][q][e] = pnext[p][q][e];
+    }
   }
 
   // ---- carried state out ---------------------------------------------------------------------------
 #pragma unroll
-  for (int p = 0; p < MP; ++p)
+  for (int gi = 0; gi < NG; ++gi)
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+    for (int p = 0; p < MP; ++p)
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const int s = seq0 + nt * 8 + tig * 2 + e;
+        const int s = seq0 + gi * NS + tig * 2 + e;
         const int ug = (int)rank * HU + warp * UW + p * 8 + g;
         if (s < a.S && alive) {
-          a.lstm_c[(long long)s * DG + ug] = c[p][nt][e];
-          a.lstm_h[(long long)s * DG + ug] = hlast[p][nt][e];
+          a.lstm_c[(long long)s * DG + ug] = c[gi][p][e];
+          a.lstm_h[(long long)s * DG + ug] = hlast[gi][p][e];
         }
       }
   // nobody leaves while a peer may still be sending into its shared memory
@@ -414,18 +402,18 @@ __global__ void __launch_bounds__(256) kve_gate_score_kernel(const float* __rest
   }
 }
 
-template <int DG, int CL, int NT>
+template <int DG, int CL, int NG>
 static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
-  constexpr int NS = 8 * NT;
-  constexpr int smem = 2 * RNN_PLANES * NS * DG * 2 + RNN_PLANES * NS * (DG / CL) * 2 + 2 * 8;
+  constexpr int NS = 8 * NG;      // sequences per cluster
+  constexpr int smem = 2 * RNN_PLANES * NS * DG * 2 + RNN_PLANES * NS * (DG / CL) * 2 + NG * 2 * 8;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kve_gate_rnn_kernel<DG, CL, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(kve_gate_rnn_kernel<DG, CL, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const int clusters = (a.S + NS - 1) / NS;
-  return launch_pdl(kve_gate_rnn_kernel<DG, CL, NT>, dim3(clusters * CL), dim3(RNN_THREADS), smem, st, a);
+  return launch_pdl(kve_gate_rnn_kernel<DG, CL, NG>, dim3(clusters * CL), dim3(RNN_THREADS), smem, st, a);
 }
 
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
@@ -435,7 +423,7 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
   a.P = P; a.W_hh = W_hh; a.w_s = w_s; a.b_s = b_s;
   a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c; a.status = v.status;
   a.S = v.S; a.max_chunks = v.max_chunks; a.t0 = t0; a.n_range = t1 - t0; a.reset = reset_state ? 1 : 0;
-  // 16 sequences per cluster once 8 per cluster would need more than one wave of clusters
+  // two 8-sequence groups per cluster once one group per cluster would need more than one wave of clusters
   cudaError_t e;
   switch (d_g) {
     case 256: e = (v.S > 8 * (148 / 4)) ? launch_rnn_t<256, 4, 2>(a, st) : launch_rnn_t<256, 4, 1>(a, st); break;
