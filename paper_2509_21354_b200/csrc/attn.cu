@@ -9,8 +9,8 @@
 //    rows that are contiguous in memory into runs with a ballot, and issues one bulk copy
 //    (TMA engine, global -> shared, mbarrier byte counting) per run into a 3-stage ring of
 //    64-row K and V tiles.
-//  * four consumer warps each take 16 rows of a tile: q.k partial sums per lane (4 head dims per
-//    lane), a butterfly transpose-reduce that leaves one row's logit per lane pair, online softmax
+//  * eight consumer warps each take 8 rows of a tile: q.k partial sums per lane (4 head dims per
+//    lane), a butterfly transpose-reduce that leaves one row's logit per group of four lanes, online softmax
 //    with warp shuffles, then p.V with each lane owning 4 output dims.
 //  * per-CTA (m, l, acc) partials go to the workspace; the last CTA of a sequence to finish (atomic
 //    ticket, nobody spins) merges them by log-sum-exp and writes the bf16 output.
@@ -22,12 +22,12 @@ namespace kve {
 
 constexpr int AT_TILE = ATTN_TILE_ROWS;       // rows per stage
 constexpr int AT_STAGES = 3;
-constexpr int AT_CWARPS = 4;                  // consumer warps
-constexpr int AT_SUB = AT_TILE / AT_CWARPS;   // 16 rows per consumer warp per tile
+constexpr int AT_CWARPS = 8;                  // consumer warps
+constexpr int AT_SUB = AT_TILE / AT_CWARPS;   // 8 rows per consumer warp per tile
 constexpr int AT_THREADS = (AT_CWARPS + 1) * 32;
 constexpr int AT_STAGE_ELEMS = AT_TILE * D;   // bf16 elements of one K (or V) tile
 constexpr int AT_SMEM_BYTES = 2 * AT_STAGES * AT_STAGE_ELEMS * 2 + AT_CWARPS * ATTN_PARTIAL_FLOATS * 4 + 2 * AT_STAGES * 8 + 16;
-static_assert(AT_SUB == 16, "the transpose-reduce below is written for 16 rows per warp");
+static_assert(AT_SUB == 8, "the transpose-reduce below is written for 8 rows per warp");
 
 int attn_smem_bytes() { return AT_SMEM_BYTES; }
 
@@ -210,22 +210,22 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
           part[r] = fmaf(qf[2], bf16lo(w.y), part[r]);
           part[r] = fmaf(qf[3], bf16hi(w.y), part[r]);
         }
-        KVE_TR_ROUND(16, 8)
-        KVE_TR_ROUND(8, 4)
-        KVE_TR_ROUND(4, 2)
-        KVE_TR_ROUND(2, 1)
-        const float dot = part[0] + __shfl_xor_sync(0xffffffffu, part[0], 1);   // row (lane >> 1), full sum
-        const float logit = ((lane >> 1) < nvalid) ? dot * sl2 : -INFINITY;
+        KVE_TR_ROUND(16, 4)
+        KVE_TR_ROUND(8, 2)
+        KVE_TR_ROUND(4, 1)
+        float dot = part[0] + __shfl_xor_sync(0xffffffffu, part[0], 2);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 1);                             // row (lane >> 2), full sum
+        const float logit = ((lane >> 2) < nvalid) ? dot * sl2 : -INFINITY;
         const float m_new = fmaxf(m, warp_max(logit));
         const float p = exp2f(logit - m_new);
         const float alpha = exp2f(m - m_new);
-        l = fmaf(l, alpha, 0.5f * warp_sum(p));     // every row sits on two lanes
+        l = fmaf(l, alpha, 0.25f * warp_sum(p));    // every row sits on four lanes
         m = m_new;
 #pragma unroll
         for (int x = 0; x < 4; ++x) acc[x] *= alpha;
 #pragma unroll
         for (int r = 0; r < AT_SUB; ++r) {
-          const float pr = __shfl_sync(0xffffffffu, p, 2 * r);
+          const float pr = __shfl_sync(0xffffffffu, p, 4 * r);
           if (r < nvalid) {
             const uint2 w = *reinterpret_cast<const uint2*>(vt + r * D);
             acc[0] = fmaf(pr, bf16lo(w.x), acc[0]);
