@@ -34,7 +34,7 @@ METRIC = "gated_decode_attention_steps_per_sec"
 UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 SCALE = 1.0 / math.sqrt(128.0)
-KERNELS_PER_STEP = 10  # set_len, append (copy + length), chunk mean, chunk MLP, gate projection, gate recurrence, score head, compact, attention
+KERNELS_PER_STEP = 9   # set_len, append, chunk mean, chunk MLP, gate projection, gate recurrence, score head, compact, attention
 
 
 def load_peaks():

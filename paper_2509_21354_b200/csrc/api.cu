@@ -215,7 +215,7 @@ int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, i
   if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   if (n_new > 0) {
     Prof prof(st, KVE_K_APPEND, static_cast<cudaStream_t>(stream));
-    cudaError_t e = launch_append(view(st, layer), k_new, v_new, n_new, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_append(view(st, layer), k_new, v_new, n_new, ls.n_tokens, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(st, e);
     ls.n_tokens += n_new;
   }

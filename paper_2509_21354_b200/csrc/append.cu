@@ -6,8 +6,10 @@
 namespace kve {
 
 // One thread moves 16 bytes.  idx -> (row of k_new/v_new, K-or-V, 16-byte lane within the 256-byte row).
+// pos0 = tokens stored before the call (the handle tracks it on the host, so no device read sits in
+// front of the page-table look-up); the first threads also publish the new length.
 __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint4* __restrict__ k_new,
-                                                         const uint4* __restrict__ v_new, int n_new) {
+                                                         const uint4* __restrict__ v_new, int n_new, int pos0) {
   pdl_launch_dependents();
   pdl_wait();
   const long long total = (long long)v.S * n_new * 32;
@@ -18,8 +20,7 @@ __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint
     const long long row = idx >> 5;              // s * n_new + i
     const int s = (int)(row / n_new);
     const int i = (int)(row - (long long)s * n_new);
-    const int b = s / v.H;
-    const int pos = v.seq_len[b] + i;
+    const int pos = pos0 + i;
     if (pos < 0 || pos >= v.max_tokens) { set_status(v.status, ERR_CAPACITY); continue; }
     const int chunk = pos / v.C;
     const int r = pos - chunk * v.C;
@@ -29,13 +30,8 @@ __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint
     const uint4* src = (is_v ? v_new : k_new) + row * 16 + lane16;
     *dst = __ldg(src);
   }
-}
-
-__global__ void kve_advance_len_kernel(int32_t* seq_len, int B, int n_new) {
-  pdl_launch_dependents();
-  pdl_wait();
-  int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < B) seq_len[b] += n_new;
+  if (blockIdx.x == 0)
+    for (int b = threadIdx.x; b < v.B; b += blockDim.x) v.seq_len[b] = pos0 + n_new;
 }
 
 __global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
@@ -45,15 +41,13 @@ __global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
   if (b < B) seq_len[b] = n;
 }
 
-cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st) {
+cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, int pos0, cudaStream_t st) {
   const long long total = (long long)v.S * n_new * 32;
   long long blocks = (total + 255) / 256;
   if (blocks > 148LL * 32) blocks = 148LL * 32;   // grid-stride beyond 32 CTAs per SM
   if (blocks < 1) blocks = 1;
-  cudaError_t e = launch_pdl(kve_append_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v, static_cast<const uint4*>(k_new),
-                             static_cast<const uint4*>(v_new), n_new);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(kve_advance_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n_new);
+  return launch_pdl(kve_append_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v, static_cast<const uint4*>(k_new),
+                    static_cast<const uint4*>(v_new), n_new, pos0);
 }
 
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st) {

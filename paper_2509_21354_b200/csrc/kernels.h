@@ -41,7 +41,7 @@ struct AttnPlan {
 constexpr int ATTN_TILE_ROWS = 64;
 constexpr int ATTN_PARTIAL_FLOATS = 132;       // acc[128], m, l, 2 pad: keeps every record 16-byte aligned
 
-cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st);
+cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, int pos0, cudaStream_t st);
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st);
 cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, cudaStream_t st);
 cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st);
