@@ -18,6 +18,7 @@
  *   kvo_summarize   Sec. 3.2, Eq. 2 (aggregator; mean / mean->2-layer MLP / identity)
  *   kvo_gate        Sec. 3.2, Eq. 3 (LSTM over chunk summaries, score s_t in [0,1])
  *   kvo_compact     Sec. 3.2 retention rule "s_t >= tau"
+ *   kvo_compact_topk  the top-k gating variant (Sec. 5 names gating strategies as an ablation)
  *   kvo_reclaim     Sec. 3.3 memory reduction: pages of gated chunks handed back
  *   kvo_attn        Sec. 3.3 attention over window + retained chunks, with Eq. 1 as the softmax
  *   kvo_attn_dense  Eq. 1 over the full cache (the baseline of Sec. 3.3)
@@ -220,6 +221,30 @@ int kvo_compact(const real* scores, int S, int stride, int n_chunks, double tau,
     int m = 0;
     for (int t = 0; t < n_chunks; ++t)
       if (scores[(size_t)s * stride + t] >= tr) keep_idx[(size_t)s * stride + m++] = t;
+    keep_cnt[s] = m;
+    for (int t = m; t < stride; ++t) keep_idx[(size_t)s * stride + t] = -1;
+  }
+  return 0;
+}
+
+/* ---- gating-strategy variant (Sec. 5, planned ablation): keep the k best chunks instead of thresholding ---- */
+/*
+ * keep chunk t iff fewer than k chunks rank before it, where u ranks before t when s_u > s_t, or
+ * s_u == s_t and u < t (equal scores: the older chunk first, which makes the result unique).
+ * Output as kvo_compact: ascending ids, count, -1 padding.  k <= 0 keeps nothing, k >= n_chunks all.
+ */
+int kvo_compact_topk(const real* scores, int S, int stride, int n_chunks, int k,
+                     int32_t* keep_idx, int32_t* keep_cnt) {
+  if (S < 0 || n_chunks < 0 || n_chunks > stride) return -1;
+  for (int s = 0; s < S; ++s) {
+    const real* sc = scores + (size_t)s * stride;
+    int m = 0;
+    for (int t = 0; t < n_chunks; ++t) {
+      int before = 0;
+      for (int u = 0; u < n_chunks; ++u)
+        if (sc[u] > sc[t] || (sc[u] == sc[t] && u < t)) ++before;
+      if (before < k) keep_idx[(size_t)s * stride + m++] = t;
+    }
     keep_cnt[s] = m;
     for (int t = m; t < stride; ++t) keep_idx[(size_t)s * stride + t] = -1;
   }

@@ -116,6 +116,17 @@ class Oracle:
             raise ValueError(f"kvo_compact rc={rc}")
         return keep_idx, keep_cnt
 
+    # -- gating variant: keep the k highest-scoring chunks (ties: older chunk first) --
+    def compact_topk(self, scores, n_chunks, k):
+        S, stride = scores.shape
+        keep_idx = np.full((S, stride), -1, np.int32)
+        keep_cnt = np.zeros((S,), np.int32)
+        rc = self.lib.kvo_compact_topk(_ptr(scores, self._realp), C.c_int(S), C.c_int(stride), C.c_int(n_chunks),
+                                       C.c_int(int(k)), _ptr(keep_idx, _i32p), _ptr(keep_cnt, _i32p))
+        if rc != 0:
+            raise ValueError(f"kvo_compact_topk rc={rc}")
+        return keep_idx, keep_cnt
+
     # -- Sec. 3.3 memory reduction: pages of gated chunks handed back --
     def reclaim(self, page_table, scores, t0, t1, tau, mode):
         """page_table [S, stride] int32 is edited in place (-1 where a page was handed back);

@@ -499,3 +499,36 @@ def test_reclaim_ranges_and_bad_arguments(o64):
         o64.reclaim(pt, scores, 0, 7, 0.5, 0)
     with pytest.raises(ValueError):
         o64.reclaim(pt, scores, 0, 6, 0.5, 2)
+
+
+# ---- gating variant: top-k retention ---------------------------------------------------------------
+def test_topk_matches_a_stable_sort_and_the_threshold_rule(o64, o32):
+    rng = np.random.default_rng(11)
+    S, stride, Nc = 6, 40, 33
+    for o in (o64, o32):
+        scores = rng.random((S, stride)).astype(o.real)
+        scores[1, 5] = scores[1, 9] = scores[1, 20] = 0.77            # ties: the older chunk ranks first
+        for k in (0, 1, 7, 16, Nc, Nc + 5):
+            idx, cnt = o.compact_topk(scores, Nc, k)
+            for s in range(S):
+                order = np.argsort(-scores[s, :Nc].astype(np.float64), kind="stable")   # descending, ties keep index order
+                want = np.sort(order[:max(0, min(k, Nc))])
+                assert cnt[s] == len(want) and np.array_equal(idx[s, :cnt[s]], want)
+                assert (idx[s, cnt[s]:] == -1).all()
+        # thresholding at a value strictly between the k-th and (k+1)-th score keeps exactly the top k
+        k = 12
+        idx, cnt = o.compact_topk(scores, Nc, k)
+        for s in range(S):
+            srt = np.sort(scores[s, :Nc].astype(np.float64))[::-1]
+            if srt[k - 1] > srt[k]:
+                tau = 0.5 * (srt[k - 1] + srt[k])
+                tidx, tcnt = o.compact(scores[s:s + 1].copy(), Nc, tau)
+                assert tcnt[0] == k and np.array_equal(tidx[0, :k], idx[s, :k])
+
+
+def test_topk_ties_at_the_boundary_prefer_older_chunks(o64):
+    scores = np.array([[0.5, 0.9, 0.5, 0.5, 0.1, 0.5]], np.float64)
+    idx, cnt = o64.compact_topk(scores, 6, 3)
+    assert cnt[0] == 3 and idx[0, :3].tolist() == [0, 1, 2]           # 0.9, then the two oldest 0.5s
+    idx, cnt = o64.compact_topk(scores, 6, 0)
+    assert cnt[0] == 0 and (idx == -1).all()
