@@ -133,6 +133,13 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
  * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw. */
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream);
 
+/* The gating-strategy variant the paper names for its ablations (Sec. 5): keep the k highest-scoring gated
+ * chunks of every sequence instead of thresholding.  Equal scores: the older chunk ranks first, so the
+ * list is unique.  Writes keep_idx / keep_cnt like kvE_compact (ascending ids; k <= 0 keeps nothing,
+ * k >= gated chunks keeps all).  At most 2048 gated chunks, else KVE_ERR_GEOMETRY.  After it,
+ * kvE_reclaim_pages(KVE_RECLAIM_DISCARDED) returns KVE_ERR_STATE (there is no threshold to judge by). */
+int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream);
+
 /* Sec. 3.3 (n' = W + M, memory ratio n / (W + M)) and the KV-memory reduction of Sec. 4.2: hand the pages
  * of gated chunks back to the caller.  Chunks [chunk_begin, chunk_end) of every sequence of `layer` must
  * be covered by the keep list (kvE_compact; its tau decides "discarded").

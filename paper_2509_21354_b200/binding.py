@@ -22,7 +22,7 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
-           "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_decode_attn", "kvE_decode_attn_dense",
+           "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense"]
@@ -80,6 +80,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
     lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
     lib.kvE_compact.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_void_p]
+    lib.kvE_compact_topk.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
     lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
     lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
     lib.kvE_decode_attn_static.argtypes = lib.kvE_decode_attn.argtypes
@@ -243,6 +244,9 @@ class Store:
     def compact(self, layer, tau, stream=None):
         kvE_compact(self, layer, tau, stream)
 
+    def compact_topk(self, layer, k, stream=None):
+        kvE_compact_topk(self, layer, k, stream)
+
     def decode_attn(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn(self, layer, q, out, lse, scale, stream)
 
@@ -298,6 +302,10 @@ def kvE_gate(st: Store, layer, chunk_begin, chunk_end, lstm_weights, stream=None
 
 def kvE_compact(st: Store, layer, tau, stream=None):
     _check("kvE_compact", st.lib.kvE_compact(st.handle, layer, C.c_float(tau), _stream(stream)), st.handle)
+
+
+def kvE_compact_topk(st: Store, layer, k, stream=None):
+    _check("kvE_compact_topk", st.lib.kvE_compact_topk(st.handle, layer, int(k), _stream(stream)), st.handle)
 
 
 def _attn(fn_name, st, layer, q, out, lse, scale, stream):

@@ -17,6 +17,7 @@ struct LayerState {
   int n_gated = 0;       // chunks [0, n_gated) have scores; LSTM state stands after chunk n_gated-1
   int n_compacted = 0;   // keep list covers chunks [0, n_compacted); attention reads raw rows from there on
   float tau = 0.f;       // threshold of the last kvE_compact
+  bool by_topk = false;  // the keep list came from kvE_compact_topk (no threshold to tell "discarded" by)
 };
 
 struct kvE_store {
@@ -304,6 +305,19 @@ int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_compacted = ls.n_gated;
   ls.tau = tau;
+  ls.by_topk = false;
+  return KVE_OK;
+}
+
+int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  if (ls.n_gated > 2048) return KVE_ERR_GEOMETRY;      // the kernel stages one sequence's scores per warp
+  Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_compact_topk(view(st, layer), ls.n_gated, k, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  ls.n_compacted = ls.n_gated;
+  ls.by_topk = true;
   return KVE_OK;
 }
 
@@ -315,6 +329,7 @@ int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, 
   const LayerState& ls = st->layers[layer];
   if (chunk_end > ls.n_compacted) return KVE_ERR_STATE;                        // only chunks the retention rule has judged
   if (mode == KVE_RECLAIM_GATED && st->cfg.attend != KVE_ATTEND_SUMMARY) return KVE_ERR_STATE;   // RAW attention still reads kept pages
+  if (mode == KVE_RECLAIM_DISCARDED && ls.by_topk) return KVE_ERR_STATE;       // "discarded" is defined by the threshold rule
   if (chunk_end == chunk_begin) {
     cudaError_t e = cudaMemsetAsync(free_count, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);

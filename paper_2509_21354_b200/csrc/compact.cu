@@ -32,6 +32,53 @@ cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStre
   return launch_pdl(kve_compact_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), 0, st, v, n_chunks, tau);
 }
 
+// ---- kvE_compact_topk kernel: keep the k highest-scoring chunks of every sequence --------------------------
+// One warp per sequence.  Chunk t is kept iff fewer than k chunks rank before it; u ranks before t when
+// s_u > s_t, or s_u == s_t and u < t (the older chunk first), so the result is unique.  Each lane counts
+// the chunks ranking before its own by walking the sequence's scores in shared memory; the kept ids are
+// then written in ascending order with the same ballot + popcount as the threshold rule.
+constexpr int TOPK_MAX_CHUNKS = 2048;      // scores of one sequence staged per warp
+
+__global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_topk_kernel(LayerView v, int n_chunks, int k) {
+  extern __shared__ float topk_scores[];   // [COMPACT_WARPS][n_chunks]
+  pdl_launch_dependents();
+  pdl_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s = blockIdx.x * COMPACT_WARPS + warp;
+  if (s >= v.S) return;
+  const float* sc = v.scores + (long long)s * v.max_chunks;
+  float* mine = topk_scores + warp * n_chunks;
+  int32_t* idx = v.keep_idx + (long long)s * v.max_chunks;
+  for (int t = lane; t < n_chunks; t += 32) mine[t] = sc[t];
+  __syncwarp();
+  int base = 0;
+  for (int t0 = 0; t0 < n_chunks; t0 += 32) {
+    const int t = t0 + lane;
+    bool keep = false;
+    if (t < n_chunks) {
+      const float st = mine[t];
+      int before = 0;
+      for (int u = 0; u < n_chunks; ++u) {
+        const float su = mine[u];
+        before += (su > st || (su == st && u < t)) ? 1 : 0;
+      }
+      keep = before < k;
+    }
+    const unsigned mask = __ballot_sync(0xffffffffu, keep);
+    if (keep) idx[base + __popc(mask & ((1u << lane) - 1u))] = t;
+    base += __popc(mask);
+  }
+  for (int t = base + lane; t < v.max_chunks; t += 32) idx[t] = -1;
+  if (lane == 0) v.keep_cnt[s] = base;
+}
+
+cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, cudaStream_t st) {
+  if (n_chunks > TOPK_MAX_CHUNKS) return cudaErrorInvalidValue;
+  const size_t smem = sizeof(float) * (size_t)COMPACT_WARPS * (n_chunks > 0 ? n_chunks : 1);
+  return launch_pdl(kve_compact_topk_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), smem, st, v,
+                    n_chunks, k);
+}
+
 // ---- kvE_reclaim_pages kernels (Sec. 3.3, memory ratio n / (W + M)): pages of gated chunks go back to the caller ----
 // A chunk gives its page back if it was discarded (score < tau) or, with mode 1, in any case (retained
 // chunks live on as their summary row).  Free-list order: sequences in order, chunks ascending, so the

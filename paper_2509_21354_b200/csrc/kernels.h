@@ -50,6 +50,7 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
                             int d_g, float* P, bool reset_state, cudaStream_t st);
 cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStream_t st);
+cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, cudaStream_t st);
 cudaError_t launch_reclaim(const LayerView& v, int t0, int t1, float tau, int mode, int32_t* scratch, int32_t* free_list,
                            long long capacity, int32_t* free_count, cudaStream_t st);
 cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_tokens_upper, AttnPlan plan,

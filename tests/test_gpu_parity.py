@@ -502,3 +502,40 @@ def test_reclaim_pages_host_errors_and_overflow():
     _, cnt = st.reclaim_pages(0, 0, 0, "discarded")             # empty range
     torch.cuda.synchronize()
     assert int(cnt.item()) == 0 and st.poll_status() == 0
+
+
+# ---- gating variant: top-k retention ---------------------------------------------------------------
+@pytest.mark.parametrize("attend", ["summary", "raw"])
+def test_compact_topk_matches_oracle_and_feeds_attention(attend):
+    b = _binding()
+    wl = wlm.CFG2.small(B=2, H=8, n=3000, W=256, seed=31)            # 42 gated chunks, ragged tail
+    st, pb, _, _ = full_check(wl, attend)
+    Nc = pb.Nc
+    sc_gpu = st.scores[0].cpu().numpy()                               # the ranking is an integer function of these floats
+    for k in (0, 1, 13, Nc - 1, Nc, Nc + 9):
+        st.compact_topk(0, k)
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        want_idx, want_cnt = pb.o32.compact_topk(sc_gpu.astype(np.float32), Nc, k)
+        assert np.array_equal(st.keep_cnt[0].cpu().numpy(), want_cnt)
+        assert np.array_equal(st.keep_idx[0].cpu().numpy(), want_idx)                # bit-exact
+        # and, where the k-th and (k+1)-th oracle scores are clearly apart, the same list as the oracle's own scores give
+        o_idx, o_cnt = pb.o64.compact_topk(pb.sc64, Nc, k)
+        srt = -np.sort(-pb.sc64[:, :Nc], axis=1)
+        clear = np.ones(st.S, bool) if (k <= 0 or k >= Nc) else (srt[:, k - 1] - srt[:, k] > 1e-3)
+        assert clear.any()
+        assert np.array_equal(st.keep_idx[0].cpu().numpy()[clear], o_idx[clear])
+    # attention over a top-k list: the oracle's attention with that list
+    k = 13
+    st.compact_topk(0, k)
+    q = wlm.gen_q(wl, 0, 3)
+    out = st.decode_attn(0, b.bits_to_bf16(q))
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    idx, cnt = st.keep_idx[0].cpu().numpy(), st.keep_cnt[0].cpu().numpy()
+    want = pb.o64.attn(q, pb.K, pb.V, wl.C, Nc, idx, cnt, pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT[attend], hz.SCALE)[0]
+    hz.check_output(b.bf16_to_bits(out), want, f"attn after top-k/{attend}")
+    # "discarded" has no meaning without a threshold
+    with pytest.raises(b.KveError) as e:
+        st.reclaim_pages(0, 0, Nc, "discarded")
+    assert e.value.rc == -4
