@@ -54,6 +54,17 @@ def shard_batch(B_per_gpu: int, rank: int, world: int):
     return lo, lo + B_per_gpu
 
 
+def paper_cost_model(wl, keep_mean):
+    """The paper's own FLOPs / memory model (Sec. 3.3, Eq. 4-7) at this workload's n, W, C and measured M, for a
+    LLaMA-2-7B-sized layer: context for the measured ratios, not a measurement."""
+    from paper_2509_21354_b200 import cost_model as cm
+    d_sum = wl.d_sum if wl.agg == "mlp" else 0
+    return {"n": wl.n, "W": wl.W, "C": wl.C, "M": keep_mean,
+            "memory_ratio": cm.memory_ratio(wl.n, wl.W, keep_mean),
+            "speedup_incl_ffn": cm.speedup(wl.n, wl.W, keep_mean, wl.C, d_sum, wl.d_g),
+            "attention_flops_ratio": cm.flops_base(wl.n) / cm.flops_kv_efficient(wl.n, wl.W, keep_mean, wl.C, d_sum, wl.d_g)}
+
+
 def max_over_ranks(values, world: int, device="cuda"):
     """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time of a
     multi-GPU step).  The only collective of the benchmark; identity when world == 1."""
@@ -350,6 +361,7 @@ def run_ours(args, rank, world, local_rank):
         "roofline": roofline,
         "roofline_largest_hbm_kernel": roofline_hbm,
         "steady_state": steady,
+        "paper_cost_model": paper_cost_model(wl, keep_mean),
         "kernels": kern,
         "attention_vs_dense": {"note": "attention kernels alone, L2 flushed before every launch",
                                "gated_us": us["attn_gated"], "dense_us": us["attn_dense"],
