@@ -39,6 +39,7 @@ typedef KVO_REAL real;
 #define KVO_AGG_MEAN 0
 #define KVO_AGG_MLP 1
 #define KVO_AGG_IDENTITY 2
+#define KVO_AGG_MAX 3
 #define KVO_ATTEND_SUMMARY 0
 #define KVO_ATTEND_RAW 1
 
@@ -110,6 +111,7 @@ static void mlp2(const real* m, int d, int d_sum, const float* W1, const float* 
  * agg         MEAN: Kbar = (1/C) sum_j k_j
  *             MLP : Kbar = MLP_K(mean), Vbar = MLP_V(mean)  (2 layers, hidden d_sum, erf-GELU)
  *             IDENTITY (C == 1 only): Kbar = k
+ *             MAX : Kbar = element-wise maximum of the chunk's keys ("pooling", Sec. 3.1), Vbar likewise
  * outputs     ksum, vsum [S][stride][d] real at row t; *_b16 the same values rounded to bf16
  * returns 0, or -1 on a bad argument
  */
@@ -123,7 +125,7 @@ int kvo_summarize(const uint16_t* K, const uint16_t* V, int S, int n, int d, int
   if (agg == KVO_AGG_IDENTITY && C != 1) return -1;
   if (agg == KVO_AGG_MLP && (d_sum <= 0 || !W1K || !b1K || !W2K || !b2K || !W1V || !b1V || !W2V || !b2V))
     return -1;
-  if (agg != KVO_AGG_MEAN && agg != KVO_AGG_MLP && agg != KVO_AGG_IDENTITY) return -1;
+  if (agg != KVO_AGG_MEAN && agg != KVO_AGG_MLP && agg != KVO_AGG_IDENTITY && agg != KVO_AGG_MAX) return -1;
 #pragma omp parallel for schedule(static)
   for (int s = 0; s < S; ++s) {
     real* mk = (real*)malloc(sizeof(real) * (size_t)d);
@@ -141,6 +143,17 @@ int kvo_summarize(const uint16_t* K, const uint16_t* V, int S, int n, int d, int
         }
         mk[x] = sk / (real)C;
         mv[x] = sv / (real)C;
+        if (agg == KVO_AGG_MAX) {          /* max-pool: the largest entry of the chunk in each dimension (exact) */
+          size_t row0 = ((size_t)s * n + (size_t)t * C) * d;
+          real bk = bf16_to_real(K[row0 + x]), bv = bf16_to_real(V[row0 + x]);
+          for (int j = 1; j < C; ++j) {
+            real a = bf16_to_real(K[row0 + (size_t)j * d + x]), b = bf16_to_real(V[row0 + (size_t)j * d + x]);
+            if (a > bk) bk = a;
+            if (b > bv) bv = b;
+          }
+          mk[x] = bk;
+          mv[x] = bv;
+        }
       }
       const real *ok = mk, *ov = mv;
       if (agg == KVO_AGG_MLP) {

@@ -11,7 +11,7 @@ import numpy as np
 
 from . import build as _build
 
-AGG_MEAN, AGG_MLP, AGG_IDENTITY = 0, 1, 2
+AGG_MEAN, AGG_MLP, AGG_IDENTITY, AGG_MAX = 0, 1, 2, 3
 ATTEND_SUMMARY, ATTEND_RAW = 0, 1
 
 _u16p = C.POINTER(C.c_uint16)

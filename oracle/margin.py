@@ -13,7 +13,7 @@ from paper_2509_21354_b200 import workloads as wlm
 
 from . import kvo
 
-AGG_CODE = {"mean": kvo.AGG_MEAN, "mlp": kvo.AGG_MLP, "identity": kvo.AGG_IDENTITY}
+AGG_CODE = {"mean": kvo.AGG_MEAN, "mlp": kvo.AGG_MLP, "identity": kvo.AGG_IDENTITY, "max": kvo.AGG_MAX}
 
 
 def centred_b_s(o: kvo.Oracle, wl: wlm.Workload, K, V, mlp, lstm, keep=0.5, n_chunks=None):

@@ -551,3 +551,25 @@ def test_cost_model_reproduces_the_printed_instance():
     # sanity of the closed forms: keeping everything in the window is the base model plus the gate's overhead
     assert cm.flops_kv_efficient(n, n, 0, C, d_sum, d_g) == cm.flops_base(n)
     assert cm.memory_ratio(n, n, 0) == 1.0
+
+
+# ---- "pooling" aggregator (Sec. 3.1): element-wise maximum of the chunk ---------------------------------
+def test_max_pool_aggregator_is_the_elementwise_maximum(o64, o32):
+    wl = wlm.CFG1.small(B=1, H=2, n=512, W=128)
+    K, V = wlm.gen_kv(wl)
+    Nc = wl.n_stale_chunks()
+    Kf, Vf = wlm.bf16_bits_to_f32(K), wlm.bf16_bits_to_f32(V)
+    for o in (o64, o32):
+        sm = o.summarize(K, V, wl.C, 0, Nc, kvo.AGG_MAX)
+        want_k = Kf[:, :Nc * wl.C].reshape(wl.S, Nc, wl.C, 128).max(axis=2)
+        want_v = Vf[:, :Nc * wl.C].reshape(wl.S, Nc, wl.C, 128).max(axis=2)
+        assert np.array_equal(sm["ksum"][:, :Nc].astype(np.float32), want_k)
+        assert np.array_equal(sm["vsum"][:, :Nc].astype(np.float32), want_v)
+        # a maximum of bf16 values is a bf16 value: the rounded copy is the value itself, an entry of the chunk
+        assert np.array_equal(wlm.bf16_bits_to_f32(sm["ksum_b16"][:, :Nc]), want_k)
+        assert (sm["ksum"][:, :Nc] >= o.summarize(K, V, wl.C, 0, Nc, kvo.AGG_MEAN)["ksum"][:, :Nc]).all()   # max >= mean
+    # C = 1: max-pool is the identity
+    wl1 = wlm.CFG1.small(B=1, H=1, n=40, C=1, W=8)
+    K1, V1 = wlm.gen_kv(wl1)
+    a = o64.summarize(K1, V1, 1, 0, 32, kvo.AGG_MAX)
+    assert np.array_equal(a["ksum_b16"][:, :32], K1[:, :32]) and np.array_equal(a["vsum_b16"][:, :32], V1[:, :32])
