@@ -40,7 +40,7 @@ typedef enum {
   KVE_ERR_TIMEOUT = -6    /* a bounded device-side wait ran out (reported through status_word) */
 } kvE_status;
 
-enum { KVE_AGG_MEAN = 0, KVE_AGG_MLP = 1, KVE_AGG_IDENTITY = 2 };   /* Eq. 2 aggregator */
+enum { KVE_AGG_MEAN = 0, KVE_AGG_MLP = 1, KVE_AGG_IDENTITY = 2, KVE_AGG_MAX = 3 };   /* Eq. 2 aggregator; MAX = max-pool (Sec. 3.1) */
 enum { KVE_ATTEND_SUMMARY = 0, KVE_ATTEND_RAW = 1 };                /* what a kept chunk contributes */
 
 /* Geometry, fixed at kvE_create. */
@@ -52,7 +52,7 @@ typedef struct {
   int32_t W;           /* recent window in tokens, >= 0 (Sec. 3.3): never summarised */
   int32_t max_tokens;  /* capacity of one sequence */
   int32_t n_layers;    /* independent layers sharing the handle */
-  int32_t agg;         /* KVE_AGG_* ; IDENTITY needs C == 1 */
+  int32_t agg;         /* KVE_AGG_* ; IDENTITY needs C == 1; MAX: element-wise maximum of the chunk */
   int32_t d_sum;       /* MLP hidden size (KVE_AGG_MLP), multiple of 8, <= 1024 */
   int32_t d_g;         /* LSTM hidden size: 64, 128 or 256 */
   int32_t attend;      /* KVE_ATTEND_* */

@@ -47,7 +47,7 @@ int check_config(const kvE_config* c) {
   if (!c) return KVE_ERR_ARG;
   if (c->B <= 0 || c->Hq <= 0 || c->Hkv <= 0 || c->C <= 0 || c->W < 0 || c->max_tokens <= 0 || c->n_layers <= 0)
     return KVE_ERR_ARG;
-  if (c->agg != KVE_AGG_MEAN && c->agg != KVE_AGG_MLP && c->agg != KVE_AGG_IDENTITY) return KVE_ERR_ARG;
+  if (c->agg != KVE_AGG_MEAN && c->agg != KVE_AGG_MLP && c->agg != KVE_AGG_IDENTITY && c->agg != KVE_AGG_MAX) return KVE_ERR_ARG;
   if (c->attend != KVE_ATTEND_SUMMARY && c->attend != KVE_ATTEND_RAW) return KVE_ERR_ARG;
   if (c->d != 128 || c->Hq != c->Hkv || c->C > 1024) return KVE_ERR_GEOMETRY;
   if (c->agg == KVE_AGG_IDENTITY && c->C != 1) return KVE_ERR_GEOMETRY;
@@ -252,7 +252,7 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
   cudaError_t e;
   {
     Prof prof(st, KVE_K_CHUNK_MEAN, s);
-    e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, s);
+    e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, st->cfg.agg == KVE_AGG_MAX, s);
   }
   if (e == cudaSuccess && mlp) {
     Prof prof(st, KVE_K_CHUNK_MLP, s);

@@ -20,6 +20,15 @@ __device__ __forceinline__ void add_row(float (&acc)[8], const uint4& w) {
   acc[6] += bf16lo(w.w); acc[7] += bf16hi(w.w);
 }
 
+__device__ __forceinline__ void max_row(float (&acc)[8], const uint4& w) {
+  acc[0] = fmaxf(acc[0], bf16lo(w.x)); acc[1] = fmaxf(acc[1], bf16hi(w.x));
+  acc[2] = fmaxf(acc[2], bf16lo(w.y)); acc[3] = fmaxf(acc[3], bf16hi(w.y));
+  acc[4] = fmaxf(acc[4], bf16lo(w.z)); acc[5] = fmaxf(acc[5], bf16hi(w.z));
+  acc[6] = fmaxf(acc[6], bf16lo(w.w)); acc[7] = fmaxf(acc[7], bf16hi(w.w));
+}
+
+// POOL_MAX: element-wise maximum of the chunk instead of its mean (the "pooling" aggregator of Sec. 3.1)
+template <bool POOL_MAX>
 __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerView v, int t0, int n_range,
                                                                         long long n_units, int final_output) {
   pdl_launch_dependents();
@@ -38,19 +47,26 @@ __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerVi
   const uint4* src = reinterpret_cast<const uint4*>((is_v ? v.v_pages : v.k_pages) + page * v.C * D) + l16;
   float acc[8];
 #pragma unroll
-  for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+  for (int x = 0; x < 8; ++x) acc[x] = POOL_MAX ? -INFINITY : 0.f;
   int j = 0;
   for (; j + MEAN_UNROLL <= v.C; j += MEAN_UNROLL) {
     uint4 w[MEAN_UNROLL];
 #pragma unroll
     for (int u = 0; u < MEAN_UNROLL; ++u) w[u] = __ldcs(src + (long long)(j + u) * 16);
 #pragma unroll
-    for (int u = 0; u < MEAN_UNROLL; ++u) add_row(acc, w[u]);
+    for (int u = 0; u < MEAN_UNROLL; ++u) {
+      if (POOL_MAX) max_row(acc, w[u]); else add_row(acc, w[u]);
+    }
   }
-  for (; j < v.C; ++j) add_row(acc, __ldcs(src + (long long)j * 16));
-  const float fc = (float)v.C;
+  for (; j < v.C; ++j) {
+    const uint4 w1 = __ldcs(src + (long long)j * 16);
+    if (POOL_MAX) max_row(acc, w1); else add_row(acc, w1);
+  }
+  if (!POOL_MAX) {
+    const float fc = (float)v.C;
 #pragma unroll
-  for (int x = 0; x < 8; ++x) acc[x] = __fdiv_rn(acc[x], fc);
+    for (int x = 0; x < 8; ++x) acc[x] = __fdiv_rn(acc[x], fc);
+  }
 
   const long long o = ((long long)s * v.max_chunks + t) * D + l16 * 8;
   float4* of = reinterpret_cast<float4*>((is_v ? v.vsum_f32 : v.ksum_f32) + o);
@@ -67,13 +83,16 @@ __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerVi
   }
 }
 
-cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, cudaStream_t st) {
+cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st) {
   const int n_range = t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
   long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
   if (blocks > 148LL * 8) blocks = 148LL * 8;      // 64 resident warps per SM, every CTA resident from the start
-  return launch_pdl(kve_chunk_mean_kernel, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units, final_output ? 1 : 0);
+  if (pool_max)
+    return launch_pdl(kve_chunk_mean_kernel<true>, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units, 1);
+  return launch_pdl(kve_chunk_mean_kernel<false>, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units,
+                    final_output ? 1 : 0);
 }
 
 // ---- aggregator MLP (Eq. 2 read as mean -> d_sum -> d, exact-erf GELU), fp32 FMA ------------------

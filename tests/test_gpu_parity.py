@@ -59,7 +59,7 @@ def check_summaries(st, pb, layer=0):
     vf = st.vsum_f32[layer, :, :Nc].cpu().numpy()
     kb = b.bf16_to_bits(st.ksum_bf16[layer, :, :Nc])
     vb = b.bf16_to_bits(st.vsum_bf16[layer, :, :Nc])
-    if pb.wl.agg in ("mean", "identity"):
+    if pb.wl.agg in ("mean", "identity", "max"):
         # same sequential fp32 sum and IEEE division as the f32 oracle: bit for bit
         assert np.array_equal(kf, pb.sm32["ksum"][:, :Nc]) and np.array_equal(vf, pb.sm32["vsum"][:, :Nc])
         assert np.array_equal(kb, pb.sm32["ksum_b16"][:, :Nc]) and np.array_equal(vb, pb.sm32["vsum_b16"][:, :Nc])
@@ -539,3 +539,10 @@ def test_compact_topk_matches_oracle_and_feeds_attention(attend):
     with pytest.raises(b.KveError) as e:
         st.reclaim_pages(0, 0, Nc, "discarded")
     assert e.value.rc == -4
+
+
+# ---- "pooling" aggregator: element-wise maximum ---------------------------------------------------------
+@pytest.mark.parametrize("C", [32, 64])
+def test_max_pool_aggregator_full_pipeline(C):
+    wl = wlm.CFG1.small(B=2, H=4, n=1500, C=C, W=256, agg="max", seed=17)      # ragged tail; summaries must be bit-exact
+    full_check(wl, "summary")
