@@ -175,3 +175,31 @@ class Oracle:
         if rc != 0:
             raise ValueError(f"kvo_attn_dense rc={rc}")
         return out, out_b16, lse
+
+    # -- Sec. 3.3 attention for a block of queries: T query tokens decoded together (the action
+    #    tokens of Sec. 1 / Sec. 4.2) and Hq query heads on Hkv KV heads (grouped-query attention,
+    #    Sec. 4.1: 32 heads on 8 KV heads).  Every (token, query head) pair is one independent
+    #    query of Eq. 1 against the retained set of KV head hq // (Hq / Hkv); the tokens of a block
+    #    do not see each other.  q [B, T, Hq, d] bf16 bits; results [B, T, Hq, d] / [B, T, Hq]. --
+    def attn_block(self, q, Hkv, K, V, Cs, n_chunks, keep_idx, keep_cnt, ksum_b16, vsum_b16, attend, scale,
+                   dense=False):
+        B, T, Hq, d = q.shape
+        S = K.shape[0]
+        assert S == B * Hkv and Hq % Hkv == 0
+        G = Hq // Hkv
+        out = np.zeros((B, T, Hq, d), self.real)
+        out_b16 = np.zeros((B, T, Hq, d), np.uint16)
+        lse = np.zeros((B, T, Hq), self.real)
+        for t in range(T):
+            for g in range(G):
+                # the g-th query head of every group: query head hkv * G + g reads KV head hkv
+                qs = np.ascontiguousarray(q[:, t, g::G, :].reshape(S, d))
+                if dense:
+                    o, ob, l = self.attn_dense(qs, K, V, scale)
+                else:
+                    o, ob, l, _ = self.attn(qs, K, V, Cs, n_chunks, keep_idx, keep_cnt, ksum_b16, vsum_b16,
+                                            attend, scale)
+                out[:, t, g::G, :] = o.reshape(B, Hkv, d)
+                out_b16[:, t, g::G, :] = ob.reshape(B, Hkv, d)
+                lse[:, t, g::G] = l.reshape(B, Hkv)
+        return out, out_b16, lse

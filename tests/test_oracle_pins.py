@@ -573,3 +573,77 @@ def test_max_pool_aggregator_is_the_elementwise_maximum(o64, o32):
     K1, V1 = wlm.gen_kv(wl1)
     a = o64.summarize(K1, V1, 1, 0, 32, kvo.AGG_MAX)
     assert np.array_equal(a["ksum_b16"][:, :32], K1[:, :32]) and np.array_equal(a["vsum_b16"][:, :32], V1[:, :32])
+
+
+# ---------------------------------------------------------------- query blocks: grouped-query attention (Sec. 4.1) and several query tokens at once
+def test_query_block_brute_force_grouped_heads(o64, o32):
+    """Every (token, query head) of a block against python-float softmax over an explicitly built
+    row list of ITS KV head (query head hq reads KV head hq // group), summary and raw modes."""
+    rng = np.random.default_rng(77)
+    B, Hkv, G, T, d, n, C, W = 2, 2, 3, 2, 4, 23, 4, 6
+    Hq, S = Hkv * G, B * Hkv
+    K, V = rand_bits(rng, S, n, d), rand_bits(rng, S, n, d)
+    q = rand_bits(rng, B, T, Hq, d)
+    Nc = (n - W) // C
+    for o, tol in ((o64, 1e-13), (o32, 3e-6)):
+        sm = o.summarize(K, V, C, 0, Nc, kvo.AGG_MEAN)
+        idx, cnt = o.compact(np.random.default_rng(3).uniform(size=(S, Nc)).astype(o.real), Nc, 0.5)
+        assert 0 < cnt.sum() < S * Nc
+        for mode in (kvo.ATTEND_SUMMARY, kvo.ATTEND_RAW):
+            out, out_b, lse = o.attn_block(q, Hkv, K, V, C, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"], mode, 0.4)
+            for b, t, hq in itertools.product(range(B), range(T), range(Hq)):
+                s = b * Hkv + hq // G
+                kept = idx[s, :cnt[s]]
+                if mode == kvo.ATTEND_SUMMARY:
+                    Kr = [widen(sm["ksum_b16"][s, c]).tolist() for c in kept]
+                    Vr = [widen(sm["vsum_b16"][s, c]).tolist() for c in kept]
+                else:
+                    Kr = [widen(K[s, r]).tolist() for c in kept for r in range(c * C, c * C + C)]
+                    Vr = [widen(V[s, r]).tolist() for c in kept for r in range(c * C, c * C + C)]
+                Kr += [widen(K[s, r]).tolist() for r in range(Nc * C, n)]
+                Vr += [widen(V[s, r]).tolist() for r in range(Nc * C, n)]
+                want, want_lse = brute_attention(widen(q[b, t, hq]).tolist(), Kr, Vr, 0.4)
+                assert np.allclose(out[b, t, hq], want, rtol=0, atol=tol), (mode, b, t, hq)
+                assert abs(lse[b, t, hq] - want_lse) <= 10 * tol
+            assert np.array_equal(out_b, np.vectorize(lambda v: o.bf16_rne(float(v)), otypes=[np.uint16])(out))
+        # full-cache baseline for the block
+        out, _, lse = o.attn_block(q, Hkv, K, V, C, Nc, idx, cnt, None, None, kvo.ATTEND_RAW, 0.4, dense=True)
+        for b, t, hq in itertools.product(range(B), range(T), range(Hq)):
+            s = b * Hkv + hq // G
+            want, _ = brute_attention(widen(q[b, t, hq]).tolist(), widen(K[s]).tolist(), widen(V[s]).tolist(), 0.4)
+            assert np.allclose(out[b, t, hq], want, rtol=0, atol=tol)
+
+
+def test_query_block_of_one_token_one_head_per_kv_head_is_the_single_query_path(o64):
+    q, K, V, Nc = gated_problem(seed=35)
+    sm = o64.summarize(K, V, 4, 0, Nc, kvo.AGG_MEAN)
+    idx, cnt = o64.compact(np.random.default_rng(2).uniform(size=(3, Nc)), Nc, 0.4)
+    want, want_b, want_lse, _ = o64.attn(q, K, V, 4, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"], kvo.ATTEND_SUMMARY, 0.3)
+    got, got_b, got_lse = o64.attn_block(q.reshape(1, 1, 3, 8), 3, K, V, 4, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"],
+                                         kvo.ATTEND_SUMMARY, 0.3)
+    assert np.array_equal(got[0, 0], want) and np.array_equal(got_b[0, 0], want_b) and np.array_equal(got_lse[0, 0], want_lse)
+
+
+def test_query_block_rows_are_independent_and_permutable(o64):
+    """Swapping two tokens of a block swaps their outputs; two equal queries get equal outputs;
+    heads of one group that carry the same query agree (they read the same KV head), heads of
+    different groups do not."""
+    rng = np.random.default_rng(5)
+    B, Hkv, G, T, d, n, C, W = 1, 2, 2, 3, 8, 30, 4, 8
+    S = B * Hkv
+    K, V = rand_bits(rng, S, n, d), rand_bits(rng, S, n, d)
+    q = rand_bits(rng, B, T, Hkv * G, d)
+    q[0, 2] = q[0, 0]                       # token 2 repeats token 0
+    q[0, 1, 1] = q[0, 1, 0]                 # heads 0, 1 (one group) carry one query
+    q[0, 1, 2] = q[0, 1, 0]                 # head 2 (the other group) carries it too
+    Nc = (n - W) // C
+    sm = o64.summarize(K, V, C, 0, Nc, kvo.AGG_MEAN)
+    idx, cnt = o64.compact(np.random.default_rng(9).uniform(size=(S, Nc)), Nc, 0.5)
+    args = (Hkv, K, V, C, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"], kvo.ATTEND_SUMMARY, 0.35)
+    out, _, lse = o64.attn_block(q, *args)
+    assert np.array_equal(out[0, 2], out[0, 0]) and np.array_equal(lse[0, 2], lse[0, 0])
+    assert np.array_equal(out[0, 1, 1], out[0, 1, 0])
+    assert not np.array_equal(out[0, 1, 2], out[0, 1, 0])
+    perm = [1, 0, 2]
+    out_p, _, lse_p = o64.attn_block(np.ascontiguousarray(q[:, perm]), *args)
+    assert np.array_equal(out_p, out[:, perm]) and np.array_equal(lse_p, lse[:, perm])
