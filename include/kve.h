@@ -46,7 +46,8 @@ enum { KVE_ATTEND_SUMMARY = 0, KVE_ATTEND_RAW = 1 };                /* what a ke
 /* Geometry, fixed at kvE_create. */
 typedef struct {
   int32_t B;           /* batch */
-  int32_t Hq, Hkv;     /* query heads, KV heads; Hq == Hkv required */
+  int32_t Hq, Hkv;     /* query heads, KV heads, Hq a multiple of Hkv (query head hq reads KV head hq / (Hq / Hkv));
+                          Hq > Hkv: attention only through kvE_decode_attn_block */
   int32_t d;           /* head dim, 128 */
   int32_t C;           /* chunk size in tokens, 1..1024 (Sec. 3.2) */
   int32_t W;           /* recent window in tokens, >= 0 (Sec. 3.3): never summarised */
@@ -56,6 +57,8 @@ typedef struct {
   int32_t d_sum;       /* MLP hidden size (KVE_AGG_MLP), multiple of 8, <= 1024 */
   int32_t d_g;         /* LSTM hidden size: 64, 128 or 256 */
   int32_t attend;      /* KVE_ATTEND_* */
+  int32_t max_query_tokens; /* most query tokens per kvE_decode_attn_block call; 0: that entry point is not used.
+                               max_query_tokens * (Hq / Hkv) <= 64, and C must be a multiple of 8 */
 } kvE_config;
 
 /* max_chunks = ceil(max_tokens / C) is the chunk stride of every per-chunk array below. */
@@ -165,6 +168,17 @@ int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* l
 int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse,
                           float scale, void* stream);
 
+/* Sec. 3.3 + Eq. 1 for a block of queries: n_query_tokens tokens decoded together (the action tokens of one
+ * control step) on all Hq query heads, Hq / Hkv of which share each KV head (grouped-query attention, the
+ * 32-head / 8-KV-head model of Sec. 4.1).  Every (token, head) pair is an independent query against the
+ * retained set [kept chunks ; raw tail] of its KV head (dense != 0: against all n stored tokens); the
+ * tokens of a block do not see each other.  Each retained K/V row is read once per KV head, and the
+ * products run on the tensor cores.
+ *   q, out: DEVICE bf16 [B][n_query_tokens][Hq][d]; lse: DEVICE fp32 [B][n_query_tokens][Hq] or NULL.
+ *   KVE_ERR_STATE if cfg.max_query_tokens == 0, KVE_ERR_CAPACITY if n_query_tokens exceeds it. */
+int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, void* out,
+                          float* lse, float scale, void* stream);
+
 /* kvE_decode_attn without any scratch from the caller.  (The paper has no counterpart: this is a
  * deployment aid.)  Some users of this library must not allocate device memory once they are
  * running: a robot-control loop that handed the whole GPU to its framework's memory pool at
@@ -221,7 +235,7 @@ int kvE_layer_state(const kvE_store* st, int layer, int* n_tokens, int* n_summar
  * kvE_profile_read synchronises the device and writes, per kernel id, the duration in microseconds
  * of that kernel's most recent launch, or -1 if it has not run since profiling was enabled. */
 enum { KVE_K_APPEND = 0, KVE_K_CHUNK_MEAN, KVE_K_CHUNK_MLP, KVE_K_GATE_PROJ, KVE_K_GATE_RNN, KVE_K_COMPACT,
-       KVE_K_ATTN, KVE_K_ATTN_DENSE, KVE_K_COUNT };
+       KVE_K_ATTN, KVE_K_ATTN_DENSE, KVE_K_ATTN_BLOCK, KVE_K_COUNT };
 int kvE_profile(kvE_store* st, int enable);
 int kvE_profile_read(kvE_store* st, float* us /* [KVE_K_COUNT] */);
 

@@ -22,10 +22,10 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
-           "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense",
+           "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense", "kvE_decode_attn_block",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
-KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense"]
+KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense", "attn_block"]
 
 
 class KveError(RuntimeError):
@@ -36,7 +36,7 @@ class KveError(RuntimeError):
 
 class kvE_config(C.Structure):
     _fields_ = [(k, C.c_int32) for k in ("B", "Hq", "Hkv", "d", "C", "W", "max_tokens", "n_layers", "agg",
-                                         "d_sum", "d_g", "attend")]
+                                         "d_sum", "d_g", "attend", "max_query_tokens")]
 
 
 class kvE_buffers(C.Structure):
@@ -84,6 +84,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
     lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
     lib.kvE_decode_attn_static.argtypes = lib.kvE_decode_attn.argtypes
+    lib.kvE_decode_attn_block.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                          C.c_float, C.c_void_p]
     lib.kvE_reclaim_pages.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
     lib.kvE_decode_step_host.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float,
@@ -167,13 +169,17 @@ class Store:
     """
 
     def __init__(self, B, H, C_, W, max_tokens, d_g, agg="mean", d_sum=0, attend="summary", n_layers=1,
-                 page_perm=None, device="cuda", seed=0):
+                 page_perm=None, device="cuda", seed=0, Hq=None, max_query_tokens=0):
+        """H = KV heads (S = B * H sequences); Hq = query heads (default H); max_query_tokens > 0 enables
+        decode_attn_block."""
         if not torch.cuda.is_available():
             raise RuntimeError("libkve needs a CUDA device; there is no CPU path")
         self.lib = load_library()
         self.device = torch.device(device)
-        self.cfg = kvE_config(B=B, Hq=H, Hkv=H, d=128, C=C_, W=W, max_tokens=max_tokens, n_layers=n_layers,
-                              agg=AGG[agg], d_sum=d_sum, d_g=d_g, attend=ATTEND[attend])
+        self.Hq = H if Hq is None else Hq
+        self.cfg = kvE_config(B=B, Hq=self.Hq, Hkv=H, d=128, C=C_, W=W, max_tokens=max_tokens, n_layers=n_layers,
+                              agg=AGG[agg], d_sum=d_sum, d_g=d_g, attend=ATTEND[attend],
+                              max_query_tokens=max_query_tokens)
         self.B, self.H, self.S, self.C, self.W, self.d_g = B, H, B * H, C_, W, d_g
         self.n_layers, self.max_tokens = n_layers, max_tokens
         self.max_chunks = -(-max_tokens // C_)
@@ -253,6 +259,9 @@ class Store:
     def decode_attn_dense(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)
 
+    def decode_attn_block(self, layer, q, dense=False, out=None, lse=None, scale=None, stream=None):
+        return kvE_decode_attn_block(self, layer, q, dense, out, lse, scale, stream)
+
     def reclaim_pages(self, layer, chunk_begin, chunk_end, mode="discarded", free_list=None, free_count=None, stream=None):
         return kvE_reclaim_pages(self, layer, chunk_begin, chunk_end, mode, free_list, free_count, stream)
 
@@ -324,6 +333,21 @@ def kvE_decode_attn(st: Store, layer, q, out=None, lse=None, scale=None, stream=
 
 def kvE_decode_attn_dense(st: Store, layer, q, out=None, lse=None, scale=None, stream=None):
     return _attn("kvE_decode_attn_dense", st, layer, q, out, lse, scale, stream)
+
+
+def kvE_decode_attn_block(st: Store, layer, q, dense=False, out=None, lse=None, scale=None, stream=None):
+    """q: bf16 [B, T, Hq, 128] device tensor (T query tokens on all query heads).  Returns out (same shape);
+    lse, if given, is an fp32 [B, T, Hq] device tensor."""
+    assert q.dtype == torch.bfloat16 and q.dim() == 4 and q.shape[0] == st.B and q.shape[2] == st.Hq and q.shape[3] == 128
+    if out is None:
+        out = torch.empty_like(q)
+    assert out.shape == q.shape and out.dtype == torch.bfloat16
+    if lse is not None:
+        assert lse.dtype == torch.float32 and tuple(lse.shape) == tuple(q.shape[:3])
+    scale = (1.0 / 128.0 ** 0.5) if scale is None else scale
+    _check("kvE_decode_attn_block", st.lib.kvE_decode_attn_block(st.handle, layer, _p(q), int(q.shape[1]), int(bool(dense)),
+                                                                 _p(out), _p(lse), C.c_float(scale), _stream(stream)), st.handle)
+    return out
 
 
 RECLAIM = {"discarded": 0, "gated": 1}

@@ -25,8 +25,13 @@ struct kvE_store {
   kvE_buffers buf;
   int S, max_chunks;
   // workspace carve-up (byte offsets)
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, ws_needed;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_block, ws_needed;
   int max_splits;
+  // block-of-queries attention: tensor maps over the page pools and the summary store (encoded at
+  // create when cfg.max_query_tokens > 0), rows per page box, split cap the workspace was sized for
+  alignas(64) unsigned char block_maps[4 * ATTN_BLOCK_MAP_BYTES];
+  bool block_ready = false;
+  int block_hp = 0, block_split_cap = 1;
   std::vector<LayerState> layers;
   std::string cuda_error;
   // optional per-kernel timing: one (start, stop) event pair per kernel id
@@ -49,7 +54,11 @@ int check_config(const kvE_config* c) {
     return KVE_ERR_ARG;
   if (c->agg != KVE_AGG_MEAN && c->agg != KVE_AGG_MLP && c->agg != KVE_AGG_IDENTITY && c->agg != KVE_AGG_MAX) return KVE_ERR_ARG;
   if (c->attend != KVE_ATTEND_SUMMARY && c->attend != KVE_ATTEND_RAW) return KVE_ERR_ARG;
-  if (c->d != 128 || c->Hq != c->Hkv || c->C > 1024) return KVE_ERR_GEOMETRY;
+  if (c->d != 128 || c->Hq % c->Hkv != 0 || c->C > 1024) return KVE_ERR_GEOMETRY;
+  if (c->max_query_tokens < 0) return KVE_ERR_ARG;
+  if (c->max_query_tokens > 0 &&
+      ((long long)c->max_query_tokens * (c->Hq / c->Hkv) > ATTN_BLOCK_MAX_ROWS || attn_block_hp(c->C) < 8))
+    return KVE_ERR_GEOMETRY;
   if (c->agg == KVE_AGG_IDENTITY && c->C != 1) return KVE_ERR_GEOMETRY;
   if (c->agg == KVE_AGG_MLP && (c->d_sum <= 0 || c->d_sum % 8 != 0 || c->d_sum > 1024)) return KVE_ERR_GEOMETRY;
   if (c->d_g != 64 && c->d_g != 128 && c->d_g != 256) return KVE_ERR_GEOMETRY;
@@ -58,8 +67,13 @@ int check_config(const kvE_config* c) {
 }
 
 struct Carve {
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, total;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_block, total;
 };
+// most splits per sequence the block-of-queries attention uses: one CTA per SM, one wave
+int block_split_cap(long long S) {
+  long long c = 148 / S;
+  return (int)(c < 1 ? 1 : (c > MAX_SPLITS ? MAX_SPLITS : c));
+}
 Carve carve(const kvE_config& c) {
   const size_t S = (size_t)c.B * c.Hkv;
   const size_t max_chunks = ((size_t)c.max_tokens + c.C - 1) / c.C;
@@ -70,6 +84,11 @@ Carve carve(const kvE_config& c) {
   k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
   k.off_stage = o;    o = align_up(o + 4 * S * 128 * 2);   // k_new, v_new, q, out of kvE_decode_step_host
   k.off_reclaim = o;  o = align_up(o + (2 * S + 1) * sizeof(int32_t));   // per-sequence counts and offsets of kvE_reclaim_pages
+  k.off_block = o;    // split records of kvE_decode_attn_block: [S][splits][query rows, padded to 16][132] fp32
+  if (c.max_query_tokens > 0) {
+    const size_t rows = ((size_t)c.max_query_tokens * (c.Hq / c.Hkv) + 15) / 16 * 16;
+    o = align_up(o + S * block_split_cap((long long)S) * rows * ATTN_PARTIAL_FLOATS * sizeof(float));
+  }
   k.total = o;
   return k;
 }
@@ -187,7 +206,19 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   st->S = cfg->B * cfg->Hkv;
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
   st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
-  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->ws_needed = k.total;
+  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_block = k.off_block; st->ws_needed = k.total;
+  if (cfg->max_query_tokens > 0) {
+    st->block_hp = attn_block_hp(cfg->C);
+    st->block_split_cap = block_split_cap(st->S);
+    const cudaError_t em = encode_attn_block_maps(st->block_maps, buf->k_pages, buf->v_pages, (long long)buf->n_pages * cfg->C,
+                                                  st->block_hp, buf->ksum_bf16, buf->vsum_bf16,
+                                                  (long long)cfg->n_layers * st->S * st->max_chunks);
+    if (em != cudaSuccess) {
+      delete st;
+      return KVE_ERR_CUDA;
+    }
+    st->block_ready = true;
+  }
   st->max_splits = MAX_SPLITS;
   st->layers.assign(cfg->n_layers, LayerState());
   cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.total - k.off_partials);
@@ -342,19 +373,53 @@ int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, 
 
 int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {
   if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;      // grouped query heads go through kvE_decode_attn_block
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   return run_attention(st, layer, mode, q, out, lse, scale, static_cast<cudaStream_t>(stream));
 }
 
 int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {
   if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   return run_attention(st, layer, ATTN_DENSE, q, out, lse, scale, static_cast<cudaStream_t>(stream));
+}
+
+int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, void* out, float* lse,
+                          float scale, void* stream) {
+  if (bad_layer(st, layer) || !q || !out || n_query_tokens <= 0) return KVE_ERR_ARG;
+  if (!st->block_ready) return KVE_ERR_STATE;                  // cfg.max_query_tokens was 0
+  if (n_query_tokens > st->cfg.max_query_tokens) return KVE_ERR_CAPACITY;
+  const AttnMode mode = dense ? ATTN_DENSE : (st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY);
+  const LayerState& ls = st->layers[layer];
+  // padded rows per sequence: the raw tail rounded up to whole tiles, then the kept rows
+  long long tail, lead;
+  if (mode == ATTN_DENSE) { tail = ls.n_tokens; lead = 0; }
+  else {
+    tail = ls.n_tokens - (long long)ls.n_compacted * st->cfg.C;
+    lead = (long long)ls.n_compacted * (mode == ATTN_RAW ? st->cfg.C : 1);
+  }
+  const long long tiles = (tail + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS + (lead + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS;
+  long long splits = st->block_split_cap;
+  if (splits > tiles) splits = tiles;
+  if (splits < 1) splits = 1;
+  const long long tiles_per_split = tiles > 0 ? (tiles + splits - 1) / splits : 1;
+  AttnPlan plan;
+  plan.rows_per_split = (int)(tiles_per_split * ATTN_TILE_ROWS);
+  plan.max_splits = (int)(tiles > 0 ? (tiles + tiles_per_split - 1) / tiles_per_split : 1);
+  char* ws = static_cast<char*>(st->buf.workspace);
+  Prof prof(st, KVE_K_ATTN_BLOCK, static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_attn_block(view(st, layer), st->block_maps, mode, ls.n_compacted, plan, n_query_tokens,
+                                    st->cfg.Hq / st->cfg.Hkv, st->block_hp, (long long)layer * st->S * st->max_chunks, q, out,
+                                    lse, scale, reinterpret_cast<float*>(ws + st->off_block),
+                                    reinterpret_cast<int32_t*>(ws + st->off_counters), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
 }
 
 static int decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host, const void* q_host,
                             void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
                             int from_scratch, void* stream, bool wait) {
   if (bad_layer(st, layer) || !k_new_host || !v_new_host || !q_host || !out_host || !lw) return KVE_ERR_ARG;
+  if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t row_bytes = (size_t)st->S * 128 * 2;
   char* stage = static_cast<char*>(st->buf.workspace) + st->off_stage;
@@ -492,6 +557,7 @@ cudaError_t static_scratch(unsigned char** out) {
 extern "C" int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale,
                                       void* stream) {
   if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   const LayerState& ls = st->layers[layer];
   const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;

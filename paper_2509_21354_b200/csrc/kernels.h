@@ -58,4 +58,14 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_t
                         cudaStream_t st);
 int attn_smem_bytes();
 
+// block-of-queries attention (grouped query heads x query tokens), tensor-map fed
+constexpr int ATTN_BLOCK_MAX_ROWS = 64;        // query rows (tokens x heads per KV head) per KV sequence
+constexpr int ATTN_BLOCK_MAP_BYTES = 128;      // one tensor map; a handle keeps four (K pages, V pages, K summaries, V summaries)
+int attn_block_hp(int C);                      // rows per page box: largest power of two <= 64 dividing C
+cudaError_t encode_attn_block_maps(void* maps, const void* k_pages, const void* v_pages, long long page_rows, int hp,
+                                   const void* ksum, const void* vsum, long long sum_rows);
+cudaError_t launch_attn_block(const LayerView& v, const void* maps, AttnMode mode, int n_chunks, AttnPlan plan, int T, int G,
+                              int hp, long long sum_row0, const void* q, void* out, float* lse, float scale, float* partials,
+                              int32_t* counters, cudaStream_t st);
+
 }  // namespace kve

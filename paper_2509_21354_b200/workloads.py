@@ -150,6 +150,11 @@ def gen_q(wl: Workload, layer: int = 0, step: int = 0) -> np.ndarray:
     return f32_to_bf16_bits(_rng(wl.seed, _TAG_Q, layer, step).standard_normal((wl.S, wl.d), dtype=np.float32))
 
 
+def gen_q_block(wl: Workload, T: int, Hq: int, layer: int = 0, step: int = 0) -> np.ndarray:
+    """queries of T tokens on Hq query heads, [B, T, Hq, d] bf16 bits (wl.H counts the KV heads)"""
+    return f32_to_bf16_bits(_rng(wl.seed, _TAG_Q, layer, 7919 + step).standard_normal((wl.B, T, Hq, wl.d), dtype=np.float32))
+
+
 def gen_new_tokens(wl: Workload, layer: int = 0, step: int = 0, n_new: int = 1):
     """k_new, v_new [S, n_new, d] bf16 bits for an autoregressive append."""
     rng = _rng(wl.seed, _TAG_NEW, layer, step)

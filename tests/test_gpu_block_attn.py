@@ -1,0 +1,118 @@
+"""GPU parity of kvE_decode_attn_block (query blocks: several query tokens on grouped query heads)
+against the oracle, which treats every (token, query head) pair as one independent query of Eq. 1."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_21354_b200 import workloads as wlm
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+
+
+def _prepared(wl, attend, G, T, n_layers=1, layer=0):
+    from paper_2509_21354_b200 import binding as b
+    pb = hz.Problem(wl, layer=layer)
+    st = b.Store(B=wl.B, H=wl.H, Hq=wl.H * G, C_=wl.C, W=wl.W, max_tokens=wl.max_tokens, d_g=wl.d_g, agg=wl.agg,
+                 d_sum=wl.d_sum, attend=attend, page_perm="random", seed=3, n_layers=n_layers, max_query_tokens=T)
+    st.append(layer, b.bits_to_bf16(pb.K), b.bits_to_bf16(pb.V))
+    if pb.Nc > 0:
+        st.summarize_chunks(layer, 0, pb.Nc, b.AggWeights(pb.mlp) if pb.mlp is not None else None)
+        st.gate(layer, 0, pb.Nc, b.LstmWeights(pb.lstm))
+        st.compact(layer, pb.tau)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    return b, pb, st
+
+
+def _check(b, pb, st, attend, G, T, layer=0, dense=False, step=0):
+    wl = pb.wl
+    q = wlm.gen_q_block(wl, T, wl.H * G, layer, step)
+    lse = torch.full((wl.B, T, wl.H * G), float("nan"), dtype=torch.float32, device="cuda")
+    out = st.decode_attn_block(layer, b.bits_to_bf16(q), dense=dense, lse=lse)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    want, _, want_lse = pb.o64.attn_block(q, wl.H, pb.K, pb.V, wl.C, pb.Nc, pb.idx64, pb.cnt64, pb.sm64["ksum_b16"],
+                                          pb.sm64["vsum_b16"], hz.ATT[attend], hz.SCALE, dense=dense)
+    hz.check_output(b.bf16_to_bits(out), want, f"block/{attend}/G{G}T{T}")
+    assert np.abs(lse.cpu().numpy() - want_lse).max() <= 1e-3
+    return out
+
+
+# (G query heads per KV head, T query tokens): 1..64 query rows per KV head, every row-block count
+@pytest.mark.parametrize("G,T", [(1, 1), (4, 3), (4, 7), (2, 20), (8, 8), (1, 33)])
+@pytest.mark.parametrize("attend", ["summary", "raw"])
+def test_block_attention_matches_oracle(attend, G, T):
+    # two KV sequences: many splits per sequence; ragged tail (n not a multiple of 8)
+    wl = wlm.CFG1.small(B=1, H=2, n=2443, W=300, seed=21)
+    b, pb, st = _prepared(wl, attend, G, T)
+    _check(b, pb, st, attend, G, T)
+    _check(b, pb, st, attend, G, T, dense=True, step=1)
+
+
+@pytest.mark.parametrize("C,n", [(32, 1500), (24, 1000), (128, 3001), (8, 700)])
+def test_block_attention_chunk_sizes_and_page_boxes(C, n):
+    # C = 32: boxes of 32 rows; 24 and 8: boxes of 8; 128: half pages
+    wl = wlm.CFG1.small(B=2, H=3, n=n, C=C, W=3 * C + 5, seed=22)
+    for attend in ("summary", "raw"):
+        b, pb, st = _prepared(wl, attend, 4, 7)
+        _check(b, pb, st, attend, 4, 7)
+        _check(b, pb, st, attend, 4, 7, dense=True)
+
+
+def test_block_attention_many_sequences_single_split_and_second_layer():
+    # 160 KV sequences (more than one per SM: no splits), layer 1 of 2 (summary rows of another layer)
+    wl = wlm.CFG1.small(B=20, H=8, n=900, W=128, seed=23)
+    b, pb, st = _prepared(wl, "summary", 4, 7, n_layers=2, layer=1)
+    _check(b, pb, st, "summary", 4, 7, layer=1)
+
+
+def test_block_attention_short_and_empty_caches():
+    from paper_2509_21354_b200 import binding as b
+    wl = wlm.CFG1.small(B=2, H=2, n=50, W=256, seed=24)      # nothing has left the window: raw tail only
+    bb, pb, st = _prepared(wl, "summary", 4, 7)
+    assert pb.Nc == 0
+    _check(bb, pb, st, "summary", 4, 7)
+    st.set_len(0, 0)                                          # empty cache: zeros out, lse = -inf
+    q = b.bits_to_bf16(wlm.gen_q_block(wl, 7, 8))
+    lse = torch.zeros((2, 7, 8), dtype=torch.float32, device="cuda")
+    out = st.decode_attn_block(0, q, lse=lse)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    assert torch.all(out == 0) and torch.all(torch.isinf(lse) & (lse < 0))
+
+
+def test_block_of_one_row_agrees_with_the_single_query_kernel():
+    wl = wlm.CFG1.small(B=2, H=4, n=3000, seed=25)
+    b, pb, st = _prepared(wl, "summary", 1, 1)
+    q = wlm.gen_q(wl, 0, 5)
+    one = st.decode_attn(0, b.bits_to_bf16(q))
+    blk = st.decode_attn_block(0, b.bits_to_bf16(q.reshape(wl.B, 1, wl.H, 128)))
+    torch.cuda.synchronize()
+    one_b, blk_b = b.bf16_to_bits(one).reshape(-1), b.bf16_to_bits(blk).reshape(-1)
+    # two fp32 evaluation orders, each rounded once to bf16: equal up to a rounding flip (near zero, where
+    # cancellation leaves fp32 noise of several tiny bf16 steps, up to that noise)
+    x, y = wlm.bf16_bits_to_f32(one_b).astype(np.float64), wlm.bf16_bits_to_f32(blk_b).astype(np.float64)
+    assert np.all(np.abs(x - y) <= 2.0 ** -7 * np.abs(x) + 1e-5)
+    assert (hz.bf16_ulp_distance(one_b, blk_b) > 1).mean() < 1e-2
+
+
+def test_block_attention_argument_checks():
+    from paper_2509_21354_b200 import binding as b
+    wl = wlm.CFG1.small(B=1, H=2, n=600, seed=26)
+    with pytest.raises(b.KveError):                            # 9 tokens x 8 heads per KV head > 64 query rows
+        b.Store(B=1, H=2, Hq=16, C_=64, W=256, max_tokens=1024, d_g=128, max_query_tokens=9)
+    with pytest.raises(b.KveError):                            # chunk size without a box of at least 8 rows
+        b.Store(B=1, H=2, Hq=8, C_=20, W=256, max_tokens=1024, d_g=128, max_query_tokens=4)
+    st = b.Store(B=1, H=2, Hq=8, C_=64, W=256, max_tokens=1024, d_g=128, max_query_tokens=4)
+    q = torch.zeros((1, 5, 8, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(b.KveError) as err:
+        st.decode_attn_block(0, q)
+    assert err.value.rc == -3
+    with pytest.raises(b.KveError) as err:                     # grouped heads: the single-query entry points refuse
+        st.decode_attn(0, torch.zeros((2, 128), dtype=torch.bfloat16, device="cuda"))
+    assert err.value.rc == -2
+    st0 = b.Store(B=1, H=2, C_=64, W=256, max_tokens=1024, d_g=128)
+    with pytest.raises(b.KveError) as err:                     # not enabled at create
+        st0.decode_attn_block(0, torch.zeros((1, 1, 2, 128), dtype=torch.bfloat16, device="cuda"))
+    assert err.value.rc == -4

@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_header():
-    assert C.sizeof(binding.kvE_config) == 12 * 4
+    assert C.sizeof(binding.kvE_config) == 13 * 4
     assert C.sizeof(binding.kvE_buffers) == 17 * 8
     assert C.sizeof(binding.kvE_agg_weights) == 8 * 8
     assert C.sizeof(binding.kvE_lstm_weights) == 5 * 8 + 8
@@ -47,6 +47,18 @@ def test_workspace_bytes_and_geometry_checks_need_no_device():
         c2 = binding.kvE_config.from_buffer_copy(cfg)
         setattr(c2, field, bad)
         assert lib.kvE_workspace_bytes(C.byref(c2)) == 0
+    # grouped query heads: Hq a multiple of Hkv; a query block holds at most 64 rows per KV head and
+    # enlarges the workspace by its split records
+    gq = binding.kvE_config.from_buffer_copy(cfg)
+    gq.Hkv, gq.max_query_tokens = 8, 7
+    assert lib.kvE_workspace_bytes(C.byref(gq)) > 0
+    gq.max_query_tokens = 17                                               # 17 tokens x 4 heads per KV head = 68 rows
+    assert lib.kvE_workspace_bytes(C.byref(gq)) == 0
+    gq.max_query_tokens, gq.C = 7, 12                                      # no box of 8 rows divides a 12-token chunk
+    assert lib.kvE_workspace_bytes(C.byref(gq)) == 0
+    with_block = binding.kvE_config.from_buffer_copy(cfg)
+    with_block.max_query_tokens = 4
+    assert lib.kvE_workspace_bytes(C.byref(with_block)) > ws
     out = C.c_void_p()
     assert lib.kvE_create(C.byref(cfg), None, C.byref(out)) == -1          # null buffers
     assert lib.kvE_append(None, 0, None, None, 1, None, None) == -1        # null handle
