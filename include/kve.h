@@ -58,7 +58,7 @@ typedef struct {
   int32_t d_g;         /* LSTM hidden size: 64, 128 or 256 */
   int32_t attend;      /* KVE_ATTEND_* */
   int32_t max_query_tokens; /* most query tokens per kvE_decode_attn_block call; 0: that entry point is not used.
-                               max_query_tokens * (Hq / Hkv) <= 64, and C must be a multiple of 8 */
+                               max_query_tokens * (Hq / Hkv) <= 128, and C must be a multiple of 8 */
 } kvE_config;
 
 /* max_chunks = ceil(max_tokens / C) is the chunk stride of every per-chunk array below. */

@@ -59,7 +59,7 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_t
 int attn_smem_bytes();
 
 // block-of-queries attention (grouped query heads x query tokens), tensor-map fed
-constexpr int ATTN_BLOCK_MAX_ROWS = 64;        // query rows (tokens x heads per KV head) per KV sequence
+constexpr int ATTN_BLOCK_MAX_ROWS = 128;       // query rows (tokens x heads per KV head) per KV sequence
 constexpr int ATTN_BLOCK_MAP_BYTES = 128;      // one tensor map; a handle keeps four (K pages, V pages, K summaries, V summaries)
 int attn_block_hp(int C);                      // rows per page box: largest power of two <= 64 dividing C
 cudaError_t encode_attn_block_maps(void* maps, const void* k_pages, const void* v_pages, long long page_rows, int hp,

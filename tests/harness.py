@@ -74,3 +74,22 @@ def check_output(out_bits, want_real, name=""):
     bad = err > tight
     assert not bad.any(), f"{name}: {bad.sum()} entries beyond one bf16 step, worst {err[bad].max()}"
     return float(err.max()), float(err.mean())
+
+
+def check_output_bf16_weights(out_bits, want_real, spread, name=""):
+    """The same for a kernel that rounds the softmax numerators p_i to bf16 before the product with V
+    (tensor-core operand): p_i (1 + e_i), |e_i| <= 2^-9, shifts an output by at most
+    2^-9 * sum_i p_i |v_i| / sum_i p_i = 2^-9 * spread, where `spread` is the same attention
+    evaluated on |V| (the oracle computes it).  On top: fp32 accumulation and the one bf16 rounding
+    of the result, as in check_output."""
+    got = wlm.bf16_bits_to_f32(out_bits).astype(np.float64)
+    want = np.asarray(want_real, np.float64)
+    err = np.abs(got - want)
+    assert err.max() <= 2e-2, f"{name}: max-abs {err.max()}"
+    assert err.mean() <= 2e-3, f"{name}: mean-abs {err.mean()}"
+    bound = 2.0 ** -8 * np.abs(want) + 2.0 ** -9 * np.asarray(spread, np.float64) + 2e-5
+    bad = err > bound
+    assert not bad.any(), f"{name}: {bad.sum()} entries beyond the rounding bound, worst {(err / bound).max()} x"
+    # the bound is a worst case; rounding errors of independent rows mostly cancel
+    assert err.mean() <= 0.25 * bound.mean(), f"{name}: mean error {err.mean()} vs mean bound {bound.mean()}"
+    return float(err.max()), float(err.mean())

@@ -47,12 +47,12 @@ def test_workspace_bytes_and_geometry_checks_need_no_device():
         c2 = binding.kvE_config.from_buffer_copy(cfg)
         setattr(c2, field, bad)
         assert lib.kvE_workspace_bytes(C.byref(c2)) == 0
-    # grouped query heads: Hq a multiple of Hkv; a query block holds at most 64 rows per KV head and
+    # grouped query heads: Hq a multiple of Hkv; a query block holds at most 128 rows per KV head and
     # enlarges the workspace by its split records
     gq = binding.kvE_config.from_buffer_copy(cfg)
     gq.Hkv, gq.max_query_tokens = 8, 7
     assert lib.kvE_workspace_bytes(C.byref(gq)) > 0
-    gq.max_query_tokens = 17                                               # 17 tokens x 4 heads per KV head = 68 rows
+    gq.max_query_tokens = 33                                               # 33 tokens x 4 heads per KV head = 132 rows
     assert lib.kvE_workspace_bytes(C.byref(gq)) == 0
     gq.max_query_tokens, gq.C = 7, 12                                      # no box of 8 rows divides a 12-token chunk
     assert lib.kvE_workspace_bytes(C.byref(gq)) == 0
