@@ -175,6 +175,56 @@ def algorithmic_flops(wl, Nc):
     return fl
 
 
+def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
+    """kvE_decode_attn_block on the workload's geometry with grouped query heads (the 32 query heads on
+    8 KV heads of Sec. 4.1) and 7 query tokens decoded together: gated and full-cache attention, each
+    launch timed alone with L2 flushed.  Mean aggregator (the summaries only feed the keep list here)."""
+    import torch
+    from paper_2509_21354_b200 import binding as b
+    Hkv, G, T = 8, wl.H // 8, 7
+    g = wl.small(H=Hkv, agg="mean", d_sum=0)
+    st = b.Store(B=g.B, H=Hkv, Hq=Hkv * G, C_=g.C, W=g.W, max_tokens=g.n + g.C, d_g=g.d_g, agg="mean", attend="summary",
+                 page_perm="random", seed=seed, max_query_tokens=T)
+    gen = fill_cache(st, g, seed)
+    lstm = wlm.gen_lstm_weights(g)
+    lw = b.LstmWeights(lstm)
+    n = g.n - 1
+    Nc = g.n_stale_chunks(n)
+    st.summarize_chunks(0, 0, Nc, None)
+    st.gate(0, 0, Nc, lw)
+    torch.cuda.synchronize()
+    sc = st.scores[0, :, :Nc].double().clamp(1e-9, 1 - 1e-9)
+    lw.set_b_s(float(-torch.median(torch.log(sc / (1 - sc))).item()) + lstm["b_s"])      # keep about half
+    st.gate(0, 0, Nc, lw)
+    st.compact(0, g.tau)
+    torch.cuda.synchronize()
+    keep = st.keep_cnt[0].float().mean().item()
+    q = torch.randn((g.B, T, Hkv * G, 128), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    st.profile(True)
+    res = {"what": f"kvE_decode_attn_block: {T} query tokens x {Hkv * G} query heads on {Hkv} KV heads, B={g.B}, n={n}; "
+                   "tcgen05 kernel, one launch timed alone, L2 flushed",
+           "query_rows_per_kv_head": T * G, "kept_chunks_mean": keep}
+    for name, dense, rows in (("gated", False, n - Nc * g.C + keep), ("dense", True, n)):
+        ts = []
+        for i in range(12):
+            flush.fill_(1)
+            st.decode_attn_block(0, q, dense=dense, out=out)
+            torch.cuda.synchronize()
+            if i >= 2:
+                ts.append(st.profile_read()["attn_block"])
+        us = float(np.mean(ts))
+        by = g.S * rows * 512                                  # every retained K and V row once per KV head
+        fl = 4 * 128 * T * G * g.S * rows                      # Q K^T and P V
+        res[name] = {"us": us, "kv_bytes": int(by), "GB/s": by / us / 1e3, "frac_of_hbm_peak": by / us / 1e3 / hbm,
+                     "TFLOP/s": fl / us / 1e6, "frac_of_bf16_peak": fl / us / 1e6 / tensor_peak,
+                     "peak_kind": f"of {peak_kind}"}
+    assert st.poll_status() == 0
+    res["gated_vs_dense"] = res["dense"]["us"] / res["gated"]["us"]
+    return res
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -361,6 +411,7 @@ def run_ours(args, rank, world, local_rank):
         "roofline": roofline,
         "roofline_largest_hbm_kernel": roofline_hbm,
         "steady_state": steady,
+        "query_block_attention": query_block_leg(wl, hbm, tensor_peak, peak_kind, seed + 17),
         "paper_cost_model": paper_cost_model(wl, keep_mean),
         "kernels": kern,
         "attention_vs_dense": {"note": "attention kernels alone, L2 flushed before every launch",

@@ -15,12 +15,17 @@
 //      warps 2-5, 6-9  two softmax groups, even and odd tiles, each with its own running (m_ref, l)
 //               and its own accumulator O in tensor memory (merged at the end), so two tiles are in
 //               softmax at any time.  Thread = query row = tensor-memory lane.  Reads its 64 logits of the tile,
-//               p = exp2(s * scale * log2 e - m_ref), writes P as two bf16 planes (hi + lo, so P V
-//               loses nothing against an fp32 product) into the swizzled A-operand layout.  m_ref
-//               follows the running maximum lazily: only when a row's maximum has grown by more
-//               than 8 (log2 units) does the warp rescale its rows of O in tensor memory, so p
-//               stays below 2^8 and the usual per-tile rescale of O disappears.
-//  * Q (zero-padded to 128 rows) sits in shared memory as the K-major A operand for the whole CTA.
+//               p = exp2(s * scale * log2 e - m_ref) by the special-function unit, writes P as bf16 into
+//               the swizzled A-operand layout (rounding p moves an output by at most
+//               2^-9 sum p |v| / sum p; TC_PLANES = 2 adds a second plane p - bf16(p) and removes that
+//               error at the price of a ring stage).  m_ref follows the running maximum lazily: only
+//               when a row's maximum has grown by more than 8 (log2 units) does the warp rescale its
+//               rows of O in tensor memory, so p stays below 2^8 and the usual per-tile rescale of O
+//               disappears.
+//  * with R <= 32 (<= 64) query rows the block is laid out four times (twice) down the 128 rows of the
+//    A operand, and each copy's warp takes a quarter (half) of a tile's 64 columns: the softmax of
+//    a tile then runs on all four warps of a group, one per scheduler, instead of on one.
+//  * Q sits in shared memory as the K-major A operand for the whole CTA.
 //  * tile rows beyond the valid ones (ragged tail, partial tiles of kept rows) hold stale bytes:
 //    their logits are masked and their V rows are zeroed before P V (0 * NaN would poison O).
 //  * splits leave (m_ref, l, O) records in the workspace; the last CTA of a sequence to finish (atomic
