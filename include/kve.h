@@ -174,6 +174,8 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
  * retained set [kept chunks ; raw tail] of its KV head (dense != 0: against all n stored tokens); the
  * tokens of a block do not see each other.  Each retained K/V row is read once per KV head, and the
  * products run on the tensor cores.
+ *   The softmax numerators enter the tensor core as bf16: against exact weights an output moves by at
+ *   most 2^-9 * sum_i p_i |v_i| / sum_i p_i (accumulation in fp32, one bf16 rounding of the result).
  *   q, out: DEVICE bf16 [B][n_query_tokens][Hq][d]; lse: DEVICE fp32 [B][n_query_tokens][Hq] or NULL.
  *   KVE_ERR_STATE if cfg.max_query_tokens == 0, KVE_ERR_CAPACITY if n_query_tokens exceeds it. */
 int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, void* out,
