@@ -130,7 +130,7 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------- GPU arm
-def fill_cache(st, wl, seed):
+def fill_cache(st, wl, seed, layer=0):
     """Synthetic cache of the workload's shape, generated on the device: N(0,1) keys and values, keys
     shifted by a per-(sequence, chunk) offset ~ N(0, key_offset_std^2); stored through kvE_append."""
     import torch
@@ -145,7 +145,7 @@ def fill_cache(st, wl, seed):
             nch = -(-m // wl.C)
             off = torch.randn((wl.S, nch, 128), generator=g, device="cuda", dtype=torch.float32) * wl.key_offset_std
             k += off.repeat_interleave(wl.C, dim=1)[:, :m]
-        st.append(0, k.to(torch.bfloat16).contiguous(), v.to(torch.bfloat16).contiguous())
+        st.append(layer, k.to(torch.bfloat16).contiguous(), v.to(torch.bfloat16).contiguous())
     return g
 
 
@@ -222,6 +222,80 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
                      "peak_kind": f"of {peak_kind}"}
     assert st.poll_status() == 0
     res["gated_vs_dense"] = res["dense"]["us"] / res["gated"]["us"]
+    return res
+
+
+def graph_tick_leg(wl, n_layers, seed, replays=20):
+    """One decode tick of a whole model between two gate triggers: for each of n_layers layers append the
+    new token and run the gated attention, all layers captured once in a CUDA graph and replayed.
+    (Every replay appends at the same position: the host-side length is fixed at capture, so the
+    replays do identical work.)  Compared with the same calls issued one by one."""
+    import torch
+    from paper_2509_21354_b200 import binding as b
+    g = wl.small(agg="mean", d_sum=0)                      # the aggregator only feeds the keep list here
+    per_layer = g.S * (g.n + g.C) * 512 * 1.1
+    n_layers = max(1, min(n_layers, int(40e9 // per_layer)))
+    st = b.Store(B=g.B, H=g.H, C_=g.C, W=g.W, max_tokens=g.n + g.C, d_g=g.d_g, agg="mean", attend="summary",
+                 n_layers=n_layers, page_perm="random", seed=seed)
+    lstm = wlm.gen_lstm_weights(g)
+    lw = b.LstmWeights(lstm)
+    Nc = g.n_stale_chunks(g.n - 1)                         # the cache holds n - 1 tokens; the tick appends the n-th
+    gen = None
+    for L in range(n_layers):
+        gen = fill_cache(st, g, seed + L, layer=L)
+        st.summarize_chunks(L, 0, Nc, None)
+        st.gate(L, 0, Nc, lw)
+        if L == 0:
+            torch.cuda.synchronize()
+            sc = st.scores[0, :, :Nc].double().clamp(1e-9, 1 - 1e-9)
+            lw.set_b_s(float(-torch.median(torch.log(sc / (1 - sc))).item()) + lstm["b_s"])
+            st.gate(L, 0, Nc, lw)
+        st.compact(L, g.tau)
+    torch.cuda.synchronize()
+    S = g.S
+    rnd = lambda: torch.randn((n_layers, S, 128), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    k_new, v_new, q = rnd(), rnd(), rnd()
+    out = torch.empty_like(q)
+
+    def tick():
+        for L in range(n_layers):
+            st.set_len(L, g.n - 1)
+            st.append(L, k_new[L].view(S, 1, 128), v_new[L].view(S, 1, 128))
+            st.decode_attn(L, q[L], out[L])
+
+    tick()
+    torch.cuda.synchronize()
+    eager_out = out.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        tick()
+        with torch.cuda.graph(graph, stream=side):
+            tick()
+    torch.cuda.current_stream().wait_stream(side)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    same = bool(torch.equal(out, eager_out))
+    res = {"what": f"decode tick over {n_layers} layers (per layer: set length, append one token, gated attention), "
+                   "captured once in a CUDA graph and replayed, vs the same calls issued one by one",
+           "n_layers": n_layers, "graph_equals_eager": same}
+    for name, fn in (("eager", tick), ("graph", graph.replay)):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(replays):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / replays
+        res[name] = {"ms_per_tick": ms, "us_per_layer": ms * 1e3 / n_layers, "ticks_per_s": 1e3 / ms}
+    assert st.poll_status() == 0
+    res["kv_bytes_per_tick"] = int(n_layers * S * (g.n - Nc * g.C + st.keep_cnt.float().mean().item()) * 512)
+    res["GB/s_graph"] = res["kv_bytes_per_tick"] / (res["graph"]["ms_per_tick"] * 1e-3) / 1e9
     return res
 
 
@@ -412,6 +486,7 @@ def run_ours(args, rank, world, local_rank):
         "roofline_largest_hbm_kernel": roofline_hbm,
         "steady_state": steady,
         "query_block_attention": query_block_leg(wl, hbm, tensor_peak, peak_kind, seed + 17),
+        "decode_tick_graph": graph_tick_leg(wl, args.tick_layers, seed + 31) if args.tick_layers > 0 else None,
         "paper_cost_model": paper_cost_model(wl, keep_mean),
         "kernels": kern,
         "attention_vs_dense": {"note": "attention kernels alone, L2 flushed before every launch",
@@ -499,6 +574,8 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(wlm.CONFIGS))
     ap.add_argument("--attend", default="summary", choices=["summary", "raw"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tick-layers", type=int, default=32,
+                    help="layers of the CUDA-graph decode-tick leg (0 = skip; reduced if the caches would not fit 40 GB)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
