@@ -546,3 +546,49 @@ def test_compact_topk_matches_oracle_and_feeds_attention(attend):
 def test_max_pool_aggregator_full_pipeline(C):
     wl = wlm.CFG1.small(B=2, H=4, n=1500, C=C, W=256, agg="max", seed=17)      # ragged tail; summaries must be bit-exact
     full_check(wl, "summary")
+
+
+def test_decode_tick_replays_from_a_cuda_graph():
+    """append + gated attention of two layers captured once and replayed: the calls neither synchronise nor
+    allocate, so the replay must reproduce the eager outputs bit for bit (and the oracle's within tolerance)."""
+    b = _binding()
+    wl = wlm.CFG1.small(B=2, H=4, n=1500, seed=41)
+    st = make_store(wl, n_layers=2)
+    pbs = [hz.Problem(wl, layer=L) for L in range(2)]
+    for L, pb in enumerate(pbs):
+        load_kv(st, L, pb.K[:, :-1], pb.V[:, :-1])
+        Nc = wl.n_stale_chunks(wl.n - 1)
+        st.summarize_chunks(L, 0, Nc, None)
+        st.gate(L, 0, Nc, b.LstmWeights(pb.lstm))
+        st.compact(L, pb.tau)
+    qs = [b.bits_to_bf16(wlm.gen_q(wl, L, 9)) for L in range(2)]
+    kn = [b.bits_to_bf16(pb.K[:, -1:]) for pb in pbs]
+    vn = [b.bits_to_bf16(pb.V[:, -1:]) for pb in pbs]
+    out = torch.zeros((2, st.S, 128), dtype=torch.bfloat16, device="cuda")
+
+    def tick():
+        for L in range(2):
+            st.set_len(L, wl.n - 1)
+            st.append(L, kn[L], vn[L])
+            st.decode_attn(L, qs[L], out[L])
+
+    tick()
+    torch.cuda.synchronize()
+    eager = out.clone()
+    side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            tick()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+    assert st.poll_status() == 0
+    for L, pb in enumerate(pbs):
+        Nc = wl.n_stale_chunks(wl.n - 1)
+        want, _, _, _ = pb.o64.attn(wlm.gen_q(wl, L, 9), pb.K, pb.V, wl.C, Nc, pb.idx64, pb.cnt64, pb.sm64["ksum_b16"],
+                                    pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)
+        hz.check_output(b.bf16_to_bits(out[L]), want, f"graph replay, layer {L}")
