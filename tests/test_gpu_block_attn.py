@@ -162,3 +162,13 @@ def test_block_attention_growing_maxima_force_rescales():
         assert np.ptp(want_lse) > 20                          # the rows really are far apart / peaked
         hz.check_output_bf16_weights(b.bf16_to_bits(out), want, spread, f"block/{attend}/growing maxima")
         assert np.abs(lse.cpu().numpy() - want_lse).max() <= 1e-3 * np.abs(want_lse).max()
+
+
+def test_block_attention_at_the_benchmarked_size():
+    """The geometry bench.py times for query blocks: cfg2 with 8 KV heads (64 KV sequences, n = 4096,
+    C = 64, W = 512), 4 query heads per KV head, 7 query tokens; every output against the oracle."""
+    wl = wlm.CFG2.small(H=8)
+    b, pb, st = _prepared(wl, "summary", 4, 7)
+    assert 0.4 < pb.cnt64.mean() / pb.Nc < 0.6
+    _check(b, pb, st, "summary", 4, 7)
+    _check(b, pb, st, "summary", 4, 7, dense=True, step=1)
