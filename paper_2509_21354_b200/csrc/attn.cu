@@ -217,8 +217,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
         dot += __shfl_xor_sync(0xffffffffu, dot, 1);                             // row (lane >> 2), full sum
         const float logit = ((lane >> 2) < nvalid) ? dot * sl2 : -INFINITY;
         const float m_new = fmaxf(m, warp_max(logit));
-        const float p = exp2f(logit - m_new);
-        const float alpha = exp2f(m - m_new);
+        const float p = ex2_fast(logit - m_new);
+        const float alpha = ex2_fast(m - m_new);
         l = fmaf(l, alpha, 0.25f * warp_sum(p));    // every row sits on four lanes
         m = m_new;
 #pragma unroll

@@ -57,13 +57,6 @@ constexpr int TC_THREADS = 320;
 constexpr int TC_TMEM_COLS = 512;                  // O of the two groups: 2 x 128 columns, then S: two buffers of 64
 constexpr float TC_RESCALE_STEP = 8.f;             // log2 units a row maximum may run ahead of m_ref
 
-// 2^x by the special-function unit alone (2 ulp; results below 2^-126 flush to zero, -inf gives 0)
-__device__ __forceinline__ float ex2_fast(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
 // bounded wait with one outcome for the whole warp
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
   return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity));
