@@ -226,10 +226,10 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
 
 
 def graph_tick_leg(wl, n_layers, seed, replays=20):
-    """One decode tick of a whole model between two gate triggers: for each of n_layers layers append the
-    new token and run the gated attention, all layers captured once in a CUDA graph and replayed.
-    (Every replay appends at the same position: the host-side length is fixed at capture, so the
-    replays do identical work.)  Compared with the same calls issued one by one."""
+    """The decode loop of a whole model between two gate triggers: per token, for each of n_layers layers
+    append the new token at the device-held length (kvE_append_next) and run the gated attention; all
+    layers captured once in a CUDA graph, every replay advancing by one token.  Compared with the
+    same calls issued one by one."""
     import torch
     from paper_2509_21354_b200 import binding as b
     g = wl.small(agg="mean", d_sum=0)                      # the aggregator only feeds the keep list here
@@ -257,20 +257,26 @@ def graph_tick_leg(wl, n_layers, seed, replays=20):
     k_new, v_new, q = rnd(), rnd(), rnd()
     out = torch.empty_like(q)
 
-    def tick():
+    budget = 3 + replays                                   # tokens one timed phase appends per layer
+    assert 2 * budget + 2 < g.C, "the loop must stay between two gate triggers"
+
+    def rewind():
         for L in range(n_layers):
             st.set_len(L, g.n - 1)
-            st.append(L, k_new[L].view(S, 1, 128), v_new[L].view(S, 1, 128))
+
+    def tick():                                            # every call / replay appends the NEXT token of every layer
+        for L in range(n_layers):
+            st.append_next(L, k_new[L], v_new[L], n_reserve=2 * budget)
             st.decode_attn(L, q[L], out[L])
 
     tick()
     torch.cuda.synchronize()
     eager_out = out.clone()
+    rewind()
     side = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
-        tick()
         with torch.cuda.graph(graph, stream=side):
             tick()
     torch.cuda.current_stream().wait_stream(side)
@@ -278,10 +284,12 @@ def graph_tick_leg(wl, n_layers, seed, replays=20):
     graph.replay()
     torch.cuda.synchronize()
     same = bool(torch.equal(out, eager_out))
-    res = {"what": f"decode tick over {n_layers} layers (per layer: set length, append one token, gated attention), "
-                   "captured once in a CUDA graph and replayed, vs the same calls issued one by one",
-           "n_layers": n_layers, "graph_equals_eager": same}
+    res = {"what": f"decode loop over {n_layers} layers between two gate triggers (per layer and token: kvE_append_next at the "
+                   "device-held length, gated attention), captured once in a CUDA graph and replayed - every replay "
+                   "appends the next token - vs the same calls issued one by one",
+           "n_layers": n_layers, "graph_first_tick_equals_eager": same}
     for name, fn in (("eager", tick), ("graph", graph.replay)):
+        rewind()
         for _ in range(3):
             fn()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -293,6 +301,7 @@ def graph_tick_leg(wl, n_layers, seed, replays=20):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / replays
         res[name] = {"ms_per_tick": ms, "us_per_layer": ms * 1e3 / n_layers, "ticks_per_s": 1e3 / ms}
+        assert int(st.seq_len[0, 0]) == g.n - 1 + budget   # the loop really advanced
     assert st.poll_status() == 0
     res["kv_bytes_per_tick"] = int(n_layers * S * (g.n - Nc * g.C + st.keep_cnt.float().mean().item()) * 512)
     res["GB/s_graph"] = res["kv_bytes_per_tick"] / (res["graph"]["ms_per_tick"] * 1e-3) / 1e9

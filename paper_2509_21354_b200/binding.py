@@ -21,7 +21,7 @@ ATTEND = {"summary": 0, "raw": 1}
 STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_CAPACITY",
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
-EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_set_len",
+EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_append_next", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense", "kvE_decode_attn_block",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
@@ -77,6 +77,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_destroy.argtypes = [C.c_void_p]
     lib.kvE_append.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p]
     lib.kvE_set_len.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+    lib.kvE_append_next.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
     lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
     lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
     lib.kvE_compact.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_void_p]
@@ -258,6 +259,12 @@ class Store:
 
     def decode_attn_dense(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)
+
+    def append_next(self, layer, k_new, v_new, n_reserve=0, stream=None):
+        """k_new, v_new: bf16 [S, 128] (or [S, 1, 128]); appended at the device-held length (graph-replayable)."""
+        assert k_new.dtype == torch.bfloat16 and k_new.shape == v_new.shape and k_new.numel() == self.S * 128
+        _check("kvE_append_next", self.lib.kvE_append_next(self.handle, layer, _p(k_new), _p(v_new), int(n_reserve),
+                                                           _stream(stream)), self.handle)
 
     def decode_attn_block(self, layer, q, dense=False, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_block(self, layer, q, dense, out, lse, scale, stream)

@@ -12,7 +12,8 @@
 using namespace kve;
 
 struct LayerState {
-  int n_tokens = 0;      // tokens stored (every sequence of the layer)
+  int n_tokens = 0;      // tokens stored (every sequence of the layer), as far as the host knows
+  int reserve_upper = 0; // kvE_append_next: replays may take the device-side length up to here; attention is sized for it
   int n_summarised = 0;  // chunks [0, n_summarised) have summaries
   int n_gated = 0;       // chunks [0, n_gated) have scores; LSTM state stands after chunk n_gated-1
   int n_compacted = 0;   // keep list covers chunks [0, n_compacted); attention reads raw rows from there on
@@ -163,11 +164,12 @@ AttnPlan plan_attention(const kvE_store* st, long long n_rows_upper) {
 int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* out, float* lse, float scale,
                   cudaStream_t stream) {
   const LayerState& ls = st->layers[layer];
+  const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
   long long rows_upper;
-  if (mode == ATTN_DENSE) rows_upper = ls.n_tokens;
+  if (mode == ATTN_DENSE) rows_upper = n_upper;
   else {
     const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;
-    rows_upper = (long long)ls.n_compacted * per + (ls.n_tokens - (long long)ls.n_compacted * st->cfg.C);
+    rows_upper = (long long)ls.n_compacted * per + (n_upper - (long long)ls.n_compacted * st->cfg.C);
   }
   AttnPlan plan = plan_attention(st, rows_upper);
   char* ws = static_cast<char*>(st->buf.workspace);
@@ -250,8 +252,23 @@ int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, i
     cudaError_t e = launch_append(view(st, layer), k_new, v_new, n_new, ls.n_tokens, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(st, e);
     ls.n_tokens += n_new;
+    ls.reserve_upper = 0;
   }
   if (n_ready) *n_ready = stale_chunks(st->cfg, ls.n_tokens) - ls.n_gated;
+  return KVE_OK;
+}
+
+int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_reserve, void* stream) {
+  if (bad_layer(st, layer) || !k_new || !v_new || n_reserve < 0) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  if (ls.n_tokens + 1 > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
+  Prof prof(st, KVE_K_APPEND, static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_append_next(view(st, layer), k_new, v_new, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  long long upper = (long long)ls.n_tokens + 1 + n_reserve;
+  if (upper > st->cfg.max_tokens) upper = st->cfg.max_tokens;
+  if (upper > ls.reserve_upper) ls.reserve_upper = (int)upper;
+  ls.n_tokens += 1;
   return KVE_OK;
 }
 
@@ -262,6 +279,7 @@ int kvE_set_len(kvE_store* st, int layer, int n, void* stream) {
   if (e != cudaSuccess) return cuda_fail(st, e);
   LayerState& ls = st->layers[layer];
   ls.n_tokens = n;
+  ls.reserve_upper = 0;
   const int nc = stale_chunks(st->cfg, n);
   if (ls.n_summarised > nc) ls.n_summarised = nc;
   if (ls.n_gated > nc) ls.n_gated = 0;          // the carried LSTM state is past the cut: gate again from chunk 0
@@ -393,9 +411,10 @@ int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_t
   const LayerState& ls = st->layers[layer];
   // padded rows per sequence: the raw tail rounded up to whole tiles, then the kept rows
   long long tail, lead;
-  if (mode == ATTN_DENSE) { tail = ls.n_tokens; lead = 0; }
+  const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
+  if (mode == ATTN_DENSE) { tail = n_upper; lead = 0; }
   else {
-    tail = ls.n_tokens - (long long)ls.n_compacted * st->cfg.C;
+    tail = n_upper - (long long)ls.n_compacted * st->cfg.C;
     lead = (long long)ls.n_compacted * (mode == ATTN_RAW ? st->cfg.C : 1);
   }
   const long long tiles = (tail + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS + (lead + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS;
@@ -561,7 +580,8 @@ extern "C" int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, v
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   const LayerState& ls = st->layers[layer];
   const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;
-  const long long rows_upper = (long long)ls.n_compacted * per + (ls.n_tokens - (long long)ls.n_compacted * st->cfg.C);
+  const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
+  const long long rows_upper = (long long)ls.n_compacted * per + (n_upper - (long long)ls.n_compacted * st->cfg.C);
   const AttnPlan plan = plan_attention(st, rows_upper);
   const long long records = (long long)st->S * plan.max_splits;
   if (st->S > STATIC_MAX_SEQ || records > STATIC_MAX_REC) {

@@ -107,6 +107,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   const int n_tail = max(0, n - raw0);
   const int n_rows = n_tail + n_lead;
   const int n_splits = max(1, (n_rows + a.rows_per_split - 1) / a.rows_per_split);
+  // the sequence has outgrown what this launch was sized for (a replayed launch): rows would be dropped
+  if (n_splits > (int)gridDim.x && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
   if (split >= n_splits) return;
   const int r_begin = split * a.rows_per_split;
   const int r_end = min(n_rows, r_begin + a.rows_per_split);

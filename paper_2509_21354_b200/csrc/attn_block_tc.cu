@@ -94,6 +94,8 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
   pdl_wait();      // lengths, keep lists, summaries and the queries come from earlier kernels
 
   const BlockGeom gm = block_geometry(a, s, split);
+  // the sequence has outgrown what this launch was sized for (a replayed launch): rows would be dropped
+  if (gm.n_splits > (int)gridDim.x && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
   if (split >= gm.n_splits) return;
   const int n_tiles = gm.n_tiles;
 

@@ -592,3 +592,67 @@ def test_decode_tick_replays_from_a_cuda_graph():
         want, _, _, _ = pb.o64.attn(wlm.gen_q(wl, L, 9), pb.K, pb.V, wl.C, Nc, pb.idx64, pb.cnt64, pb.sm64["ksum_b16"],
                                     pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)
         hz.check_output(b.bf16_to_bits(out[L]), want, f"graph replay, layer {L}")
+
+
+def test_decode_loop_advances_under_a_cuda_graph():
+    """kvE_append_next + gated attention captured ONCE; every replay appends the next token at the
+    device-held length and attends over the grown cache.  Each step against the oracle on the cache
+    as it then stands; afterwards the host is told the length and gates the chunk that completed."""
+    b = _binding()
+    wl = wlm.CFG1.small(B=2, H=4, n=1530, C=64, W=256, seed=43, n_append=16)   # the loop crosses a chunk boundary
+    st = make_store(wl)
+    pb = hz.Problem(wl)
+    load_kv(st, 0, pb.K, pb.V)
+    aw, lw = None, b.LstmWeights(pb.lstm)
+    run_gpu_pipeline(st, pb, 0, aw, lw)
+    steps = 12
+    k_in = torch.zeros((st.S, 128), dtype=torch.bfloat16, device="cuda")
+    v_in, q_in = torch.zeros_like(k_in), torch.zeros_like(k_in)
+    out = torch.zeros_like(k_in)
+    side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            st.append_next(0, k_in, v_in, n_reserve=steps)
+            st.decode_attn(0, q_in, out)
+    torch.cuda.current_stream().wait_stream(side)
+    K, V = pb.K, pb.V
+    for step in range(steps):
+        kn, vn = wlm.gen_new_tokens(wl, 0, step)
+        q = wlm.gen_q(wl, 0, 50 + step)
+        k_in.copy_(b.bits_to_bf16(kn[:, 0])); v_in.copy_(b.bits_to_bf16(vn[:, 0])); q_in.copy_(b.bits_to_bf16(q))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        K, V = np.concatenate([K, kn], axis=1), np.concatenate([V, vn], axis=1)
+        assert int(st.seq_len[0, 0]) == wl.n + step + 1
+        want, _, _, n_eff = pb.oracle_attn(q, "summary", "f64", K, V, pb.Nc)
+        hz.check_output(b.bf16_to_bits(out), want, f"graph loop, step {step}")
+    Kd, Vd = pages_to_plain(st, 0, wl.n + steps)
+    assert np.array_equal(Kd, K) and np.array_equal(Vd, V)          # every token landed at its own position
+    # back on the host: the true length, then the chunk that has left the window meanwhile
+    st.set_len(0, wl.n + steps)
+    nc = (wl.n + steps - wl.W) // wl.C
+    assert nc == pb.Nc + 1
+    st.summarize_chunks(0, pb.Nc, nc, aw)
+    st.gate(0, pb.Nc, nc, lw)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    # a replay beyond the reserved growth is reported, not silently truncated
+    wl2 = wlm.CFG1.small(B=1, H=2, n=300, C=64, W=64, seed=44, n_append=400)
+    st2 = make_store(wl2)
+    pb2 = hz.Problem(wl2)
+    load_kv(st2, 0, pb2.K, pb2.V)
+    run_gpu_pipeline(st2, pb2, 0, None, b.LstmWeights(pb2.lstm))
+    z = torch.zeros((st2.S, 128), dtype=torch.bfloat16, device="cuda")
+    g2 = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g2, stream=side):
+            st2.append_next(0, z, z, n_reserve=0)
+            st2.decode_attn(0, z, torch.empty_like(z))
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(200):                                           # far past the tile the launch was sized for
+        g2.replay()
+    torch.cuda.synchronize()
+    assert st2.poll_status() == -3
