@@ -116,18 +116,19 @@ int kvE_destroy(kvE_store* st);
 int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new,
                int* n_ready, void* stream);
 
-/* kvE_append for one token per sequence at the length the DEVICE holds (seq_len), which the call advances by
- * one: nothing about the position is fixed at launch, so the call can be captured in a CUDA graph and every
- * replay appends the next token (k_new, v_new: DEVICE bf16 [S][d], read at replay time).  This is the decode
+/* kvE_append of n_new tokens per sequence at the length the DEVICE holds (seq_len), which the call advances by
+ * n_new: nothing about the position is fixed at launch, so the call can be captured in a CUDA graph and every
+ * replay appends the next n_new tokens (k_new, v_new: DEVICE bf16 [S][n_new][d], read at replay time).  This is the decode
  * loop between two gate triggers of Sec. 3.3 without a host round trip per token.
- *   n_reserve: how many further such appends (replays included) may follow before the next kvE_set_len or
+ *   n_reserve: how many further tokens such appends (replays included) may add before the next kvE_set_len or
  *   kvE_append; attention launches issued after this call are sized for that much growth, so they stay valid
- *   when replayed along.  The handle's own length advances by ONE per call, not per replay: after replaying,
+ *   when replayed along.  The handle's own length advances by n_new per call, not per replay: after replaying,
  *   give it the true length with kvE_set_len(layer, n) before summarising or gating the chunks that have
  *   completed meanwhile (attention keeps reading them as raw rows until then, which is exact).
- *   Device side: a sequence already at max_tokens is left alone, and an attention launch replayed past the
+ *   Device side: a sequence without room for n_new more tokens is left alone, and an attention launch replayed past the
  *   growth it was sized for drops nothing silently: both set KVE_ERR_CAPACITY in the status word. */
-int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_reserve, void* stream);
+int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new, int n_reserve,
+                    void* stream);
 
 /* Set the stored length of `layer` (all sequences) to n tokens, n <= max_tokens; the pages keep
  * their contents.  Chunks at or beyond the new stale range lose their summarised / gated /

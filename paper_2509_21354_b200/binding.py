@@ -77,7 +77,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_destroy.argtypes = [C.c_void_p]
     lib.kvE_append.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p]
     lib.kvE_set_len.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
-    lib.kvE_append_next.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+    lib.kvE_append_next.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
     lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
     lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
     lib.kvE_compact.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_void_p]
@@ -261,9 +261,12 @@ class Store:
         return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)
 
     def append_next(self, layer, k_new, v_new, n_reserve=0, stream=None):
-        """k_new, v_new: bf16 [S, 128] (or [S, 1, 128]); appended at the device-held length (graph-replayable)."""
-        assert k_new.dtype == torch.bfloat16 and k_new.shape == v_new.shape and k_new.numel() == self.S * 128
-        _check("kvE_append_next", self.lib.kvE_append_next(self.handle, layer, _p(k_new), _p(v_new), int(n_reserve),
+        """k_new, v_new: bf16 [S, n_new, 128] (or [S, 128] for one token); appended at the device-held length
+        (graph-replayable); n_reserve: further tokens replays may add."""
+        assert k_new.dtype == torch.bfloat16 and k_new.shape == v_new.shape and k_new.shape[0] == self.S
+        n_new = k_new.numel() // (self.S * 128)
+        assert n_new * self.S * 128 == k_new.numel()
+        _check("kvE_append_next", self.lib.kvE_append_next(self.handle, layer, _p(k_new), _p(v_new), n_new, int(n_reserve),
                                                            _stream(stream)), self.handle)
 
     def decode_attn_block(self, layer, q, dense=False, out=None, lse=None, scale=None, stream=None):

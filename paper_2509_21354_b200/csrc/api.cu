@@ -258,17 +258,17 @@ int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, i
   return KVE_OK;
 }
 
-int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_reserve, void* stream) {
-  if (bad_layer(st, layer) || !k_new || !v_new || n_reserve < 0) return KVE_ERR_ARG;
+int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new, int n_reserve, void* stream) {
+  if (bad_layer(st, layer) || !k_new || !v_new || n_new <= 0 || n_reserve < 0) return KVE_ERR_ARG;
   LayerState& ls = st->layers[layer];
-  if (ls.n_tokens + 1 > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
+  if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   Prof prof(st, KVE_K_APPEND, static_cast<cudaStream_t>(stream));
-  cudaError_t e = launch_append_next(view(st, layer), k_new, v_new, static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_append_next(view(st, layer), k_new, v_new, n_new, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
-  long long upper = (long long)ls.n_tokens + 1 + n_reserve;
+  long long upper = (long long)ls.n_tokens + n_new + n_reserve;
   if (upper > st->cfg.max_tokens) upper = st->cfg.max_tokens;
   if (upper > ls.reserve_upper) ls.reserve_upper = (int)upper;
-  ls.n_tokens += 1;
+  ls.n_tokens += n_new;
   return KVE_OK;
 }
 

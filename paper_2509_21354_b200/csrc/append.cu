@@ -34,39 +34,41 @@ __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint
     for (int b = threadIdx.x; b < v.B; b += blockDim.x) v.seq_len[b] = pos0 + n_new;
 }
 
-// One token per sequence at the position the DEVICE holds in seq_len (replayable from a CUDA graph: nothing
+// n_new tokens per sequence from the position the DEVICE holds in seq_len (replayable from a CUDA graph: nothing
 // about the position is baked into the launch).  The length itself is advanced by the kernel below,
 // which runs after this one in stream order, so every thread here reads the old length.
 __global__ void __launch_bounds__(256) kve_append_next_kernel(LayerView v, const uint4* __restrict__ k_new,
-                                                              const uint4* __restrict__ v_new) {
+                                                              const uint4* __restrict__ v_new, int n_new) {
   pdl_launch_dependents();
   pdl_wait();
-  const long long total = (long long)v.S * 32;
+  const long long total = (long long)v.S * n_new * 32;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int lane16 = (int)(idx & 15);
     const int is_v = (int)((idx >> 4) & 1);
-    const int s = (int)(idx >> 5);
-    const int pos = v.seq_len[s / v.H];
-    if (pos < 0 || pos >= v.max_tokens) continue;      // flagged by the length kernel
+    const long long row = idx >> 5;              // s * n_new + i
+    const int s = (int)(row / n_new);
+    const int n0 = v.seq_len[s / v.H];
+    if (n0 < 0 || n0 + n_new > v.max_tokens) continue;  // no room: flagged by the length kernel, nothing written
+    const int pos = n0 + (int)(row - (long long)s * n_new);
     const int chunk = pos / v.C;
     const int r = pos - chunk * v.C;
     const long long page = v.page_table[(long long)s * v.max_chunks + chunk];
     if (page < 0 || page >= v.n_pages) { set_status(v.status, ERR_CAPACITY); continue; }
     uint4* dst = reinterpret_cast<uint4*>((is_v ? v.v_pages : v.k_pages) + (page * v.C + r) * D) + lane16;
-    const uint4* src = (is_v ? v_new : k_new) + (long long)s * 16 + lane16;
+    const uint4* src = (is_v ? v_new : k_new) + row * 16 + lane16;
     *dst = __ldg(src);
   }
 }
 
-__global__ void kve_advance_len_kernel(int32_t* seq_len, int B, int max_tokens, int32_t* status) {
+__global__ void kve_advance_len_kernel(int32_t* seq_len, int B, int n_new, int max_tokens, int32_t* status) {
   pdl_launch_dependents();
   pdl_wait();
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int n = seq_len[b];
-  if (n < 0 || n >= max_tokens) set_status(status, ERR_CAPACITY);      // full: nothing was written
-  else seq_len[b] = n + 1;
+  if (n < 0 || n + n_new > max_tokens) set_status(status, ERR_CAPACITY);      // no room: nothing was written
+  else seq_len[b] = n + n_new;
 }
 
 __global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
@@ -85,13 +87,14 @@ cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_n
                     static_cast<const uint4*>(v_new), n_new, pos0);
 }
 
-cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, cudaStream_t st) {
-  long long blocks = ((long long)v.S * 32 + 255) / 256;
+cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st) {
+  long long blocks = ((long long)v.S * n_new * 32 + 255) / 256;
   if (blocks > 148LL * 32) blocks = 148LL * 32;
   cudaError_t e = launch_pdl(kve_append_next_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v,
-                             static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new));
+                             static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), n_new);
   if (e != cudaSuccess) return e;
-  return launch_pdl(kve_advance_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, v.max_tokens, v.status);
+  return launch_pdl(kve_advance_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n_new, v.max_tokens,
+                    v.status);
 }
 
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st) {

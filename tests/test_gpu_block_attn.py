@@ -172,3 +172,37 @@ def test_block_attention_at_the_benchmarked_size():
     assert 0.4 < pb.cnt64.mean() / pb.Nc < 0.6
     _check(b, pb, st, "summary", 4, 7)
     _check(b, pb, st, "summary", 4, 7, dense=True, step=1)
+
+
+def test_action_token_loop_replays_from_a_cuda_graph():
+    """One control step = append the 7 new tokens of every KV head, then attend with the 7 query tokens
+    on all query heads: captured once, replayed three times, each step against the oracle on the cache
+    as it then stands."""
+    wl = wlm.CFG1.small(B=2, H=2, n=1200, C=64, W=256, seed=29, n_append=40)
+    G, T, steps = 4, 7, 3
+    b, pb, st = _prepared(wl, "summary", G, T)
+    k_in = torch.zeros((st.S, T, 128), dtype=torch.bfloat16, device="cuda")
+    v_in = torch.zeros_like(k_in)
+    q_in = torch.zeros((wl.B, T, wl.H * G, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(q_in)
+    side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            st.append_next(0, k_in, v_in, n_reserve=(steps - 1) * T)
+            st.decode_attn_block(0, q_in, out=out)
+    torch.cuda.current_stream().wait_stream(side)
+    K, V = pb.K, pb.V
+    for step in range(steps):
+        kn, vn = wlm.gen_new_tokens(wl, 0, step, n_new=T)
+        q = wlm.gen_q_block(wl, T, wl.H * G, 0, 10 + step)
+        k_in.copy_(b.bits_to_bf16(kn)); v_in.copy_(b.bits_to_bf16(vn)); q_in.copy_(b.bits_to_bf16(q))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        K, V = np.concatenate([K, kn], axis=1), np.concatenate([V, vn], axis=1)
+        args = (wl.C, pb.Nc, pb.idx64, pb.cnt64, pb.sm64["ksum_b16"])
+        want, _, _ = pb.o64.attn_block(q, wl.H, K, V, *args, pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)
+        spread, _, _ = pb.o64.attn_block(q, wl.H, K, V & 0x7FFF, *args, pb.sm64["vsum_b16"] & 0x7FFF, hz.ATT["summary"], hz.SCALE)
+        hz.check_output_bf16_weights(b.bf16_to_bits(out), want, spread, f"action-token loop, step {step}")
+    assert int(st.seq_len[0, 0]) == wl.n + steps * T
