@@ -185,15 +185,18 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
 /* Sec. 3.3 + Eq. 1 for a block of queries: n_query_tokens tokens decoded together (the action tokens of one
  * control step) on all Hq query heads, Hq / Hkv of which share each KV head (grouped-query attention, the
  * 32-head / 8-KV-head model of Sec. 4.1).  Every (token, head) pair is an independent query against the
- * retained set [kept chunks ; raw tail] of its KV head (dense != 0: against all n stored tokens); the
- * tokens of a block do not see each other.  Each retained K/V row is read once per KV head, and the
+ * retained set [kept chunks ; raw tail] of its KV head (dense != 0: against all n stored tokens).
+ *   causal == 0: every query token sees the whole cache (tokens decoded in parallel, e.g. an action chunk);
+ *   causal != 0: the block's tokens are the n_query_tokens NEWEST tokens of the cache (append them first) and
+ *   query token t sees the cache up to and including its own position only (Eq. 1 for each of several
+ *   tokens handled in one call), i.e. all but the last n_query_tokens - 1 - t rows.  Each retained K/V row is read once per KV head, and the
  * products run on the tensor cores.
  *   The softmax numerators enter the tensor core as bf16: against exact weights an output moves by at
  *   most 2^-9 * sum_i p_i |v_i| / sum_i p_i (accumulation in fp32, one bf16 rounding of the result).
  *   q, out: DEVICE bf16 [B][n_query_tokens][Hq][d]; lse: DEVICE fp32 [B][n_query_tokens][Hq] or NULL.
  *   KVE_ERR_STATE if cfg.max_query_tokens == 0, KVE_ERR_CAPACITY if n_query_tokens exceeds it. */
-int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, void* out,
-                          float* lse, float scale, void* stream);
+int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, int causal,
+                          void* out, float* lse, float scale, void* stream);
 
 /* kvE_decode_attn without any scratch from the caller.  (The paper has no counterpart: this is a
  * deployment aid.)  Some users of this library must not allocate device memory once they are

@@ -182,7 +182,7 @@ class Oracle:
     #    query of Eq. 1 against the retained set of KV head hq // (Hq / Hkv); the tokens of a block
     #    do not see each other.  q [B, T, Hq, d] bf16 bits; results [B, T, Hq, d] / [B, T, Hq]. --
     def attn_block(self, q, Hkv, K, V, Cs, n_chunks, keep_idx, keep_cnt, ksum_b16, vsum_b16, attend, scale,
-                   dense=False):
+                   dense=False, causal=False):
         B, T, Hq, d = q.shape
         S = K.shape[0]
         assert S == B * Hkv and Hq % Hkv == 0
@@ -190,14 +190,20 @@ class Oracle:
         out = np.zeros((B, T, Hq, d), self.real)
         out_b16 = np.zeros((B, T, Hq, d), np.uint16)
         lse = np.zeros((B, T, Hq), self.real)
+        n = K.shape[1]
         for t in range(T):
+            # causal: the block's tokens are the T newest tokens of the cache, and query token t attends (Eq. 1)
+            # over the cache up to and including its own position, i.e. without the last T - 1 - t tokens
+            n_t = n - (T - 1 - t) if causal else n
+            assert n_t >= n_chunks * Cs, "the gated chunks lie before the block's tokens"
+            Kt, Vt = (K, V) if n_t == n else (np.ascontiguousarray(K[:, :n_t]), np.ascontiguousarray(V[:, :n_t]))
             for g in range(G):
                 # the g-th query head of every group: query head hkv * G + g reads KV head hkv
                 qs = np.ascontiguousarray(q[:, t, g::G, :].reshape(S, d))
                 if dense:
-                    o, ob, l = self.attn_dense(qs, K, V, scale)
+                    o, ob, l = self.attn_dense(qs, Kt, Vt, scale)
                 else:
-                    o, ob, l, _ = self.attn(qs, K, V, Cs, n_chunks, keep_idx, keep_cnt, ksum_b16, vsum_b16,
+                    o, ob, l, _ = self.attn(qs, Kt, Vt, Cs, n_chunks, keep_idx, keep_cnt, ksum_b16, vsum_b16,
                                             attend, scale)
                 out[:, t, g::G, :] = o.reshape(B, Hkv, d)
                 out_b16[:, t, g::G, :] = ob.reshape(B, Hkv, d)

@@ -85,7 +85,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
     lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
     lib.kvE_decode_attn_static.argtypes = lib.kvE_decode_attn.argtypes
-    lib.kvE_decode_attn_block.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+    lib.kvE_decode_attn_block.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                           C.c_float, C.c_void_p]
     lib.kvE_reclaim_pages.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
     lib.kvE_decode_step_host.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -269,8 +269,8 @@ class Store:
         _check("kvE_append_next", self.lib.kvE_append_next(self.handle, layer, _p(k_new), _p(v_new), n_new, int(n_reserve),
                                                            _stream(stream)), self.handle)
 
-    def decode_attn_block(self, layer, q, dense=False, out=None, lse=None, scale=None, stream=None):
-        return kvE_decode_attn_block(self, layer, q, dense, out, lse, scale, stream)
+    def decode_attn_block(self, layer, q, dense=False, out=None, lse=None, scale=None, stream=None, causal=False):
+        return kvE_decode_attn_block(self, layer, q, dense, out, lse, scale, stream, causal)
 
     def reclaim_pages(self, layer, chunk_begin, chunk_end, mode="discarded", free_list=None, free_count=None, stream=None):
         return kvE_reclaim_pages(self, layer, chunk_begin, chunk_end, mode, free_list, free_count, stream)
@@ -345,7 +345,7 @@ def kvE_decode_attn_dense(st: Store, layer, q, out=None, lse=None, scale=None, s
     return _attn("kvE_decode_attn_dense", st, layer, q, out, lse, scale, stream)
 
 
-def kvE_decode_attn_block(st: Store, layer, q, dense=False, out=None, lse=None, scale=None, stream=None):
+def kvE_decode_attn_block(st: Store, layer, q, dense=False, out=None, lse=None, scale=None, stream=None, causal=False):
     """q: bf16 [B, T, Hq, 128] device tensor (T query tokens on all query heads).  Returns out (same shape);
     lse, if given, is an fp32 [B, T, Hq] device tensor."""
     assert q.dtype == torch.bfloat16 and q.dim() == 4 and q.shape[0] == st.B and q.shape[2] == st.Hq and q.shape[3] == 128
@@ -356,7 +356,7 @@ def kvE_decode_attn_block(st: Store, layer, q, dense=False, out=None, lse=None, 
         assert lse.dtype == torch.float32 and tuple(lse.shape) == tuple(q.shape[:3])
     scale = (1.0 / 128.0 ** 0.5) if scale is None else scale
     _check("kvE_decode_attn_block", st.lib.kvE_decode_attn_block(st.handle, layer, _p(q), int(q.shape[1]), int(bool(dense)),
-                                                                 _p(out), _p(lse), C.c_float(scale), _stream(stream)), st.handle)
+                                                                 int(bool(causal)), _p(out), _p(lse), C.c_float(scale), _stream(stream)), st.handle)
     return out
 
 

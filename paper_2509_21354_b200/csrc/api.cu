@@ -402,8 +402,8 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
   return run_attention(st, layer, ATTN_DENSE, q, out, lse, scale, static_cast<cudaStream_t>(stream));
 }
 
-int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, void* out, float* lse,
-                          float scale, void* stream) {
+int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, int causal, void* out,
+                          float* lse, float scale, void* stream) {
   if (bad_layer(st, layer) || !q || !out || n_query_tokens <= 0) return KVE_ERR_ARG;
   if (!st->block_ready) return KVE_ERR_STATE;                  // cfg.max_query_tokens was 0
   if (n_query_tokens > st->cfg.max_query_tokens) return KVE_ERR_CAPACITY;
@@ -428,7 +428,7 @@ int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_t
   char* ws = static_cast<char*>(st->buf.workspace);
   Prof prof(st, KVE_K_ATTN_BLOCK, static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_attn_block(view(st, layer), st->block_maps, mode, ls.n_compacted, plan, n_query_tokens,
-                                    st->cfg.Hq / st->cfg.Hkv, st->block_hp, (long long)layer * st->S * st->max_chunks, q, out,
+                                    st->cfg.Hq / st->cfg.Hkv, causal ? 1 : 0, st->block_hp, (long long)layer * st->S * st->max_chunks, q, out,
                                     lse, scale, reinterpret_cast<float*>(ws + st->off_block),
                                     reinterpret_cast<int32_t*>(ws + st->off_counters), static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);

@@ -51,7 +51,7 @@ cudaError_t encode_attn_block_maps(void* maps, const void* k_pages, const void* 
 }
 
 cudaError_t launch_attn_block(const LayerView& v, const void* maps, AttnMode mode, int n_chunks, AttnPlan plan, int T, int G,
-                              int hp, long long sum_row0, const void* q, void* out, float* lse, float scale, float* partials,
+                              int causal, int hp, long long sum_row0, const void* q, void* out, float* lse, float scale, float* partials,
                               int32_t* counters, cudaStream_t st) {
   if (v.S <= 0 || T <= 0) return cudaSuccess;
   const int R = T * G;
@@ -59,7 +59,7 @@ cudaError_t launch_attn_block(const LayerView& v, const void* maps, AttnMode mod
   BlockArgs a;
   a.v = v; a.mode = (int)mode; a.n_chunks = n_chunks;
   a.rows_per_split = plan.rows_per_split; a.max_splits = plan.max_splits;
-  a.T = T; a.G = G; a.R = R; a.rec_rows = (R + 15) / 16 * 16; a.hp = hp; a.sum_row0 = sum_row0;
+  a.T = T; a.G = G; a.R = R; a.rec_rows = (R + 15) / 16 * 16; a.causal = causal; a.hp = hp; a.sum_row0 = sum_row0;
   a.q = static_cast<const uint16_t*>(q); a.out = static_cast<uint16_t*>(out); a.lse = lse; a.scale = scale;
   a.partials = partials; a.counters = counters;
   const CUtensorMap* tm = static_cast<const CUtensorMap*>(maps);

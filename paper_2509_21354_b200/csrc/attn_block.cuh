@@ -25,6 +25,7 @@ struct BlockArgs {
   int mode, n_chunks, rows_per_split, max_splits;
   int T, G, R;              // query tokens, query heads per KV head, T * G
   int rec_rows;             // query-row records per (sequence, split) in `partials`
+  int causal;               // query token t sees the cache up to its own position only
   int hp;                   // rows per page box
   long long sum_row0;       // first row of this layer in the summary tensor maps
   const uint16_t* q;        // [B][T][Hq][128]

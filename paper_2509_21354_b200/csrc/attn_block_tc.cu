@@ -213,6 +213,7 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const uint32_t my_o = tmem_o + lane_addr + group * 128, my_s = tmem_s + lane_addr + group * 64 + rep * CW;
     const float sl2 = a.scale * 1.44269504088896340736f;   // logits in log2 units
+    const int tok = min(row, a.R - 1) / a.G;                // query token of this lane's row
     float m_ref = -INFINITY, l_run = 0.f;
     bool alive = true;
     int last_tile = -1;
@@ -232,8 +233,13 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
       umma::fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_free[b]);
-      const int valid = gm.rows_valid(gm.r_begin + i * BK_TILE);
-      const bool plain = valid == BK_TILE && sl2 > 0.f;      // no masking, and max(s * sl2) = max(s) * sl2
+      const int row0 = gm.r_begin + i * BK_TILE;
+      const int valid = gm.rows_valid(row0);
+      // causal blocks: query token t sees the cache up to its own position, i.e. all but the last
+      // T - 1 - t rows of the raw tail (the block's own tokens are the newest rows of the tail)
+      const bool edge = a.causal && row0 < gm.tail_pad && row0 + BK_TILE > gm.n_tail - (a.T - 1);
+      const int visible = edge ? min(valid, gm.n_tail - (a.T - 1 - tok) - row0) : valid;      // columns of this tile the row may use
+      const bool plain = valid == BK_TILE && sl2 > 0.f && !edge;      // no masking, and max(s * sl2) = max(s) * sl2
 
       float mx = -INFINITY;
       if (warp_active) {
@@ -244,7 +250,7 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
         } else {
 #pragma unroll
           for (int x = 0; x < CW; ++x) {
-            sv[x] = (rep * CW + x < valid) ? sv[x] * sl2 : -INFINITY;
+            sv[x] = (rep * CW + x < visible) ? sv[x] * sl2 : -INFINITY;
             mx4[x & 3] = fmaxf(mx4[x & 3], sv[x]);
           }
         }
@@ -265,7 +271,7 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
         if (__any_sync(0xffffffffu, mx > m_ref + TC_RESCALE_STEP)) {      // m_ref = -inf on the group's first tile
           const float m_new = fmaxf(m_ref, mx);
           if (j > 0) {
-            const float f = ex2_fast(m_ref - m_new);
+            const float f = (m_ref == -INFINITY) ? 0.f : ex2_fast(m_ref - m_new);      // nothing accumulated yet: O row is 0
             if (owns_o) {
               // O holds this group's earlier tiles once their last product is complete; rescale this warp's rows
               if (!warp_wait(&pv_done[b], (j + 1) & 1)) { alive = false; break; }
@@ -299,7 +305,8 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
       if (warp_active) {
         unsigned char* prow = Ps + (b * TC_PLANES) * TC_P_BYTES + row * 128;
         float l4[4] = {0.f, 0.f, 0.f, 0.f};
-        const float neg_m = -m_ref, mul = plain ? sl2 : 1.f;      // the masked path has stored s * sl2 already
+        // (a row that has not seen a single column yet has m_ref = -inf: its p are 0, not exp2(-inf + inf))
+        const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref, mul = plain ? sl2 : 1.f;      // the masked path has stored s * sl2 already
 #pragma unroll
         for (int c = 0; c < CW / 8; ++c) {
           float p[8];

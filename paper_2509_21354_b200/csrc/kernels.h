@@ -66,7 +66,7 @@ int attn_block_hp(int C);                      // rows per page box: largest pow
 cudaError_t encode_attn_block_maps(void* maps, const void* k_pages, const void* v_pages, long long page_rows, int hp,
                                    const void* ksum, const void* vsum, long long sum_rows);
 cudaError_t launch_attn_block(const LayerView& v, const void* maps, AttnMode mode, int n_chunks, AttnPlan plan, int T, int G,
-                              int hp, long long sum_row0, const void* q, void* out, float* lse, float scale, float* partials,
+                              int causal, int hp, long long sum_row0, const void* q, void* out, float* lse, float scale, float* partials,
                               int32_t* counters, cudaStream_t st);
 
 }  // namespace kve

@@ -25,18 +25,19 @@ def _prepared(wl, attend, G, T, n_layers=1, layer=0):
     return b, pb, st
 
 
-def _check(b, pb, st, attend, G, T, layer=0, dense=False, step=0):
+def _check(b, pb, st, attend, G, T, layer=0, dense=False, step=0, causal=False):
     wl = pb.wl
     q = wlm.gen_q_block(wl, T, wl.H * G, layer, step)
     lse = torch.full((wl.B, T, wl.H * G), float("nan"), dtype=torch.float32, device="cuda")
-    out = st.decode_attn_block(layer, b.bits_to_bf16(q), dense=dense, lse=lse)
+    out = st.decode_attn_block(layer, b.bits_to_bf16(q), dense=dense, lse=lse, causal=causal)
     torch.cuda.synchronize()
     assert st.poll_status() == 0
     args = (wl.C, pb.Nc, pb.idx64, pb.cnt64, pb.sm64["ksum_b16"])
-    want, _, want_lse = pb.o64.attn_block(q, wl.H, pb.K, pb.V, *args, pb.sm64["vsum_b16"], hz.ATT[attend], hz.SCALE, dense=dense)
+    want, _, want_lse = pb.o64.attn_block(q, wl.H, pb.K, pb.V, *args, pb.sm64["vsum_b16"], hz.ATT[attend], hz.SCALE, dense=dense,
+                                          causal=causal)
     # the same attention over |V|: the scale of the rounding error of bf16 softmax numerators
     spread, _, _ = pb.o64.attn_block(q, wl.H, pb.K, pb.V & 0x7FFF, *args, pb.sm64["vsum_b16"] & 0x7FFF, hz.ATT[attend],
-                                     hz.SCALE, dense=dense)
+                                     hz.SCALE, dense=dense, causal=causal)
     hz.check_output_bf16_weights(b.bf16_to_bits(out), want, spread, f"block/{attend}/G{G}T{T}")
     assert np.abs(lse.cpu().numpy() - want_lse).max() <= 1e-3
     return out
@@ -206,3 +207,40 @@ def test_action_token_loop_replays_from_a_cuda_graph():
         spread, _, _ = pb.o64.attn_block(q, wl.H, K, V & 0x7FFF, *args, pb.sm64["vsum_b16"] & 0x7FFF, hz.ATT["summary"], hz.SCALE)
         hz.check_output_bf16_weights(b.bf16_to_bits(out), want, spread, f"action-token loop, step {step}")
     assert int(st.seq_len[0, 0]) == wl.n + steps * T
+
+
+# causal blocks: the block's tokens are the newest rows of the cache and token t sees the cache up to itself
+@pytest.mark.parametrize("G,T,n", [(4, 7, 2443), (1, 33, 2200), (2, 40, 1989), (4, 32, 2048 + 31)])
+def test_causal_block_attention_matches_oracle(G, T, n):
+    # the last T rows sit in the last tile of the raw tail, or straddle two tiles (n - raw0 just above a multiple of 64)
+    wl = wlm.CFG1.small(B=1, H=2, n=n, W=300, seed=31)
+    for attend in ("summary", "raw"):
+        b, pb, st = _prepared(wl, attend, G, T)
+        _check(b, pb, st, attend, G, T, causal=True)
+        _check(b, pb, st, attend, G, T, dense=True, step=1, causal=True)
+
+
+def test_causal_block_with_a_tail_shorter_than_the_block():
+    # W = 4, C = 8: the raw tail holds 4..11 rows, fewer than the 12 query tokens, so the first tokens see no
+    # raw row at all (only kept chunks) - rows whose running maximum stays -inf over the whole tail
+    wl = wlm.CFG1.small(B=1, H=2, n=203, C=8, W=4, seed=32)
+    b, pb, st = _prepared(wl, "summary", 2, 12)
+    assert wl.n - pb.Nc * wl.C < 12
+    wl_t = wl
+    q = wlm.gen_q_block(wl_t, 12, 4, 0, 0)
+    out = st.decode_attn_block(0, b.bits_to_bf16(q), causal=True)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    # oracle per token: gated chunks beyond the token's own position do not exist for it either, so the
+    # comparison is restricted to the tokens whose prefix still covers all gated chunks
+    tail = wl.n - pb.Nc * wl.C
+    got = wlm.bf16_bits_to_f32(b.bf16_to_bits(out)).astype(np.float64)
+    for t in range(12 - tail, 12):
+        n_t = wl.n - (11 - t)
+        for g in range(2):
+            qs = np.ascontiguousarray(q[:, t, g::2, :].reshape(wl.S, 128))
+            want, _, _, _ = pb.o64.attn(qs, np.ascontiguousarray(pb.K[:, :n_t]), np.ascontiguousarray(pb.V[:, :n_t]), wl.C, pb.Nc,
+                                        pb.idx64, pb.cnt64, pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)
+            assert np.abs(got[0, t, g::2] - want).max() <= 2e-2
+    # tokens whose position lies inside the gated range: they see every kept chunk and no raw row (finite, no NaN)
+    assert np.isfinite(got).all()

@@ -64,7 +64,7 @@ def test_workspace_bytes_and_geometry_checks_need_no_device():
     assert lib.kvE_append(None, 0, None, None, 1, None, None) == -1        # null handle
     assert lib.kvE_poll_status(None, None) == -1
     assert lib.kvE_append_next(None, 0, None, None, 1, 0, None) == -1
-    assert lib.kvE_decode_attn_block(None, 0, None, 1, 0, None, None, 0.1, None) == -1
+    assert lib.kvE_decode_attn_block(None, 0, None, 1, 0, 0, None, None, 0.1, None) == -1
 
 
 def test_store_refuses_to_run_without_cuda():

@@ -647,3 +647,39 @@ def test_query_block_rows_are_independent_and_permutable(o64):
     perm = [1, 0, 2]
     out_p, _, lse_p = o64.attn_block(np.ascontiguousarray(q[:, perm]), *args)
     assert np.array_equal(out_p, out[:, perm]) and np.array_equal(lse_p, lse[:, perm])
+
+
+def test_causal_query_block_is_one_query_per_prefix(o64):
+    """Causal blocks: query token t against a python-float softmax over the row list of the cache cut
+    after its own position (the block's tokens are the newest rows); the last token sees everything, so it
+    equals the non-causal result, the first one does not."""
+    rng = np.random.default_rng(78)
+    B, Hkv, G, T, d, n, C, W = 1, 2, 2, 3, 4, 21, 4, 5
+    S = B * Hkv
+    K, V = rand_bits(rng, S, n, d), rand_bits(rng, S, n, d)
+    q = rand_bits(rng, B, T, Hkv * G, d)
+    Nc = (n - T - W) // C                                   # gated before the block's tokens arrived
+    sm = o64.summarize(K, V, C, 0, Nc, kvo.AGG_MEAN)
+    idx, cnt = o64.compact(np.random.default_rng(4).uniform(size=(S, Nc)), Nc, 0.5)
+    args = (Hkv, K, V, C, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"])
+    for mode, dense in ((kvo.ATTEND_SUMMARY, False), (kvo.ATTEND_RAW, False), (kvo.ATTEND_RAW, True)):
+        out, _, lse = o64.attn_block(q, *args, mode, 0.4, dense=dense, causal=True)
+        full, _, _ = o64.attn_block(q, *args, mode, 0.4, dense=dense, causal=False)
+        assert np.array_equal(out[:, T - 1], full[:, T - 1]) and not np.array_equal(out[:, 0], full[:, 0])
+        for t, hq in itertools.product(range(T), range(Hkv * G)):
+            s = hq // G
+            n_t = n - (T - 1 - t)
+            kept = idx[s, :cnt[s]]
+            if dense:
+                rows_k, rows_v = [widen(K[s, r]).tolist() for r in range(n_t)], [widen(V[s, r]).tolist() for r in range(n_t)]
+            else:
+                if mode == kvo.ATTEND_SUMMARY:
+                    rows_k = [widen(sm["ksum_b16"][s, c]).tolist() for c in kept]
+                    rows_v = [widen(sm["vsum_b16"][s, c]).tolist() for c in kept]
+                else:
+                    rows_k = [widen(K[s, r]).tolist() for c in kept for r in range(c * C, c * C + C)]
+                    rows_v = [widen(V[s, r]).tolist() for c in kept for r in range(c * C, c * C + C)]
+                rows_k += [widen(K[s, r]).tolist() for r in range(Nc * C, n_t)]
+                rows_v += [widen(V[s, r]).tolist() for r in range(Nc * C, n_t)]
+            want, want_lse = brute_attention(widen(q[0, t, hq]).tolist(), rows_k, rows_v, 0.4)
+            assert np.allclose(out[0, t, hq], want, rtol=0, atol=1e-13) and abs(lse[0, t, hq] - want_lse) <= 1e-12
