@@ -26,7 +26,7 @@ struct kvE_store {
   kvE_buffers buf;
   int S, max_chunks;
   // workspace carve-up (byte offsets)
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_block, ws_needed;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, ws_needed;
   int max_splits;
   // block-of-queries attention: tensor maps over the page pools and the summary store (encoded at
   // create when cfg.max_query_tokens > 0), rows per page box, split cap the workspace was sized for
@@ -68,7 +68,7 @@ int check_config(const kvE_config* c) {
 }
 
 struct Carve {
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_block, total;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, total;
 };
 // most splits per sequence the block-of-queries attention uses: one CTA per SM, one wave
 int block_split_cap(long long S) {
@@ -85,6 +85,7 @@ Carve carve(const kvE_config& c) {
   k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
   k.off_stage = o;    o = align_up(o + 4 * S * 128 * 2);   // k_new, v_new, q, out of kvE_decode_step_host
   k.off_reclaim = o;  o = align_up(o + (2 * S + 1) * sizeof(int32_t));   // per-sequence counts and offsets of kvE_reclaim_pages
+  k.off_ticket = o;   o = align_up(o + sizeof(int32_t));       // last-CTA ticket of kvE_append_next
   k.off_block = o;    // split records of kvE_decode_attn_block: [S][splits][query rows, padded to 16][132] fp32
   if (c.max_query_tokens > 0) {
     const size_t rows = ((size_t)c.max_query_tokens * (c.Hq / c.Hkv) + 15) / 16 * 16;
@@ -208,7 +209,7 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   st->S = cfg->B * cfg->Hkv;
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
   st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
-  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_block = k.off_block; st->ws_needed = k.total;
+  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_ticket = k.off_ticket; st->off_block = k.off_block; st->ws_needed = k.total;
   if (cfg->max_query_tokens > 0) {
     st->block_hp = attn_block_hp(cfg->C);
     st->block_split_cap = block_split_cap(st->S);
@@ -263,7 +264,8 @@ int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_n
   LayerState& ls = st->layers[layer];
   if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   Prof prof(st, KVE_K_APPEND, static_cast<cudaStream_t>(stream));
-  cudaError_t e = launch_append_next(view(st, layer), k_new, v_new, n_new, static_cast<cudaStream_t>(stream));
+  int32_t* ticket = reinterpret_cast<int32_t*>(static_cast<char*>(st->buf.workspace) + st->off_ticket);
+  cudaError_t e = launch_append_next(view(st, layer), k_new, v_new, n_new, ticket, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
   long long upper = (long long)ls.n_tokens + n_new + n_reserve;
   if (upper > st->cfg.max_tokens) upper = st->cfg.max_tokens;

@@ -35,10 +35,11 @@ __global__ void __launch_bounds__(256) kve_append_kernel(LayerView v, const uint
 }
 
 // n_new tokens per sequence from the position the DEVICE holds in seq_len (replayable from a CUDA graph: nothing
-// about the position is baked into the launch).  The length itself is advanced by the kernel below,
-// which runs after this one in stream order, so every thread here reads the old length.
+// about the position is baked into the launch).  Every CTA reads the old length before it writes; the
+// last CTA to finish (atomic ticket, nobody spins) advances the length and resets the ticket, so no CTA
+// can see the new length while it is still placing rows.
 __global__ void __launch_bounds__(256) kve_append_next_kernel(LayerView v, const uint4* __restrict__ k_new,
-                                                              const uint4* __restrict__ v_new, int n_new) {
+                                                              const uint4* __restrict__ v_new, int n_new, int32_t* ticket) {
   pdl_launch_dependents();
   pdl_wait();
   const long long total = (long long)v.S * n_new * 32;
@@ -49,7 +50,7 @@ __global__ void __launch_bounds__(256) kve_append_next_kernel(LayerView v, const
     const long long row = idx >> 5;              // s * n_new + i
     const int s = (int)(row / n_new);
     const int n0 = v.seq_len[s / v.H];
-    if (n0 < 0 || n0 + n_new > v.max_tokens) continue;  // no room: flagged by the length kernel, nothing written
+    if (n0 < 0 || n0 + n_new > v.max_tokens) continue;  // no room: flagged below, nothing written
     const int pos = n0 + (int)(row - (long long)s * n_new);
     const int chunk = pos / v.C;
     const int r = pos - chunk * v.C;
@@ -59,16 +60,18 @@ __global__ void __launch_bounds__(256) kve_append_next_kernel(LayerView v, const
     const uint4* src = (is_v ? v_new : k_new) + row * 16 + lane16;
     *dst = __ldg(src);
   }
-}
-
-__global__ void kve_advance_len_kernel(int32_t* seq_len, int B, int n_new, int max_tokens, int32_t* status) {
-  pdl_launch_dependents();
-  pdl_wait();
-  int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= B) return;
-  const int n = seq_len[b];
-  if (n < 0 || n + n_new > max_tokens) set_status(status, ERR_CAPACITY);      // no room: nothing was written
-  else seq_len[b] = n + n_new;
+  __shared__ int last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1) ? 1 : 0;
+  __syncthreads();
+  if (!last) return;
+  for (int b = threadIdx.x; b < v.B; b += blockDim.x) {
+    const int n = v.seq_len[b];
+    if (n < 0 || n + n_new > v.max_tokens) set_status(v.status, ERR_CAPACITY);      // no room: nothing was written
+    else v.seq_len[b] = n + n_new;
+  }
+  if (threadIdx.x == 0) *ticket = 0;      // clean for the next launch
 }
 
 __global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
@@ -87,14 +90,12 @@ cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_n
                     static_cast<const uint4*>(v_new), n_new, pos0);
 }
 
-cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st) {
+cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, int32_t* ticket,
+                               cudaStream_t st) {
   long long blocks = ((long long)v.S * n_new * 32 + 255) / 256;
   if (blocks > 148LL * 32) blocks = 148LL * 32;
-  cudaError_t e = launch_pdl(kve_append_next_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v,
-                             static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), n_new);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(kve_advance_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n_new, v.max_tokens,
-                    v.status);
+  return launch_pdl(kve_append_next_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v, static_cast<const uint4*>(k_new),
+                    static_cast<const uint4*>(v_new), n_new, ticket);
 }
 
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st) {

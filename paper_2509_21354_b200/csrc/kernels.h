@@ -43,7 +43,8 @@ constexpr int ATTN_PARTIAL_FLOATS = 132;       // acc[128], m, l, 2 pad: keeps e
 
 cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, int pos0, cudaStream_t st);
 cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st);
-cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, cudaStream_t st);
+cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, int32_t* ticket,
+                               cudaStream_t st);
 cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st);
 cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st);
 cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t* W_ih, const float* b_ih,
