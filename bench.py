@@ -437,6 +437,24 @@ def run_ours(args, rank, world, local_rank):
     us["attn_dense"] = float(np.mean(cold["attn_dense"]))
     us_attn_cold = float(np.mean(cold["attn"]))
     by = algorithmic_bytes(wl, Nc, keep_mean, R, args.attend)
+
+    def copy_us(total_bytes):
+        """a plain device copy that moves total_bytes (read + write), timed like the kernels: L2 flushed, events"""
+        src = torch.empty(max(1, int(total_bytes) // 2), dtype=torch.uint8, device="cuda")
+        dst = torch.empty_like(src)
+        ts = []
+        for i in range(8):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            dst.copy_(src)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.mean(ts))
+
+    copy_gated_us, copy_dense_us = copy_us(by["attn_gated"]), copy_us(by["attn_dense"])
     by_kernel = {"append": S * 4 * 256, "chunk_mean": by["chunk_mean"], "chunk_mlp": by["chunk_mlp"],
                  "gate_proj": by["gate_proj"], "gate_rnn": by["gate_rnn"], "compact": by["compact"],
                  "attn": by["attn_gated"], "attn_dense": by["attn_dense"]}
@@ -505,6 +523,12 @@ def run_ours(args, rank, world, local_rank):
                                "gated_GB/s": kern["attn"]["GB/s_l2_flushed"], "dense_GB/s": kern["attn_dense"]["GB/s"],
                                "gated_frac_of_measured_peak": kern["attn"]["GB/s_l2_flushed"] / hbm,
                                "dense_frac_of_measured_peak": kern["attn_dense"]["GB/s"] / hbm,
+                               "size_matched_copy": {
+                                   "note": "a plain torch device copy moving the same number of bytes (read + write), "
+                                           "same timing method: what this transfer size allows on this GPU",
+                                   "gated_bytes_copy_us": copy_gated_us, "dense_bytes_copy_us": copy_dense_us,
+                                   "gated_frac_of_copy": copy_gated_us / us["attn_gated"],
+                                   "dense_frac_of_copy": copy_dense_us / us["attn_dense"]},
                                "gated_frac_of_nominal_8TBps": kern["attn"]["GB/s_l2_flushed"] / 8000.0,
                                "dense_frac_of_nominal_8TBps": kern["attn_dense"]["GB/s"] / 8000.0},
     }
