@@ -192,7 +192,7 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
  *   tokens handled in one call), i.e. all but the last n_query_tokens - 1 - t rows.  Each retained K/V row is read once per KV head, and the
  * products run on the tensor cores.
  *   The softmax numerators enter the tensor core as bf16: against exact weights an output moves by at
- *   most 2^-9 * sum_i p_i |v_i| / sum_i p_i (accumulation in fp32, one bf16 rounding of the result).
+ *   most 2^-8 * sum_i p_i |v_i| / sum_i p_i (accumulation in fp32, one bf16 rounding of the result).
  *   q, out: DEVICE bf16 [B][n_query_tokens][Hq][d]; lse: DEVICE fp32 [B][n_query_tokens][Hq] or NULL.
  *   KVE_ERR_STATE if cfg.max_query_tokens == 0, KVE_ERR_CAPACITY if n_query_tokens exceeds it. */
 int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, int causal,

@@ -17,7 +17,7 @@
 //               softmax at any time.  Thread = query row = tensor-memory lane.  Reads its 64 logits of the tile,
 //               p = exp2(s * scale * log2 e - m_ref) by the special-function unit, writes P as bf16 into
 //               the swizzled A-operand layout (rounding p moves an output by at most
-//               2^-9 sum p |v| / sum p; TC_PLANES = 2 adds a second plane p - bf16(p) and removes that
+//               2^-8 sum p |v| / sum p (bf16 keeps 8 significant bits: half a step is 2^-8 relative); TC_PLANES = 2 adds a second plane p - bf16(p) and removes that
 //               error at the price of a ring stage).  m_ref follows the running maximum lazily: only
 //               when a row's maximum has grown by more than 8 (log2 units) does the warp rescale its
 //               rows of O in tensor memory, so p stays below 2^8 and the usual per-tile rescale of O
@@ -38,7 +38,7 @@
 namespace kve {
 
 constexpr int TC_STAGES = 5;
-constexpr int TC_PLANES = 1;                       // bf16 planes of P (2: hi + lo, P exact to 2^-17, at the price of a ring stage)
+constexpr int TC_PLANES = 1;                       // bf16 planes of P (2: hi + lo, P exact to 2^-16, at the price of a ring stage)
 constexpr int TC_Q_BYTES = 2 * 128 * 128;          // two K-blocks [128 rows][128 bytes]
 constexpr int TC_P_BYTES = 128 * 128;              // one plane of one P buffer: [128 rows][64 bf16]
 constexpr int TC_OFF_Q = 0;

@@ -96,7 +96,7 @@ def test_block_of_one_row_agrees_with_the_single_query_kernel():
     torch.cuda.synchronize()
     one_b, blk_b = b.bf16_to_bits(one).reshape(-1), b.bf16_to_bits(blk).reshape(-1)
     # the block kernel rounds the softmax numerators to bf16, the single-query kernel does not: the two agree
-    # within that rounding (2^-9 of the typical |v| ~ 1) plus one bf16 step of the result
+    # within that rounding (2^-8 of the typical |v| ~ 1, in practice far less) plus one bf16 step of the result
     x, y = wlm.bf16_bits_to_f32(one_b).astype(np.float64), wlm.bf16_bits_to_f32(blk_b).astype(np.float64)
     assert np.all(np.abs(x - y) <= 2.0 ** -7 * np.abs(x) + 2.0 ** -9)
     assert np.abs(x - y).mean() <= 2e-4
@@ -244,3 +244,15 @@ def test_causal_block_with_a_tail_shorter_than_the_block():
             assert np.abs(got[0, t, g::2] - want).max() <= 2e-2
     # tokens whose position lies inside the gated range: they see every kept chunk and no raw row (finite, no NaN)
     assert np.isfinite(got).all()
+
+
+@pytest.mark.parametrize("n", [2048, 2051])
+def test_block_attention_without_window_and_with_large_chunks(n):
+    # W = 0 and n a multiple of C = 512: no raw row at all, the retained set is the kept chunks only
+    # (summary rows, or four tiles of raw rows per kept chunk); n = 2051: a three-row tail
+    wl = wlm.CFG1.small(B=1, H=3, n=n, C=512, W=0, seed=33)
+    for attend in ("summary", "raw"):
+        b, pb, st = _prepared(wl, attend, 4, 7)
+        assert pb.Nc == 4 and 0 < pb.cnt64.sum() < 12
+        _check(b, pb, st, attend, 4, 7)
+        _check(b, pb, st, attend, 4, 7, dense=True, step=2)
