@@ -256,3 +256,21 @@ def test_block_attention_without_window_and_with_large_chunks(n):
         assert pb.Nc == 4 and 0 < pb.cnt64.sum() < 12
         _check(b, pb, st, attend, 4, 7)
         _check(b, pb, st, attend, 4, 7, dense=True, step=2)
+
+
+def test_block_attention_after_the_gated_pages_were_handed_back():
+    """Sec. 3.3 memory reduction: once every gated chunk's page is back on the free list, the gated query-block
+    attention (summary rows + raw tail) still answers as before; the full-cache variant cannot and says so
+    through the status word instead of reading a page it no longer owns."""
+    wl = wlm.CFG1.small(B=1, H=2, n=1800, seed=34)
+    b, pb, st = _prepared(wl, "summary", 4, 7)
+    before = _check(b, pb, st, "summary", 4, 7).clone()
+    free_list, free_count = st.reclaim_pages(0, 0, pb.Nc, mode="gated")
+    torch.cuda.synchronize()
+    assert int(free_count) == wl.S * pb.Nc and st.poll_status() == 0
+    after = _check(b, pb, st, "summary", 4, 7)
+    assert torch.equal(before, after)
+    q = b.bits_to_bf16(wlm.gen_q_block(wl, 7, 8))
+    st.decode_attn_block(0, q, dense=True)
+    torch.cuda.synchronize()
+    assert st.poll_status() == -3
