@@ -101,7 +101,9 @@ typedef struct {
 
 typedef struct kvE_store kvE_store;
 
-/* Bytes of workspace the handle needs (gate projection buffer + attention split partials). */
+/* Bytes of workspace the handle needs: the gate projection buffer, the split-K partial records and tickets of
+ * the attention kernels (those of kvE_decode_attn_block only when cfg.max_query_tokens > 0), staging rows of the
+ * host-buffer step, scratch of kvE_reclaim_pages.  0 if the geometry is not supported. */
 size_t kvE_workspace_bytes(const kvE_config* cfg);
 
 /* Host-side handle.  Validates the geometry, zeroes workspace, status_word, seq_len and keep_cnt
