@@ -10,10 +10,12 @@
 //    HU = d_g / CL hidden units, i.e. 4*HU rows of W_hh, and keeps them in REGISTERS as mma A
 //    fragments for the whole kernel (128 registers per thread at d_g = 256, CL = 4).
 //  * Per step the CTA computes its rows of W_hh h for all its sequences with warp-level tensor-core
-//    MMAs (m16n8k16, bf16 x bf16 -> fp32).  W_hh is bf16 by definition; the fp32 state h is split
-//    exactly into three bf16 planes (h = hi + mid + lo), so the products are exact and only the
-//    accumulation order differs from a plain fp32 loop.  Each plane has its own accumulators
-//    (three times as many independent MMA chains), added smallest plane first at the end.
+//    MMAs (m16n8k16, bf16 x bf16 -> fp32).  W_hh is bf16 by definition; the fp32 state h enters as
+//    RNN_PLANES = 2 bf16 planes (h = hi + lo up to 2^-17 |h|: 16 of its 24 significant bits; a third
+//    plane makes the products exact, moves the scores by 1e-7 - far below what the fast
+//    exponentials of the cell update contribute, 5e-5 - and costs a third more MMAs: 119 vs 99 us
+//    on 256 sequences x 56 chunks).  Each plane has its own accumulators (as many independent MMA
+//    chains), added smallest plane first at the end.
 //  * MMA rows are ordered so that one thread ends up holding the i, f, g, o pre-activations of the
 //    same (hidden unit, sequence): the cell update is thread-local, c lives in registers.
 //  * Exchange of h_t: a warp gathers the planes of its 8 hidden units in a small staging area of
@@ -94,7 +96,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       const float2 hv = *reinterpret_cast<const float2*>(a.lstm_h + (long long)s * DG + k2 * 2);
       h0 = hv.x; h1 = hv.y;
     }
-    uint32_t p0[3], p1[3];
+    uint32_t p0[3], p1[3];      // the leading RNN_PLANES pieces are used
     split3(h0, p0);
     split3(h1, p1);
 #pragma unroll
@@ -212,7 +214,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
 #pragma unroll
           for (int q = 0; q < 4; ++q) {   // q: 0 = i, 1 = f (tile 2p, rows g / g+8), 2 = g, 3 = o (tile 2p+1)
             const int mt = 2 * p + (q >> 1), ai = (q & 1) * 2 + e;
-            pre[q] = ((acc[2][mt][ai] + acc[1][mt][ai]) + acc[0][mt][ai]) + pin[gi][p][q][e];
+            float sum = acc[RNN_PLANES - 1][mt][ai];      // smallest plane first
+#pragma unroll
+            for (int pl = RNN_PLANES - 2; pl >= 0; --pl) sum += acc[pl][mt][ai];
+            pre[q] = sum + pin[gi][p][q][e];
           }
           const float ig = fast_sigmoid(pre[0]);
           const float fg = fast_sigmoid(pre[1]);

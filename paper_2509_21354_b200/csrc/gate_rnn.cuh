@@ -9,7 +9,7 @@ namespace kve {
 
 constexpr int RNN_WARPS = 8;
 constexpr int RNN_THREADS = RNN_WARPS * 32;
-constexpr int RNN_PLANES = 3;
+constexpr int RNN_PLANES = 2;      // bf16 planes of h that enter the recurrent product (3 = exact)
 
 struct RnnArgs {
   float* P;                // [S * n_range][4 d_g]; columns [0, d_g) of row (s, t) receive h_t once P_t is consumed
