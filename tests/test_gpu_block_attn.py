@@ -274,3 +274,23 @@ def test_block_attention_after_the_gated_pages_were_handed_back():
     st.decode_attn_block(0, q, dense=True)
     torch.cuda.synchronize()
     assert st.poll_status() == -3
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_block_attention_random_geometries(seed):
+    """Seeded random small geometries (chunk size, window, length, heads, block shape, mode, causal or not)
+    against the oracle: the cases nobody thought of."""
+    rng = np.random.default_rng(1000 + seed)
+    C = int(rng.choice([8, 16, 24, 32, 64, 128]))
+    W = int(rng.integers(0, 3 * C + 1))
+    G = int(rng.choice([1, 2, 4, 8]))
+    T = int(rng.integers(1, 128 // G + 1)) if rng.random() < 0.3 else int(rng.integers(1, max(2, 32 // G) + 1))
+    n = int(rng.integers(max(T, 1), 1500))
+    attend = str(rng.choice(["summary", "raw"]))
+    causal = bool(rng.random() < 0.5)
+    wl = wlm.CFG1.small(B=int(rng.integers(1, 3)), H=int(rng.integers(1, 4)), n=n, C=C, W=W, seed=40 + seed)
+    b, pb, st = _prepared(wl, attend, G, T)
+    if causal and n - pb.Nc * C < T:
+        causal = False                      # the oracle's causal form wants the block's tokens inside the raw tail
+    _check(b, pb, st, attend, G, T, causal=causal)
+    _check(b, pb, st, attend, G, T, dense=True, step=1, causal=causal)

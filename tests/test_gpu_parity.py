@@ -656,3 +656,19 @@ def test_decode_loop_advances_under_a_cuda_graph():
         g2.replay()
     torch.cuda.synchronize()
     assert st2.poll_status() == -3
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_whole_path_random_geometries(seed):
+    """Seeded random small geometries (chunk size, window, length, gate width, aggregator, keep ratio, append
+    pattern) through append, summaries, gate, keep list and both attentions against the oracle."""
+    rng = np.random.default_rng(2000 + seed)
+    C = int(rng.choice([1, 3, 8, 16, 50, 64, 128]))
+    agg = "identity" if C == 1 else str(rng.choice(["mean", "mlp", "max"]))
+    W = int(rng.integers(0, 3 * C + 2))
+    n = int(rng.integers(1, 1200 if C > 1 else 300))
+    d_sum = int(rng.choice([8, 64, 200, 256])) if agg == "mlp" else 0
+    wl = wlm.CFG1.small(B=int(rng.integers(1, 4)), H=int(rng.integers(1, 5)), n=n, C=C, W=W, d_g=int(rng.choice([64, 128, 256])),
+                        agg=agg, d_sum=d_sum, seed=60 + seed)
+    pieces = tuple(sorted(rng.random(int(rng.integers(0, 3))).tolist())) + (1.0,)
+    full_check(wl, str(rng.choice(["summary", "raw"])), pieces=pieces, keep=float(rng.choice([0.25, 0.5, 0.75])))
