@@ -78,6 +78,9 @@ def check_summaries(st, pb, layer=0):
 
 def check_gate_and_keep(st, pb, layer=0):
     Nc = pb.Nc
+    if Nc == 0:                                    # nothing has left the window: no scores, empty keep lists
+        assert int(st.keep_cnt[layer].abs().sum()) == 0
+        return
     sc = st.scores[layer, :, :Nc].cpu().numpy()
     assert np.abs(sc - pb.sc32[:, :Nc]).max() <= 2e-4
     assert np.abs(sc - pb.sc64[:, :Nc]).max() <= 2e-4
@@ -658,7 +661,7 @@ def test_decode_loop_advances_under_a_cuda_graph():
     assert st2.poll_status() == -3
 
 
-@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("seed", list(range(12)) + [104])      # 104: nothing has left the window yet
 def test_whole_path_random_geometries(seed):
     """Seeded random small geometries (chunk size, window, length, gate width, aggregator, keep ratio, append
     pattern) through append, summaries, gate, keep list and both attentions against the oracle."""
