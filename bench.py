@@ -1,15 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the gated chunked-KV decode path (one JSON line on stdout).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg4] [--legs ...]
 
-A *step* is one pass of the whole hot path over one layer of the workload, from scratch:
+The headline workload is the largest single-GPU configuration (cfg4: batch 16, 32 heads, 16512 tokens,
+chunk 128, window 1024), one layer.  A *step* is one pass of the whole hot path over that layer, from scratch:
 append one token to every sequence, summarise every chunk that lies outside the window, run the
 LSTM gate over all of them, compact the keep list, run the gated decode attention.  `value` is
 whole-job steps per second with all inputs resident in HBM; `e2e` is the same step through
 kvE_decode_step_host with pinned HOST buffers (H2D of k_new, v_new, q and D2H of the output inside
-the timed region).  Under torchrun every rank runs the same per-GPU workload on its own batch
-shard (weak scaling, no data-path collective: (layer, batch, head) units are independent).
+the timed region).  The K-step loop is repeated R times (R in the line) so that the timed device work
+lasts at least --min-timed-s; the median loop gives `value`.  Under torchrun every rank runs the same
+per-GPU workload on its own batch shard (weak scaling, no data-path collective: (layer, batch, head)
+units are independent).
+
+The single-GPU run adds, in the same JSON line: `per_config` (cfg1..cfg4: from-scratch step, steady
+step, every kernel in-step and alone with L2 flushed, gated vs full-cache attention; cfg3 also as 7
+action tokens x 32 layers replayed from a CUDA graph), `sweep` (the stress sweep, bounded), `trigger`
+(the aggregation-and-gating step for one new chunk, and the step amortised over a chunk's tokens),
+`cpu_baseline` and `cpu_oracle_per_config` (the oracle on the host cores, single-threaded and OpenMP).
 
 `--impl reference` times the CPU oracle (oracle/, as it stands) on the host cores on a bounded
 sample of the same workload.
@@ -214,7 +223,7 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
             torch.cuda.synchronize()
             if i >= 2:
                 ts.append(st.profile_read()["attn_block"])
-        us = float(np.mean(ts))
+        us = float(np.median(ts))
         by = g.S * rows * 512                                  # every retained K and V row once per KV head
         fl = 4 * 128 * T * G * g.S * rows                      # Q K^T and P V
         res[name] = {"us": us, "kv_bytes": int(by), "GB/s": by / us / 1e3, "frac_of_hbm_peak": by / us / 1e3 / hbm,
@@ -225,7 +234,7 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
     return res
 
 
-def graph_tick_leg(wl, n_layers, seed, replays=20):
+def graph_tick_leg(wl, n_layers, seed, replays=20, mem_cap=40e9):
     """The decode loop of a whole model between two gate triggers: per token, for each of n_layers layers
     append the new token at the device-held length (kvE_append_next) and run the gated attention; all
     layers captured once in a CUDA graph, every replay advancing by one token.  Compared with the
@@ -234,7 +243,7 @@ def graph_tick_leg(wl, n_layers, seed, replays=20):
     from paper_2509_21354_b200 import binding as b
     g = wl.small(agg="mean", d_sum=0)                      # the aggregator only feeds the keep list here
     per_layer = g.S * (g.n + g.C) * 512 * 1.1
-    n_layers = max(1, min(n_layers, int(40e9 // per_layer)))
+    n_layers = max(1, min(n_layers, int(mem_cap // per_layer)))
     st = b.Store(B=g.B, H=g.H, C_=g.C, W=g.W, max_tokens=g.n + g.C, d_g=g.d_g, agg="mean", attend="summary",
                  n_layers=n_layers, page_perm="random", seed=seed)
     lstm = wlm.gen_lstm_weights(g)
@@ -308,193 +317,424 @@ def graph_tick_leg(wl, n_layers, seed, replays=20):
     return res
 
 
+# ---------------------------------------------------------------------------------------------- one workload on the device
+class Rig:
+    """One layer of a workload resident on the device: the cache holds n - 1 tokens, the gate's head bias is
+    tuned so that about `keep` of the stale chunks are retained (deterministic given the seed)."""
+
+    def __init__(self, wl, attend, seed, extra_tokens=0, keep=0.5):
+        import torch
+        from paper_2509_21354_b200 import binding as b
+        self.wl, self.attend, self.b = wl, attend, b
+        self.st = st = b.Store(B=wl.B, H=wl.H, C_=wl.C, W=wl.W, max_tokens=wl.n + wl.C + extra_tokens, d_g=wl.d_g, agg=wl.agg,
+                               d_sum=wl.d_sum, attend=attend, page_perm="random", seed=seed)
+        self.gen = g = fill_cache(st, wl, seed)
+        mlp, lstm = wlm.gen_mlp_weights(wl), wlm.gen_lstm_weights(wl)
+        self.aw = b.AggWeights(mlp) if mlp is not None else None
+        self.lw = b.LstmWeights(lstm)
+        S = self.S = wl.S
+        rnd = lambda: torch.randn((S, 128), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16).contiguous()
+        self.k_new, self.v_new, self.q = rnd(), rnd(), rnd()
+        self.k3, self.v3 = self.k_new.view(S, 1, 128), self.v_new.view(S, 1, 128)
+        self.out = torch.empty_like(self.q)
+        self.n0 = wl.n
+        self.Nc = wl.n_stale_chunks(wl.n)
+        self.R = wl.n - self.Nc * wl.C
+        self.step_full()
+        torch.cuda.synchronize()
+        if self.Nc > 0:
+            sc = st.scores[0, :, :self.Nc].double().clamp(1e-9, 1 - 1e-9)
+            logit = torch.log(sc / (1 - sc))
+            self.lw.set_b_s(float(-torch.quantile(logit.flatten()[:1 << 20], 1.0 - keep).item()) + lstm["b_s"])
+        self.step_full()
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        self.keep_mean = st.keep_cnt[0].float().mean().item()
+        self.rows_per_kept = wl.C if attend == "raw" else 1
+        self.n_eff = self.R + self.keep_mean * self.rows_per_kept
+
+    def step_full(self):
+        """the whole hot path from scratch: roll the last token back, append it, summarise every stale
+        chunk, gate them all, compact, gated attention"""
+        st, wl = self.st, self.wl
+        st.set_len(0, self.n0 - 1)
+        st.append(0, self.k3, self.v3)
+        st.summarize_chunks(0, 0, self.Nc, self.aw)
+        st.gate(0, 0, self.Nc, self.lw)
+        st.compact(0, wl.tau)
+        st.decode_attn(0, self.q, self.out)
+
+    def step_steady(self):
+        """the step between two gate triggers (token n0 + 1: no chunk leaves the window, the keep list stands)"""
+        st = self.st
+        st.set_len(0, self.n0)
+        st.append(0, self.k3, self.v3)
+        st.decode_attn(0, self.q, self.out)
+
+
+def time_loop(fn, iters, repeats=1, sync=None):
+    """`repeats` loops of `iters` calls, each loop bracketed by CUDA events on the current stream (and by `sync`
+    = barrier + device synchronise when given); list of milliseconds per loop"""
+    import torch
+    sync = sync or torch.cuda.synchronize
+    out = []
+    for _ in range(repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sync()
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        sync()
+        out.append(e0.elapsed_time(e1))
+    return out
+
+
+def iters_for(fn, target_s=0.15, lo=10, hi=400):
+    """how many calls of fn fill about target_s (pilot of 5 calls after 3 warm-up calls)"""
+    for _ in range(3):
+        fn()
+    ms = time_loop(fn, 5)[0] / 5
+    return int(min(hi, max(lo, target_s * 1e3 / max(ms, 1e-3))))
+
+
+class Flusher:
+    """writes a buffer larger than L2 (126 MB) so that the next launch starts cold"""
+
+    def __init__(self):
+        import torch
+        self.buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def __call__(self):
+        self.buf.fill_(1)
+
+
+def copy_us(total_bytes, flush):
+    """a plain device copy that moves total_bytes (read + write), timed like the kernels: L2 flushed, events"""
+    import torch
+    src = torch.empty(max(1, int(total_bytes) // 2), dtype=torch.uint8, device="cuda")
+    dst = torch.empty_like(src)
+    ts = []
+    for i in range(8):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dst.copy_(src)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            ts.append(e0.elapsed_time(e1) * 1e3)
+    return float(np.median(ts))
+
+
+def kernel_times(rig, flush, n_in_step=20, n_cold=8):
+    """microseconds per kernel from the library's own event pairs: inside the from-scratch step (caches as the
+    step leaves them) and with L2 flushed before the call that launches the kernel"""
+    st, b = rig.st, rig.b
+    st.profile(True)
+    in_step = {k: [] for k in b.KERNEL_IDS}
+    for _ in range(n_in_step):
+        rig.step_full()
+        for k, v in st.profile_read().items():
+            if v is not None and k not in ("attn_dense", "attn_block"):
+                in_step[k].append(v)
+    cold = {k: [] for k in ("chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense")}
+    for _ in range(n_cold):
+        # each call after a flush; the kernels a call launches back to back share what the first one left in L2
+        flush(); st.summarize_chunks(0, 0, rig.Nc, rig.aw); r = st.profile_read()
+        cold["chunk_mean"].append(r["chunk_mean"])
+        if r["chunk_mlp"] is not None:
+            cold["chunk_mlp"].append(r["chunk_mlp"])
+        flush(); st.gate(0, 0, rig.Nc, rig.lw); r = st.profile_read()
+        cold["gate_proj"].append(r["gate_proj"]); cold["gate_rnn"].append(r["gate_rnn"])
+        flush(); st.compact(0, rig.wl.tau); cold["compact"].append(st.profile_read()["compact"])
+        flush(); st.decode_attn(0, rig.q, rig.out); cold["attn"].append(st.profile_read()["attn"])
+        flush(); st.decode_attn_dense(0, rig.q, rig.out); cold["attn_dense"].append(st.profile_read()["attn_dense"])
+    st.profile(False)
+    rig.step_full()
+    med = lambda v: float(np.median(v))
+    return ({k: med(v) for k, v in in_step.items() if v}, {k: med(v) for k, v in cold.items() if v})
+
+
+def measure_config(rig, peaks, peak_kind, flush, headline=False):
+    """Everything the report gives per configuration: the from-scratch step, the steady step, every kernel in-step
+    and L2-flushed with its algorithmic bytes / flops and fractions of the measured peaks, gated vs dense."""
+    import torch
+    wl, st = rig.wl, rig.st
+    hbm = peaks["hbm_gbs"]
+    tensor_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    res = {"workload": wl.name, "S": wl.S, "n": wl.n, "C": wl.C, "W": wl.W, "attend": rig.attend, "stale_chunks": rig.Nc,
+           "kept_chunks_mean": rig.keep_mean, "n_eff": rig.n_eff, "memory_ratio_n_over_n_eff": wl.n / rig.n_eff}
+    if not headline:
+        it = iters_for(rig.step_full)
+        ms = float(np.median(time_loop(rig.step_full, it, 3))) / it
+        res["full_step"] = {"ms": ms, "steps_per_s": 1e3 / ms, "iters": it, "repeats": 3}
+        it = iters_for(rig.step_steady)
+        ms = float(np.median(time_loop(rig.step_steady, it, 3))) / it
+        res["steady_step"] = {"ms": ms, "steps_per_s": 1e3 / ms, "iters": it, "repeats": 3}
+        rig.step_full()
+    us_in, us_cold = kernel_times(rig, flush)
+    by = algorithmic_bytes(wl, rig.Nc, rig.keep_mean, rig.R, rig.attend)
+    by_kernel = {"append": wl.S * 4 * 256, "chunk_mean": by["chunk_mean"], "chunk_mlp": by["chunk_mlp"],
+                 "gate_proj": by["gate_proj"], "gate_rnn": by["gate_rnn"], "compact": by["compact"],
+                 "attn": by["attn_gated"], "attn_dense": by["attn_dense"]}
+    fl = algorithmic_flops(wl, rig.Nc)
+    kern = {}
+    for k in sorted(set(us_in) | set(us_cold)):
+        e = {"bytes": by_kernel[k]}
+        if k in us_in:
+            e["us"] = us_in[k]
+            e["GB/s"] = by_kernel[k] / us_in[k] / 1e3
+            e["frac_of_hbm_peak"] = e["GB/s"] / hbm
+        if k in us_cold:
+            e["us_l2_flushed"] = us_cold[k]
+            e["GB/s_l2_flushed"] = by_kernel[k] / us_cold[k] / 1e3
+            e["frac_of_hbm_peak_l2_flushed"] = e["GB/s_l2_flushed"] / hbm
+        if k in fl:
+            t = us_in.get(k, us_cold.get(k))
+            e["flops"] = fl[k]
+            e["TFLOP/s"] = fl[k] / t / 1e6
+            e["frac_of_bf16_peak"] = e["TFLOP/s"] / tensor_peak
+        kern[k] = e
+    res["kernels"] = kern
+    g_us, d_us = us_cold["attn"], us_cold["attn_dense"]
+    cg, cd = copy_us(by["attn_gated"], flush), copy_us(by["attn_dense"], flush)
+    res["attention_vs_dense"] = {
+        "note": "attention kernels alone, L2 flushed before every launch",
+        "gated_us": g_us, "dense_us": d_us, "speedup": d_us / g_us,
+        "kv_bytes_gated": by["attn_gated"], "kv_bytes_dense": by["attn_dense"],
+        "gated_GB/s": by["attn_gated"] / g_us / 1e3, "dense_GB/s": by["attn_dense"] / d_us / 1e3,
+        "gated_frac_of_measured_peak": by["attn_gated"] / g_us / 1e3 / hbm,
+        "dense_frac_of_measured_peak": by["attn_dense"] / d_us / 1e3 / hbm,
+        "gated_frac_of_nominal_8TBps": by["attn_gated"] / g_us / 1e3 / 8000.0,
+        "dense_frac_of_nominal_8TBps": by["attn_dense"] / d_us / 1e3 / 8000.0,
+        "size_matched_copy": {"note": "a plain torch device copy moving the same number of bytes (read + write), same timing "
+                                      "method: what this transfer size allows on this GPU",
+                              "gated_bytes_copy_us": cg, "dense_bytes_copy_us": cd,
+                              "gated_time_over_copy": g_us / cg, "dense_time_over_copy": d_us / cd},
+        "peak_kind": f"of {peak_kind}"}
+    assert st.poll_status() == 0
+    return res
+
+
+def trigger_leg(wl, attend, seed, steady_ms, n_triggers=24):
+    """The aggregation-and-gating step of Sec. 3.3 as it happens while decoding: C more tokens have arrived, ONE chunk
+    per sequence leaves the window; it is summarised, takes one LSTM step with the carried (h, c), and the keep list
+    is rebuilt.  Timed per trigger (events around the three calls), n_triggers triggers in a row on a growing cache."""
+    import torch
+    rig = Rig(wl, attend, seed, extra_tokens=(n_triggers + 1) * wl.C)
+    st = rig.st
+    kC = torch.randn((wl.S, wl.C, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    vC = torch.randn((wl.S, wl.C, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    ts = []
+    for i in range(n_triggers):
+        ready = st.append(0, kC, vC)
+        assert ready == 1
+        t = rig.Nc + i
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        st.summarize_chunks(0, t, t + 1, rig.aw)
+        st.gate(0, t, t + 1, rig.lw)
+        st.compact(0, wl.tau)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 4:
+            ts.append(e0.elapsed_time(e1))
+    assert st.poll_status() == 0
+    trig = float(np.median(ts))
+    return {"what": "one chunk per sequence leaves the window: kvE_summarize_chunks(t, t+1) + kvE_gate(t, t+1) with carried "
+                    "state + kvE_compact, per layer; the amortised step spreads it over the C tokens between two triggers",
+            "trigger_ms": trig, "triggers_timed": len(ts), "steady_ms": steady_ms, "C": wl.C,
+            "amortised_ms_per_token": (wl.C * steady_ms + trig) / wl.C,
+            "amortised_steps_per_s": 1e3 * wl.C / (wl.C * steady_ms + trig),
+            "trigger_share_of_amortised_step": trig / (wl.C * steady_ms + trig)}
+
+
+SWEEP_GEOMETRIES = [  # (B, n, C): every corner of the grid, then a diagonal through its middle
+    (1, 2048, 32), (1, 2048, 256), (1, 32768, 32), (1, 32768, 256),
+    (64, 2048, 32), (64, 2048, 256), (64, 32768, 32), (64, 32768, 256),
+    (2, 4096, 64), (4, 8192, 128), (8, 16384, 64), (16, 8192, 128), (32, 4096, 64), (16, 32768, 128)]
+SWEEP_KEEPS = {"corner": (0.25, 1.0), "diagonal": (0.5, 0.75)}
+
+
+def sweep_leg(peaks, peak_kind, flush, seed, mem_cap=120e9):
+    """cfg5: a bounded walk over workloads.sweep_points() - all 16 corners of (batch 1/64, context 2k/32k, chunk
+    32/256, keep 0.25/1.0) plus a diagonal - 32 heads, W = 512, single layer.  Per point: dense attention, gated
+    attention with kept chunks as summary rows and as raw rows, each launch alone with L2 flushed: microseconds,
+    steps/s, KV bytes, GB/s, fraction of the measured HBM peak.  The keep ratio is set by thresholding the scores at
+    the matching quantile."""
+    import torch
+    from paper_2509_21354_b200 import binding as b
+    hbm = peaks["hbm_gbs"]
+    grid = {(w.B, w.n, w.C, k) for w, k in wlm.sweep_points()}
+    points, skipped = [], []
+    for gi, (B, n, Cs) in enumerate(SWEEP_GEOMETRIES):
+        keeps = SWEEP_KEEPS["corner" if gi < 8 else "diagonal"]
+        wl = wlm.Workload(f"sweep_b{B}_n{n}_c{Cs}", B=B, H=32, n=n, C=Cs, W=512, d_g=256, agg="mean", key_offset_std=0.5)
+        assert all((B, n, Cs, k) in grid for k in keeps)
+        need = wl.S * (n + Cs) * 512 * 1.35 + wl.S * wl.max_chunks * 4096 * 1.1
+        if need > mem_cap:
+            skipped.append({"B": B, "n": n, "C": Cs, "why": f"needs {need / 1e9:.0f} GB on the device"})
+            continue
+        st = b.Store(B=B, H=32, C_=Cs, W=512, max_tokens=n + Cs, d_g=256, agg="mean", attend="summary", page_perm="random",
+                     seed=seed + gi)
+        gen = fill_cache(st, wl.small(n=n + 1), seed + gi)               # fill_cache leaves the last token out
+        lw = b.LstmWeights(wlm.gen_lstm_weights(wl))
+        Nc = wl.n_stale_chunks()
+        st.summarize_chunks(0, 0, Nc, None)
+        st.gate(0, 0, Nc, lw)
+        torch.cuda.synchronize()
+        sc = st.scores[0, :, :Nc].flatten()
+        q = torch.randn((wl.S, 128), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        out = torch.empty_like(q)
+        st.profile(True)
+
+        def timed(fn, key):
+            ts = []
+            for i in range(7):
+                flush()
+                fn(0, q, out)
+                ts.append(st.profile_read()[key])
+            return float(np.median(ts[2:]))
+
+        d_us = timed(st.decode_attn_dense, "attn_dense")
+        d_by = wl.S * (2 * n * 256 + 512)
+        for keep in keeps:
+            tau = 0.0 if keep >= 1.0 else float(torch.quantile(sc[:1 << 22].float(), 1.0 - keep).item())
+            st.compact(0, tau)
+            torch.cuda.synchronize()
+            M = st.keep_cnt[0].float().mean().item()
+            pt = {"B": B, "n": n, "C": Cs, "keep": keep, "kept_chunks_mean": M, "stale_chunks": Nc,
+                  "dense": {"us": d_us, "steps_per_s": 1e6 / d_us, "kv_bytes": d_by, "GB/s": d_by / d_us / 1e3,
+                            "frac_of_hbm_peak": d_by / d_us / 1e3 / hbm}}
+            for attend, per in (("summary", 1), ("raw", Cs)):
+                st.set_attend(attend)
+                us = timed(st.decode_attn, "attn")
+                by = wl.S * (2 * (n - Nc * Cs + M * per) * 256 + 512)
+                pt["gated_" + attend] = {"us": us, "steps_per_s": 1e6 / us, "kv_bytes": int(by), "GB/s": by / us / 1e3,
+                                         "frac_of_hbm_peak": by / us / 1e3 / hbm, "speedup_vs_dense": d_us / us}
+            points.append(pt)
+        assert st.poll_status() == 0
+        st.close()
+        del st, q, out, sc
+        torch.cuda.empty_cache()
+    big = [p for p in points if p["gated_summary"]["kv_bytes"] >= 256e6]
+    return {"what": "stress sweep (cfg5), bounded: 16 corner points + a diagonal; attention launches alone, L2 flushed; "
+                    f"fractions of the {peak_kind} HBM copy figure",
+            "n_points": len(points), "points": points, "skipped": skipped,
+            "gated_summary_min_frac_at_256MB_or_more": min((p["gated_summary"]["frac_of_hbm_peak"] for p in big), default=None)}
+
+
+def action_step_leg(seed):
+    """cfg3 in its stated form: one control step = 7 action tokens appended autoregressively, each through all 32
+    layers (append at the device-held length + gated attention per layer and token), the 32-layer tick captured in a
+    CUDA graph and replayed 7 times."""
+    wl = wlm.CFG3
+    r = graph_tick_leg(wl, wl.n_layers, seed, replays=wl.n_append)
+    ms = r["graph"]["ms_per_tick"] * wl.n_append
+    return {"what": f"{wl.n_append} action tokens x {r['n_layers']} layers, graph-replayed (B={wl.B}, H={wl.H}, n={wl.n})",
+            "ms_per_action_step": ms, "action_steps_per_s": 1e3 / ms, "attention_calls_per_action_step": wl.n_append * r["n_layers"],
+            "us_per_layer_and_token": r["graph"]["us_per_layer"], "eager_ms_per_action_step": r["eager"]["ms_per_tick"] * wl.n_append,
+            "kv_bytes_per_token": r["kv_bytes_per_tick"], "GB/s": r["GB/s_graph"], "graph_first_tick_equals_eager": r["graph_first_tick_equals_eager"]}
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
-    from paper_2509_21354_b200 import binding as b
 
     torch.cuda.set_device(local_rank)
     wl = wlm.CONFIGS[args.workload].small(n_layers=1)
     lo, _ = shard_batch(wl.B, rank, world)
     seed = 1000 + lo
-    st = b.Store(B=wl.B, H=wl.H, C_=wl.C, W=wl.W, max_tokens=wl.n + wl.C, d_g=wl.d_g, agg=wl.agg, d_sum=wl.d_sum,
-                 attend=args.attend, page_perm="random", seed=seed)
-    g = fill_cache(st, wl, seed)
-    mlp = wlm.gen_mlp_weights(wl)
-    lstm = wlm.gen_lstm_weights(wl)
-    aw = b.AggWeights(mlp) if mlp is not None else None
-    lw = b.LstmWeights(lstm)
-    S = wl.S
-    rnd = lambda: torch.randn((S, 128), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16).contiguous()
-    k_new, v_new, q = rnd(), rnd(), rnd()
-    k3, v3 = k_new.view(S, 1, 128), v_new.view(S, 1, 128)
-    out = torch.empty_like(q)
-    n0 = wl.n
-    Nc = wl.n_stale_chunks(n0)
-
-    def step():
-        st.set_len(0, n0 - 1)
-        st.append(0, k3, v3)
-        st.summarize_chunks(0, 0, Nc, aw)
-        st.gate(0, 0, Nc, lw)
-        st.compact(0, wl.tau)
-        st.decode_attn(0, q, out)
-
-    # head bias that retains about half of the chunks (deterministic given the seed)
-    step()
-    torch.cuda.synchronize()
-    sc = st.scores[0, :, :Nc].double().clamp(1e-9, 1 - 1e-9)
-    lw.set_b_s(float(-torch.median(torch.log(sc / (1 - sc))).item()) + lstm["b_s"])
-    step()
-    torch.cuda.synchronize()
-    assert st.poll_status() == 0
-    keep_mean = st.keep_cnt[0].float().mean().item()
-    R = n0 - Nc * wl.C
+    rig = Rig(wl, args.attend, seed)
+    st, S = rig.st, wl.S
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    # ---- the headline: K from-scratch steps, repeated so that the timed work lasts long enough -------------
     for _ in range(args.warmup):
-        step()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+        rig.step_full()
+    pilot = time_loop(rig.step_full, 3, 1, barrier)[0] / 3                       # ms per step
+    repeats = int(min(50, max(1, math.ceil(args.min_timed_s * 1e3 / max(pilot * args.steps, 1e-6)))))
+    repeats = int(max_over_ranks([repeats], world)[0])
     with ClockSampler(local_rank) as clk:
-        ev0.record()
-        for _ in range(args.steps):
-            step()
-        ev1.record()
-        barrier()
-    ms_total = ev0.elapsed_time(ev1)
+        loops = time_loop(rig.step_full, args.steps, repeats, barrier)
     assert st.poll_status() == 0
+    loops = [max_over_ranks([t], world)[0] for t in loops] if world > 1 else loops
+    ms_total = float(np.median(loops))
 
     # ---- steady-state decode step (between two gate triggers): append one token, gated attention ----
-    # (token n0 + 1: no chunk leaves the window, so the keep list of the last full step stands)
-    def step_steady():
-        st.set_len(0, n0)
-        st.append(0, k3, v3)
-        st.decode_attn(0, q, out)
-
     for _ in range(3):
-        step_steady()
-    barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        step_steady()
-    ev1.record()
-    barrier()
-    ms_steady = max_over_ranks([ev0.elapsed_time(ev1)], world)[0]
+        rig.step_steady()
+    ms_steady = float(np.median(max_over_ranks(time_loop(rig.step_steady, args.steps, min(repeats, 5), barrier), world)))
     assert st.poll_status() == 0
-    step()                      # back to the state and output of a full step
+    rig.step_full()                      # back to the state and output of a full step
     torch.cuda.synchronize()
     steady = {"what": "append + gated attention only (summaries, gate and keep list reused: the state between two triggers)",
               "value": world * args.steps / (ms_steady * 1e-3), "unit": UNIT, "ms_per_step": ms_steady / args.steps}
 
     # ---- end to end: the same step through kvE_decode_step_host, host buffers, copies timed ----
-    hk, hv, hq = (t.cpu().pin_memory() for t in (k_new, v_new, q))
+    hk, hv, hq = (t.cpu().pin_memory() for t in (rig.k_new, rig.v_new, rig.q))
     hout = torch.zeros((S, 128), dtype=torch.bfloat16).pin_memory()
 
     # every step: H2D of its inputs and D2H of its result inside the timed region; steps are enqueued
     # back to back (kvE_decode_step_host_async) and the stream is waited for once, at the end
     def step_e2e():
-        st.set_len(0, n0 - 1)
-        st.decode_step_host(0, hk, hv, hq, hout, aw, lw, wl.tau, from_scratch=True, wait=False)
+        st.set_len(0, rig.n0 - 1)
+        st.decode_step_host(0, hk, hv, hq, hout, rig.aw, rig.lw, wl.tau, from_scratch=True, wait=False)
 
-    for _ in range(min(args.warmup, 3)):
+    for _ in range(3):
         step_e2e()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        step_e2e()
-    barrier()
-    e2e_s = time.perf_counter() - t0
-    same = bool(torch.equal(hout.cuda(), out))
-
-    ms_total, e2e_s = max_over_ranks([ms_total, e2e_s], world)
+    e2e_runs = []
+    for _ in range(min(repeats, 5)):
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            step_e2e()
+        barrier()
+        e2e_runs.append(time.perf_counter() - t0)
+    e2e_s = float(np.median(max_over_ranks(e2e_runs, world)))
+    same = bool(torch.equal(hout.cuda(), rig.out))
     if rank != 0:
         return None
 
-    # ---- per-kernel timing (rank 0): the library brackets every launch with CUDA events on its stream ----
+    # ---- rank 0: per-kernel figures, rooflines, and (single GPU only) the other configurations and legs ----
     peaks, peak_kind = load_peaks()
     hbm = peaks["hbm_gbs"]
-    st.profile(True)
-    in_step = {k: [] for k in b.KERNEL_IDS}
-    for _ in range(min(args.steps, 30)):          # same step as the timed region
-        step()
-        for k, v in st.profile_read().items():
-            if v is not None and k != "attn_dense":
-                in_step[k].append(v)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    cold = {"attn": [], "attn_dense": []}
-    for _ in range(10):                            # attention alone, L2 flushed before every launch
-        for name, fn in (("attn", st.decode_attn), ("attn_dense", st.decode_attn_dense)):
-            flush.fill_(1)
-            fn(0, q, out)
-            cold[name].append(st.profile_read()[name])
-    st.profile(False)
-    us = {k: float(np.mean(v)) for k, v in in_step.items() if v}
-    us["attn_dense"] = float(np.mean(cold["attn_dense"]))
-    us_attn_cold = float(np.mean(cold["attn"]))
-    by = algorithmic_bytes(wl, Nc, keep_mean, R, args.attend)
-
-    def copy_us(total_bytes):
-        """a plain device copy that moves total_bytes (read + write), timed like the kernels: L2 flushed, events"""
-        src = torch.empty(max(1, int(total_bytes) // 2), dtype=torch.uint8, device="cuda")
-        dst = torch.empty_like(src)
-        ts = []
-        for i in range(8):
-            flush.fill_(1)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            dst.copy_(src)
-            e1.record()
-            torch.cuda.synchronize()
-            if i >= 2:
-                ts.append(e0.elapsed_time(e1) * 1e3)
-        return float(np.mean(ts))
-
-    copy_gated_us, copy_dense_us = copy_us(by["attn_gated"]), copy_us(by["attn_dense"])
-    by_kernel = {"append": S * 4 * 256, "chunk_mean": by["chunk_mean"], "chunk_mlp": by["chunk_mlp"],
-                 "gate_proj": by["gate_proj"], "gate_rnn": by["gate_rnn"], "compact": by["compact"],
-                 "attn": by["attn_gated"], "attn_dense": by["attn_dense"]}
-    fl = algorithmic_flops(wl, Nc)
     tensor_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])     # kernels timed inside a long step
-    kern = {}
-    for k, t in us.items():
-        kern[k] = {"us": t, "bytes": by_kernel[k], "GB/s": by_kernel[k] / (t * 1e-6) / 1e9}
-        kern[k]["frac_of_hbm_peak"] = kern[k]["GB/s"] / hbm
-        if k in fl:
-            kern[k]["flops"] = fl[k]
-            kern[k]["TFLOP/s"] = fl[k] / (t * 1e-6) / 1e12
-            kern[k]["frac_of_bf16_peak"] = kern[k]["TFLOP/s"] / tensor_peak
-    kern["attn"]["us_l2_flushed"] = us_attn_cold
-    kern["attn"]["GB/s_l2_flushed"] = by_kernel["attn"] / (us_attn_cold * 1e-6) / 1e9
-    dominant = max((k for k in kern if k != "attn_dense"), key=lambda k: kern[k]["us"])
+    flush = Flusher()
+    head = measure_config(rig, peaks, peak_kind, flush, headline=True)
+    kern = head["kernels"]
+    in_step = {k: v for k, v in kern.items() if "us" in v and k != "attn_dense"}
+    dominant = max(in_step, key=lambda k: in_step[k]["us"])
     traffic = None
     tp = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.txt")
     if os.path.exists(tp) and args.attend == "summary":
         with open(tp) as f:
-            tab = dict(line.split() for line in f if line.strip() and not line.startswith("#"))
+            tab = dict(line.split()[:2] for line in f if line.strip() and not line.startswith("#"))
         traffic = int(tab[dominant]) if dominant in tab else None
-    if dominant in fl:
+    if "flops" in kern[dominant]:
         roofline = {"kernel": dominant, "bound": "tensor", "achieved": kern[dominant]["TFLOP/s"], "peak": tensor_peak,
                     "unit": "TFLOP/s", "frac": kern[dominant]["frac_of_bf16_peak"], "traffic": traffic,
-                    "peak_kind": f"of {peak_kind} (sustained bf16)", "algorithmic_flops": fl[dominant],
+                    "peak_kind": f"of {peak_kind} (sustained bf16)", "algorithmic_flops": kern[dominant]["flops"],
                     "us_per_launch": kern[dominant]["us"]}
         if dominant == "gate_rnn":
-            roofline["note"] = (f"{Nc} strictly sequential LSTM steps per sequence: bounded by per-step latency "
-                                f"({kern[dominant]['us'] / Nc:.2f} us per step), not by tensor throughput")
+            roofline["note"] = (f"{rig.Nc} strictly sequential LSTM steps per sequence: bounded by per-step latency "
+                                f"({kern[dominant]['us'] / rig.Nc:.2f} us per step), not by tensor throughput")
     else:
         roofline = {"kernel": dominant, "bound": "hbm", "achieved": kern[dominant]["GB/s"], "peak": hbm, "unit": "GB/s",
                     "frac": kern[dominant]["GB/s"] / hbm, "traffic": traffic, "peak_kind": f"of {peak_kind}",
                     "algorithmic_bytes": kern[dominant]["bytes"], "us_per_launch": kern[dominant]["us"]}
-    hbm_kernel = max((k for k in ("chunk_mean", "attn")), key=lambda k: kern[k]["us"])
+    hbm_kernel = max((k for k in ("chunk_mean", "attn") if k in in_step), key=lambda k: in_step[k]["us"])
     roofline_hbm = {"kernel": hbm_kernel, "bound": "hbm", "achieved": kern[hbm_kernel]["GB/s"], "peak": hbm, "unit": "GB/s",
                     "frac": kern[hbm_kernel]["GB/s"] / hbm, "algorithmic_bytes": kern[hbm_kernel]["bytes"],
                     "us_per_launch": kern[hbm_kernel]["us"], "peak_kind": f"of {peak_kind}"}
-    us["attn_gated"] = us_attn_cold
-
+    avd = head["attention_vs_dense"]
+    kv_stale_gb = S * rig.Nc * wl.C * 512 / 1e9
     ms_step = ms_total / args.steps
     res = {
         "metric": METRIC, "value": world * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -502,62 +742,100 @@ def run_ours(args, rank, world, local_rank):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "d": 128, "n": wl.n, "C": wl.C, "W": wl.W,
                    "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend, "n_layers_timed": 1,
-                   "stale_chunks": Nc, "kept_chunks_mean": keep_mean, "n_eff": R + keep_mean * (wl.C if args.attend == "raw" else 1),
-                   "memory_ratio_n_over_n_eff": n0 / (R + keep_mean * (wl.C if args.attend == "raw" else 1)),
-                   "l2": "inputs larger than L2 (each step streams 0.45 GB of stale KV + 0.06 GB window); per-kernel timings flush L2 before every launch"},
+                   "stale_chunks": rig.Nc, "kept_chunks_mean": rig.keep_mean, "n_eff": rig.n_eff,
+                   "memory_ratio_n_over_n_eff": wl.n / rig.n_eff,
+                   "l2": f"inputs larger than L2 (each step streams {kv_stale_gb:.2f} GB of stale KV + "
+                         f"{S * rig.R * 512 / 1e9:.2f} GB of window); kernels are also timed alone with L2 flushed before the launch"},
+        "timing": {"repeats": repeats, "statistic": "median over repeats of one K-step loop (events, max over ranks)",
+                   "loops_ms": loops, "timed_s_total": sum(loops) / 1e3},
         "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * S * 256,
                 "d2h_bytes_per_step": S * 256, "matches_device_path": same},
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "gpu_launches": KERNELS_PER_STEP * args.steps * repeats,
         "clocks": clk.summary(),
         "roofline": roofline,
         "roofline_largest_hbm_kernel": roofline_hbm,
+        "gated_attention": {"us_l2_flushed": avd["gated_us"], "GB/s": avd["gated_GB/s"], "frac_of_hbm_peak": avd["gated_frac_of_measured_peak"],
+                            "target": 0.70, "dense_us_l2_flushed": avd["dense_us"], "dense_frac_of_hbm_peak": avd["dense_frac_of_measured_peak"],
+                            "kv_bytes_gated": avd["kv_bytes_gated"], "kv_bytes_dense": avd["kv_bytes_dense"], "speedup_vs_dense": avd["speedup"]},
         "steady_state": steady,
-        "query_block_attention": query_block_leg(wl, hbm, tensor_peak, peak_kind, seed + 17),
-        "decode_tick_graph": graph_tick_leg(wl, args.tick_layers, seed + 31) if args.tick_layers > 0 else None,
-        "paper_cost_model": paper_cost_model(wl, keep_mean),
+        "paper_cost_model": paper_cost_model(wl, rig.keep_mean),
         "kernels": kern,
-        "attention_vs_dense": {"note": "attention kernels alone, L2 flushed before every launch",
-                               "gated_us": us["attn_gated"], "dense_us": us["attn_dense"],
-                               "speedup": us["attn_dense"] / us["attn_gated"],
-                               "kv_bytes_gated": by["attn_gated"], "kv_bytes_dense": by["attn_dense"],
-                               "gated_GB/s": kern["attn"]["GB/s_l2_flushed"], "dense_GB/s": kern["attn_dense"]["GB/s"],
-                               "gated_frac_of_measured_peak": kern["attn"]["GB/s_l2_flushed"] / hbm,
-                               "dense_frac_of_measured_peak": kern["attn_dense"]["GB/s"] / hbm,
-                               "size_matched_copy": {
-                                   "note": "a plain torch device copy moving the same number of bytes (read + write), "
-                                           "same timing method: what this transfer size allows on this GPU",
-                                   "gated_bytes_copy_us": copy_gated_us, "dense_bytes_copy_us": copy_dense_us,
-                                   "gated_frac_of_copy": copy_gated_us / us["attn_gated"],
-                                   "dense_frac_of_copy": copy_dense_us / us["attn_dense"]},
-                               "gated_frac_of_nominal_8TBps": kern["attn"]["GB/s_l2_flushed"] / 8000.0,
-                               "dense_frac_of_nominal_8TBps": kern["attn_dense"]["GB/s"] / 8000.0},
+        "attention_vs_dense": avd,
     }
-    if not args.no_cpu_baseline and world == 1:
-        res["cpu_baseline"] = cpu_baseline(wl, args.attend, budget_s=15.0)
+    legs = set(args.legs.split(",")) if args.legs else set()
+    if world > 1:
+        legs = set()                     # the other legs are single-GPU properties: reported by the N = 1 run
+    short = args.workload
+    per = {short: {k: head[k] for k in head if k != "kernels"}}
+    per[short]["full_step"] = {"ms": ms_step, "steps_per_s": 1e3 / ms_step}
+    per[short]["steady_step"] = {"ms": steady["ms_per_step"], "steps_per_s": 1e3 / steady["ms_per_step"]}
+    per[short]["kernels_us"] = {k: {a: v[a] for a in ("us", "us_l2_flushed", "frac_of_hbm_peak_l2_flushed") if a in v} for k, v in kern.items()}
+    if "trigger" in legs:
+        res["trigger"] = trigger_leg(wl, args.attend, seed + 5, steady["ms_per_step"])
+    rig.st.close()
+    del rig, st
+    torch.cuda.empty_cache()
+    if "per_config" in legs:
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+            if name == short:
+                continue
+            w2 = wlm.CONFIGS[name].small(n_layers=1)
+            r2 = Rig(w2, args.attend, seed + 100)
+            m = measure_config(r2, peaks, peak_kind, flush)
+            m["kernels_us"] = {k: {a: v[a] for a in ("us", "us_l2_flushed", "frac_of_hbm_peak_l2_flushed") if a in v}
+                               for k, v in m.pop("kernels").items()}
+            per[name] = m
+            r2.st.close()
+            del r2
+            torch.cuda.empty_cache()
+        per["cfg3"]["action_step_32_layers"] = action_step_leg(seed + 41)
+    res["per_config"] = per
+    if "sweep" in legs:
+        res["sweep"] = sweep_leg(peaks, peak_kind, flush, seed + 200)
+    if "query_block" in legs:
+        res["query_block_attention"] = query_block_leg(wl, hbm, tensor_peak, peak_kind, seed + 17)
+    if "tick_graph" in legs and args.tick_layers > 0:
+        res["decode_tick_graph"] = graph_tick_leg(wl, args.tick_layers, seed + 31)
+    if "cpu" in legs:
+        res["cpu_baseline"] = cpu_baseline(wl, args.attend, budget_s=12.0)
+        res["cpu_oracle_per_config"] = oracle_per_config(args.attend)
     return res
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle arm
-def oracle_step_time(wl, attend, n_seq, repeat=1):
-    """Seconds the oracle (f64 build, OpenMP over sequences) needs for the whole path on n_seq sequences."""
+def oracle_times(wl, attend, n_seq, threads=None):
+    """Seconds the oracle (f64 build, OpenMP over sequences, `threads` threads) needs on n_seq sequences of the
+    workload: T1 = the whole path (summaries, gate, keep list, gated attention), T2 = its gated attention alone,
+    T0 = full-cache attention (Eq. 1 over all n tokens)."""
     from oracle import kvo, margin
-    o = kvo.Oracle("f64")
-    seqs = list(range(n_seq))
-    K, V = wlm.gen_kv(wl, 0, seqs=seqs)
-    mlp, lstm = wlm.gen_mlp_weights(wl), wlm.gen_lstm_weights(wl)
-    q = wlm.gen_q(wl)[seqs]
-    Nc = wl.n_stale_chunks()
-    agg = margin.AGG_CODE[wl.agg]
-    att = kvo.ATTEND_RAW if attend == "raw" else kvo.ATTEND_SUMMARY
-    best = float("inf")
-    for _ in range(repeat):
+    cores = os.cpu_count() or 1
+    kvo.set_threads(threads or cores)
+    try:
+        o = kvo.Oracle("f64")
+        seqs = list(range(n_seq))
+        K, V = wlm.gen_kv(wl, 0, seqs=seqs)
+        mlp, lstm = wlm.gen_mlp_weights(wl), wlm.gen_lstm_weights(wl)
+        q = wlm.gen_q(wl)[seqs]
+        Nc = wl.n_stale_chunks()
+        agg = margin.AGG_CODE[wl.agg]
+        att = kvo.ATTEND_RAW if attend == "raw" else kvo.ATTEND_SUMMARY
         t0 = time.perf_counter()
         sm = o.summarize(K, V, wl.C, 0, Nc, agg, mlp, stride=max(wl.max_chunks, 1))
         sc, _, _ = o.gate(sm["ksum_b16"], sm["vsum_b16"], 0, Nc, lstm)
         idx, cnt = o.compact(sc, Nc, wl.tau)
+        t1 = time.perf_counter()
         o.attn(q, K, V, wl.C, Nc, idx, cnt, sm["ksum_b16"], sm["vsum_b16"], att, SCALE)
-        best = min(best, time.perf_counter() - t0)
-    return best
+        t2 = time.perf_counter()
+        o.attn_dense(q, K, V, SCALE)
+        t3 = time.perf_counter()
+    finally:
+        kvo.set_threads(cores)
+    return {"T1": t2 - t0, "T2": t2 - t1, "T0": t3 - t2}
+
+
+def oracle_step_time(wl, attend, n_seq, repeat=1):
+    """Seconds the oracle needs for the whole path (T1) on n_seq sequences, all host cores."""
+    return min(oracle_times(wl, attend, n_seq)["T1"] for _ in range(repeat))
 
 
 def cpu_baseline(wl, attend, budget_s=15.0):
@@ -572,6 +850,24 @@ def cpu_baseline(wl, attend, budget_s=15.0):
     return {"value": 1.0 / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n_seq} of {wl.S} sequences of {wl.name} (whole path, f64 oracle, OpenMP over sequences), "
                       f"{t:.2f} s measured, scaled to the full step"}
+
+
+def oracle_per_config(attend):
+    """The oracle on every fixed configuration (one layer), single-threaded and with OpenMP on all host cores, on a
+    bounded sample of sequences scaled to the layer: ms per step for T0 (full-cache attention), T1 (whole path) and T2
+    (gated attention only)."""
+    cores = os.cpu_count() or 1
+    out = {"cores": cores, "note": "f64 oracle as it stands; sample of sequences scaled to one full layer; ms"}
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+        wl = wlm.CONFIGS[name].small(n_layers=1)
+        n_seq = min(wl.S, max(cores, 8))
+        scale = wl.S / n_seq * 1e3
+        one = oracle_times(wl, attend, n_seq, threads=1)
+        omp = oracle_times(wl, attend, n_seq, threads=cores)
+        out[name] = {"sample_sequences": n_seq, "of": wl.S,
+                     "single_thread_ms": {k: v * scale for k, v in one.items()},
+                     "openmp_ms": {k: v * scale for k, v in omp.items()}}
+    return out
 
 
 def run_reference(args, rank):
@@ -592,24 +888,35 @@ def run_reference(args, rank):
             "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "d": 128, "n": wl.n, "C": wl.C, "W": wl.W,
-                       "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend},
+                       "d_g": wl.d_g, "agg": wl.agg, "d_sum": wl.d_sum, "attend": args.attend, "n_layers_timed": 1},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0, "wall_s": wall}
 
 
+ALL_LEGS = "per_config,sweep,trigger,query_block,tick_graph,cpu"
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=sorted(wlm.CONFIGS))
+    ap.add_argument("--workload", default="cfg4", choices=sorted(wlm.CONFIGS),
+                    help="the configuration the headline step is timed on (default: the largest single-GPU one)")
     ap.add_argument("--attend", default="summary", choices=["summary", "raw"])
+    ap.add_argument("--legs", default=ALL_LEGS,
+                    help="comma-separated extra legs of the single-GPU report (per_config, sweep, trigger, query_block, "
+                         "tick_graph, cpu); empty string: the headline only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-timed-s", type=float, default=0.25,
+                    help="the K-step loop is repeated until at least this much device time has been timed")
     ap.add_argument("--tick-layers", type=int, default=32,
                     help="layers of the CUDA-graph decode-tick leg (0 = skip; reduced if the caches would not fit 40 GB)")
     args = ap.parse_args()
+    if args.no_cpu_baseline:
+        args.legs = ",".join(x for x in args.legs.split(",") if x != "cpu")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

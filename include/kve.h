@@ -17,6 +17,9 @@
  *     (a page id out of range, a wait that ran out) set *status_word to a kvE_status and the kernel
  *     skips the access; nothing traps and no wait is unbounded.
  *   - one stream at a time per handle; calls on one handle are not thread-safe.
+ *   - a handle belongs to the device that was current at kvE_create (where its buffers live); a call
+ *     made with another device current returns KVE_ERR_STATE.  Several handles on several devices
+ *     may live in one process.
  *   - "bf16" is the 16-bit brain float bit pattern; matrices are row-major; S = B * Hkv sequences,
  *     sequence index s = b * Hkv + h.  d (head dim) must be 128.
  */
@@ -133,9 +136,18 @@ int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_n
                     void* stream);
 
 /* Set the stored length of `layer` (all sequences) to n tokens, n <= max_tokens; the pages keep
- * their contents.  Chunks at or beyond the new stale range lose their summarised / gated /
- * compacted marks.  Used to load a prefilled cache and to roll a decode step back. */
+ * their contents.  Chunks at or beyond the new stale range lose their summarised mark; if the new
+ * stale range is shorter than the gated range, the carried LSTM state is past the cut, so the gated mark
+ * returns to 0 (gate again from chunk 0); if it is shorter than the range the keep list covers, the
+ * keep list is dropped (attention then reads every stored row, which is exact, until the next
+ * kvE_compact).  Used to load a prefilled cache and to roll a decode step back. */
 int kvE_set_len(kvE_store* st, int layer, int n, void* stream);
+
+/* Switch what a kept chunk contributes to attention (cfg.attend) for all later calls on this handle:
+ * its one summary row (KVE_ATTEND_SUMMARY, the method of Sec. 3.3) or its C raw rows (KVE_ATTEND_RAW).
+ * Host-side only; summaries, scores and keep lists do not depend on it.  Pages handed back with
+ * KVE_RECLAIM_GATED are gone for KVE_ATTEND_RAW (reading them flags KVE_ERR_CAPACITY). */
+int kvE_set_attend(kvE_store* st, int attend);
 
 /* Eq. 2: summaries of chunks [chunk_begin, chunk_end) of every sequence of `layer`;
  * chunk_end <= floor((n - W) / C).  w is NULL unless agg == KVE_AGG_MLP. */
@@ -196,7 +208,9 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
  *   The softmax numerators enter the tensor core as bf16: against exact weights an output moves by at
  *   most 2^-8 * sum_i p_i |v_i| / sum_i p_i (accumulation in fp32, one bf16 rounding of the result).
  *   q, out: DEVICE bf16 [B][n_query_tokens][Hq][d]; lse: DEVICE fp32 [B][n_query_tokens][Hq] or NULL.
- *   KVE_ERR_STATE if cfg.max_query_tokens == 0, KVE_ERR_CAPACITY if n_query_tokens exceeds it. */
+ *   KVE_ERR_STATE if cfg.max_query_tokens == 0, or if causal != 0 and the raw tail (all stored tokens when
+ *   dense != 0) holds fewer rows than n_query_tokens; KVE_ERR_CAPACITY if n_query_tokens exceeds
+ *   cfg.max_query_tokens. */
 int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, int causal,
                           void* out, float* lse, float scale, void* stream);
 

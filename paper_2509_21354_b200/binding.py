@@ -21,7 +21,7 @@ ATTEND = {"summary": 0, "raw": 1}
 STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_CAPACITY",
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
-EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_append", "kvE_append_next", "kvE_set_len",
+EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_set_attend", "kvE_append", "kvE_append_next", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense", "kvE_decode_attn_block",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read"]
@@ -77,6 +77,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_destroy.argtypes = [C.c_void_p]
     lib.kvE_append.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p]
     lib.kvE_set_len.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+    lib.kvE_set_attend.argtypes = [C.c_void_p, C.c_int]
     lib.kvE_append_next.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
     lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
     lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
@@ -241,6 +242,10 @@ class Store:
 
     def set_len(self, layer, n, stream=None):
         kvE_set_len(self, layer, n, stream)
+
+    def set_attend(self, attend: str):
+        """"summary" | "raw": what a kept chunk contributes to attention from now on"""
+        _check("kvE_set_attend", self.lib.kvE_set_attend(self.handle, ATTEND[attend]))
 
     def summarize_chunks(self, layer, chunk_begin, chunk_end, agg_weights=None, stream=None):
         kvE_summarize_chunks(self, layer, chunk_begin, chunk_end, agg_weights, stream)

@@ -24,6 +24,7 @@ struct LayerState {
 struct kvE_store {
   kvE_config cfg;
   kvE_buffers buf;
+  int device = -1;       // the device that was current at kvE_create: owner of every buffer; calls check it
   int S, max_chunks;
   // workspace carve-up (byte offsets)
   size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, ws_needed;
@@ -41,6 +42,18 @@ struct kvE_store {
   bool ev_made = false;
   bool ev_used[KVE_K_COUNT] = {};
 };
+
+// SM count of the current device, looked up once per device
+int kve::sm_count() {
+  static std::atomic<int> cached[MAX_DEVICES];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 148;
+  int n = cached[dev].load(std::memory_order_acquire);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  cached[dev].store(n, std::memory_order_release);
+  return n;
+}
 
 namespace {
 
@@ -72,7 +85,7 @@ struct Carve {
 };
 // most splits per sequence the block-of-queries attention uses: one CTA per SM, one wave
 int block_split_cap(long long S) {
-  long long c = 148 / S;
+  long long c = sm_count() / S;
   return (int)(c < 1 ? 1 : (c > MAX_SPLITS ? MAX_SPLITS : c));
 }
 Carve carve(const kvE_config& c) {
@@ -144,9 +157,15 @@ int stale_chunks(const kvE_config& c, int n) { return n > c.W ? (n - c.W) / c.C 
 
 bool bad_layer(const kvE_store* st, int layer) { return !st || layer < 0 || layer >= st->cfg.n_layers; }
 
+// every launch goes to the current device: it must be the one the handle's buffers live on
+bool wrong_device(const kvE_store* st) {
+  int dev = -1;
+  return cudaGetDevice(&dev) != cudaSuccess || dev != st->device;
+}
+
 // rows per split and grid width for `n_rows_upper` logical rows per sequence
 AttnPlan plan_attention(const kvE_store* st, long long n_rows_upper) {
-  const long long one_wave = 148LL * 2;            // two CTAs per SM: everything resident at once, fewest merges
+  const long long one_wave = sm_count() * 2LL;     // two CTAs per SM: everything resident at once, fewest merges
   long long splits = one_wave / st->S;
   const long long max_useful = (n_rows_upper + 2 * ATTN_TILE_ROWS - 1) / (2 * ATTN_TILE_ROWS);   // >= 128 rows per split
   if (splits > max_useful) splits = max_useful;
@@ -206,6 +225,10 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   if (!st) return KVE_ERR_ARG;
   st->cfg = *cfg;
   st->buf = *buf;
+  if (cudaGetDevice(&st->device) != cudaSuccess) {
+    delete st;
+    return KVE_ERR_CUDA;
+  }
   st->S = cfg->B * cfg->Hkv;
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
   st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
@@ -246,6 +269,7 @@ int kvE_destroy(kvE_store* st) {
 
 int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new, int* n_ready, void* stream) {
   if (bad_layer(st, layer) || !k_new || !v_new || n_new < 0) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   if (n_new > 0) {
@@ -261,6 +285,7 @@ int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, i
 
 int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new, int n_reserve, void* stream) {
   if (bad_layer(st, layer) || !k_new || !v_new || n_new <= 0 || n_reserve < 0) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   if ((long long)ls.n_tokens + n_new > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   Prof prof(st, KVE_K_APPEND, static_cast<cudaStream_t>(stream));
@@ -276,6 +301,7 @@ int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_n
 
 int kvE_set_len(kvE_store* st, int layer, int n, void* stream) {
   if (bad_layer(st, layer) || n < 0) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (n > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
   cudaError_t e = launch_set_len(view(st, layer), n, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
@@ -285,13 +311,25 @@ int kvE_set_len(kvE_store* st, int layer, int n, void* stream) {
   const int nc = stale_chunks(st->cfg, n);
   if (ls.n_summarised > nc) ls.n_summarised = nc;
   if (ls.n_gated > nc) ls.n_gated = 0;          // the carried LSTM state is past the cut: gate again from chunk 0
-  if (ls.n_compacted > nc) ls.n_compacted = nc;
+  if (ls.n_compacted > nc) {
+    // the keep list on the device may name chunks that are raw tail again: drop it; attention reads
+    // every stored row until the next kvE_compact / kvE_compact_topk, which is exact
+    ls.n_compacted = 0;
+    ls.by_topk = false;
+  }
+  return KVE_OK;
+}
+
+int kvE_set_attend(kvE_store* st, int attend) {
+  if (!st || (attend != KVE_ATTEND_SUMMARY && attend != KVE_ATTEND_RAW)) return KVE_ERR_ARG;
+  st->cfg.attend = attend;
   return KVE_OK;
 }
 
 int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE_agg_weights* w,
                          void* stream) {
   if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   if (chunk_end > stale_chunks(st->cfg, ls.n_tokens)) return KVE_ERR_STATE;   // the window is never summarised
   const bool mlp = st->cfg.agg == KVE_AGG_MLP;
@@ -320,6 +358,7 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
 
 int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE_lstm_weights* w, void* stream) {
   if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (!w || !w->W_ih || !w->W_hh || !w->b_ih || !w->b_hh || !w->w_s) return KVE_ERR_ARG;
   LayerState& ls = st->layers[layer];
   if (chunk_end > ls.n_summarised) return KVE_ERR_STATE;
@@ -350,6 +389,7 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE
 
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_compact(view(st, layer), ls.n_gated, tau, static_cast<cudaStream_t>(stream));
@@ -362,6 +402,7 @@ int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
 
 int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream) {
   if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   if (ls.n_gated > 2048) return KVE_ERR_GEOMETRY;      // the kernel stages one sequence's scores per warp
   Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
@@ -376,6 +417,7 @@ int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, 
                       int64_t capacity, int32_t* free_count, void* stream) {
   if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin || !free_list || !free_count || capacity < 0)
     return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (mode != KVE_RECLAIM_DISCARDED && mode != KVE_RECLAIM_GATED) return KVE_ERR_ARG;
   const LayerState& ls = st->layers[layer];
   if (chunk_end > ls.n_compacted) return KVE_ERR_STATE;                        // only chunks the retention rule has judged
@@ -393,6 +435,7 @@ int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, 
 
 int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {
   if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;      // grouped query heads go through kvE_decode_attn_block
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   return run_attention(st, layer, mode, q, out, lse, scale, static_cast<cudaStream_t>(stream));
@@ -400,6 +443,7 @@ int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* l
 
 int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {
   if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   return run_attention(st, layer, ATTN_DENSE, q, out, lse, scale, static_cast<cudaStream_t>(stream));
 }
@@ -407,6 +451,7 @@ int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, fl
 int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_tokens, int dense, int causal, void* out,
                           float* lse, float scale, void* stream) {
   if (bad_layer(st, layer) || !q || !out || n_query_tokens <= 0) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (!st->block_ready) return KVE_ERR_STATE;                  // cfg.max_query_tokens was 0
   if (n_query_tokens > st->cfg.max_query_tokens) return KVE_ERR_CAPACITY;
   const AttnMode mode = dense ? ATTN_DENSE : (st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY);
@@ -419,6 +464,10 @@ int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_t
     tail = n_upper - (long long)ls.n_compacted * st->cfg.C;
     lead = (long long)ls.n_compacted * (mode == ATTN_RAW ? st->cfg.C : 1);
   }
+  // causal: the block's tokens are the newest rows of the raw tail; a tail shorter than the block would
+  // leave the first tokens without a defined position
+  if (causal && (long long)ls.n_tokens - (mode == ATTN_DENSE ? 0 : (long long)ls.n_compacted * st->cfg.C) < n_query_tokens)
+    return KVE_ERR_STATE;
   const long long tiles = (tail + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS + (lead + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS;
   long long splits = st->block_split_cap;
   if (splits > tiles) splits = tiles;
@@ -440,6 +489,7 @@ static int decode_step_host(kvE_store* st, int layer, const void* k_new_host, co
                             void* out_host, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, float scale,
                             int from_scratch, void* stream, bool wait) {
   if (bad_layer(st, layer) || !k_new_host || !v_new_host || !q_host || !out_host || !lw) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t row_bytes = (size_t)st->S * 128 * 2;
@@ -578,6 +628,7 @@ cudaError_t static_scratch(unsigned char** out) {
 extern "C" int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale,
                                       void* stream) {
   if (bad_layer(st, layer) || !q || !out) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
   if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   const LayerState& ls = st->layers[layer];

@@ -84,7 +84,7 @@ __global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
 cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, int pos0, cudaStream_t st) {
   const long long total = (long long)v.S * n_new * 32;
   long long blocks = (total + 255) / 256;
-  if (blocks > 148LL * 32) blocks = 148LL * 32;   // grid-stride beyond 32 CTAs per SM
+  if (blocks > sm_count() * 32LL) blocks = sm_count() * 32LL;   // grid-stride beyond 32 CTAs per SM
   if (blocks < 1) blocks = 1;
   return launch_pdl(kve_append_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v, static_cast<const uint4*>(k_new),
                     static_cast<const uint4*>(v_new), n_new, pos0);
@@ -93,7 +93,7 @@ cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_n
 cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, int32_t* ticket,
                                cudaStream_t st) {
   long long blocks = ((long long)v.S * n_new * 32 + 255) / 256;
-  if (blocks > 148LL * 32) blocks = 148LL * 32;
+  if (blocks > sm_count() * 32LL) blocks = sm_count() * 32LL;
   return launch_pdl(kve_append_next_kernel, dim3((unsigned)blocks), dim3(256), 0, st, v, static_cast<const uint4*>(k_new),
                     static_cast<const uint4*>(v_new), n_new, ticket);
 }

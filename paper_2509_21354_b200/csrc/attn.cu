@@ -106,9 +106,14 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   const int n_lead = (a.mode == ATTN_RAW) ? M * v.C : M;
   const int n_tail = max(0, n - raw0);
   const int n_rows = n_tail + n_lead;
-  const int n_splits = max(1, (n_rows + a.rows_per_split - 1) / a.rows_per_split);
-  // the sequence has outgrown what this launch was sized for (a replayed launch): rows would be dropped
-  if (n_splits > (int)gridDim.x && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
+  int n_splits = max(1, (n_rows + a.rows_per_split - 1) / a.rows_per_split);
+  // the sequence has outgrown what this launch was sized for (a replayed launch): rows beyond the grid
+  // are dropped, which the status word reports; the splits that exist still merge, so the ticket
+  // counter returns to zero and a later, correctly sized launch starts clean
+  if (n_splits > (int)gridDim.x) {
+    if (split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
+    n_splits = (int)gridDim.x;
+  }
   if (split >= n_splits) return;
   const int r_begin = split * a.rows_per_split;
   const int r_end = min(n_rows, r_begin + a.rows_per_split);
@@ -303,11 +308,10 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_t
                         cudaStream_t st) {
   (void)n_tokens_upper;
   if (v.S <= 0) return cudaSuccess;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kve_decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);
+  static DeviceFlags opted;
+  {
+    cudaError_t e = smem_opt_in(opted, kve_decode_attn_kernel, AT_SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   AttnArgs a;
   a.v = v; a.mode = (int)mode; a.n_chunks = n_chunks;

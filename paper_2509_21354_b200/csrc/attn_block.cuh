@@ -38,6 +38,7 @@ struct BlockArgs {
 
 struct BlockGeom {
   int raw0, n_tail, tail_pad, n_rows, n_splits, r_begin, r_end, n_tiles;
+  bool outgrown;      // the sequence needs more splits than the launch has: rows beyond the grid are dropped (flagged)
   // valid rows of the tile that starts at padded row `row0`
   __device__ __forceinline__ int rows_valid(int row0) const {
     return row0 < tail_pad ? min(BK_TILE, n_tail - row0) : min(BK_TILE, n_rows - row0);
@@ -56,6 +57,10 @@ __device__ __forceinline__ BlockGeom block_geometry(const BlockArgs& a, int s, i
   g.tail_pad = (g.n_tail + BK_TILE - 1) / BK_TILE * BK_TILE;
   g.n_rows = g.tail_pad + n_lead;
   g.n_splits = max(1, (g.n_rows + a.rows_per_split - 1) / a.rows_per_split);
+  // a replayed launch the sequence has outgrown: the splits that exist still merge and the ticket
+  // counter still returns to zero; the caller learns about the dropped rows from the status word
+  g.outgrown = g.n_splits > (int)gridDim.x;
+  g.n_splits = min(g.n_splits, (int)gridDim.x);
   g.r_begin = split * a.rows_per_split;
   g.r_end = min(g.n_rows, g.r_begin + a.rows_per_split);
   g.n_tiles = (max(g.r_end - g.r_begin, 0) + BK_TILE - 1) / BK_TILE;

@@ -95,7 +95,7 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
 
   const BlockGeom gm = block_geometry(a, s, split);
   // the sequence has outgrown what this launch was sized for (a replayed launch): rows would be dropped
-  if (gm.n_splits > (int)gridDim.x && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
+  if (gm.outgrown && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
   if (split >= gm.n_splits) return;
   const int n_tiles = gm.n_tiles;
 
@@ -421,12 +421,10 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
 
 template <int REP>
 static cudaError_t launch_tc(const CUtensorMap* tm, const BlockArgs& a, dim3 grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kve_decode_attn_block_tc_kernel<REP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         TC_SMEM_BYTES);
+  static DeviceFlags opted;
+  {
+    cudaError_t e = smem_opt_in(opted, kve_decode_attn_block_tc_kernel<REP>, TC_SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   return launch_pdl(kve_decode_attn_block_tc_kernel<REP>, grid, dim3(TC_THREADS), TC_SMEM_BYTES, st, tm[0], tm[1], tm[2], tm[3], a);
 }

@@ -175,15 +175,14 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
   const int n_cols = 4 * d_g;                     // 256, 512 or 1024: whole 256-column slices
   if (n_cols % PJ_N != 0) return cudaErrorInvalidValue;
   if (n_rows + PJ_M >= (1LL << 31) || (long long)v.S * v.max_chunks >= (1LL << 31)) return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kve_gate_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PJ_SMEM_BYTES);
+  static DeviceFlags opted;
+  {
+    cudaError_t e = smem_opt_in(opted, kve_gate_proj_kernel, PJ_SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   const int col_slices = n_cols / PJ_N;
   const long long n_tiles = (n_rows + PJ_M - 1) / PJ_M;
-  long long row_ctas = 148 / col_slices;          // one CTA per SM (shared memory), every slice equally served
+  long long row_ctas = sm_count() / col_slices;          // one CTA per SM (shared memory), every slice equally served
   if (row_ctas > n_tiles) row_ctas = n_tiles;
   if (row_ctas < 1) row_ctas = 1;
   dim3 grid((unsigned)col_slices, (unsigned)row_ctas);

@@ -319,11 +319,10 @@ template <int DG, int CL, int NG>
 static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
   constexpr int NS = 8 * NG;      // sequences per cluster
   constexpr int smem = 2 * RNN_PLANES * NS * DG * 2 + RNN_PLANES * NS * (DG / CL) * 2 + NG * 2 * 8;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kve_gate_rnn_kernel<DG, CL, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  static DeviceFlags opted;
+  {
+    cudaError_t e = smem_opt_in(opted, kve_gate_rnn_kernel<DG, CL, NG>, smem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   const int clusters = (a.S + NS - 1) / NS;
   return launch_pdl(kve_gate_rnn_kernel<DG, CL, NG>, dim3(clusters * CL), dim3(RNN_THREADS), smem, st, a);
@@ -339,9 +338,9 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
   // two 8-sequence groups per cluster once one group per cluster would need more than one wave of clusters
   cudaError_t e;
   switch (d_g) {
-    case 256: e = (v.S > 8 * (148 / 4)) ? launch_rnn_t<256, 4, 2>(a, st) : launch_rnn_t<256, 4, 1>(a, st); break;
+    case 256: e = (v.S > 8 * (sm_count() / 4)) ? launch_rnn_t<256, 4, 2>(a, st) : launch_rnn_t<256, 4, 1>(a, st); break;
     case 128: e = launch_rnn_t<128, 1, 1>(a, st); break;
-    case 64:  e = (v.S > 8 * 148) ? launch_rnn_t<64, 1, 2>(a, st) : launch_rnn_t<64, 1, 1>(a, st); break;
+    case 64:  e = (v.S > 8 * sm_count()) ? launch_rnn_t<64, 1, 2>(a, st) : launch_rnn_t<64, 1, 1>(a, st); break;
     default:  return cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;

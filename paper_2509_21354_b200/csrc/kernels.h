@@ -4,7 +4,28 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 namespace kve {
+
+// ---- per-device launch state ------------------------------------------------------------------------
+// A process may drive several GPUs.  The opt-in for more than 48 KB of dynamic shared memory is a
+// property of (kernel, device), and grids are sized from the SM count of the device that runs them,
+// so both are looked up once per device (the device that is current when the launch is issued).
+constexpr int MAX_DEVICES = 64;
+int sm_count();                                   // SMs of the current device (cached per device; 148 on a B200)
+struct DeviceFlags { std::atomic<unsigned char> done[MAX_DEVICES]; };
+template <typename Kernel>
+inline cudaError_t smem_opt_in(DeviceFlags& f, Kernel kernel, int bytes) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (f.done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) f.done[dev].store(1, std::memory_order_release);
+  return e;
+}
 
 // Device pointers of ONE layer plus the geometry the kernels need.
 struct LayerView {

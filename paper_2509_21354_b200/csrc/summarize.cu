@@ -88,7 +88,7 @@ cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_out
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
   long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
-  if (blocks > 148LL * 8) blocks = 148LL * 8;      // 64 resident warps per SM, every CTA resident from the start
+  if (blocks > sm_count() * 8LL) blocks = sm_count() * 8LL;      // 64 resident warps per SM, every CTA resident from the start
   if (pool_max)
     return launch_pdl(kve_chunk_mean_kernel<true>, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units, 1);
   return launch_pdl(kve_chunk_mean_kernel<false>, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units,
@@ -474,24 +474,22 @@ cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeight
   if (n_units <= 0) return cudaSuccess;
   if (d_sum % 64 == 0 && d_sum <= MT_MAX_DSUM && n_units + MT_M < (1LL << 31) &&
       (long long)v.S * v.max_chunks < (1LL << 31)) {
-    static bool attr_tc = false;
-    if (!attr_tc) {
-      cudaError_t e = cudaFuncSetAttribute(kve_chunk_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MT_SMEM_BYTES);
+    static DeviceFlags opted_tc;
+    {
+      cudaError_t e = smem_opt_in(opted_tc, kve_chunk_mlp_tc_kernel, MT_SMEM_BYTES);
       if (e != cudaSuccess) return e;
-      attr_tc = true;
     }
     const long long n_tiles = (n_units + MT_M - 1) / MT_M;
-    const long long per_side = n_tiles < 74 ? n_tiles : 74;      // one CTA per SM: half of the 148 SMs per side
+    const long long half = sm_count() / 2;
+    const long long per_side = n_tiles < half ? n_tiles : half;  // one CTA per SM: half of the SMs per side
     dim3 grid((unsigned)per_side, 2);
     return launch_pdl(kve_chunk_mlp_tc_kernel, grid, dim3(MT_THREADS), MT_SMEM_BYTES, st, v, t0, n_range, n_units, w, d_sum);
   }
   const size_t smem = sizeof(float) * (size_t)MLP_ROWS * (D + d_sum);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kve_chunk_mlp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(sizeof(float) * MLP_ROWS * (D + 1024)));
+  static DeviceFlags opted;
+  {
+    cudaError_t e = smem_opt_in(opted, kve_chunk_mlp_kernel, (int)(sizeof(float) * MLP_ROWS * (D + 1024)));
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   dim3 grid((unsigned)((n_units + MLP_ROWS - 1) / MLP_ROWS), 2);
   return launch_pdl(kve_chunk_mlp_kernel, grid, dim3(MLP_THREADS), smem, st, v, t0, n_range, n_units, w, d_sum);

@@ -220,30 +220,35 @@ def test_causal_block_attention_matches_oracle(G, T, n):
         _check(b, pb, st, attend, G, T, dense=True, step=1, causal=True)
 
 
-def test_causal_block_with_a_tail_shorter_than_the_block():
-    # W = 4, C = 8: the raw tail holds 4..11 rows, fewer than the 12 query tokens, so the first tokens see no
-    # raw row at all (only kept chunks) - rows whose running maximum stays -inf over the whole tail
+def test_causal_block_with_a_tail_shorter_than_the_block_is_refused():
+    # W = 4, C = 8: the raw tail holds 4..11 rows, fewer than the 12 query tokens, so the first tokens would
+    # have no position inside the raw tail (the oracle refuses that case as well): KVE_ERR_STATE, nothing runs
     wl = wlm.CFG1.small(B=1, H=2, n=203, C=8, W=4, seed=32)
     b, pb, st = _prepared(wl, "summary", 2, 12)
-    assert wl.n - pb.Nc * wl.C < 12
-    wl_t = wl
-    q = wlm.gen_q_block(wl_t, 12, 4, 0, 0)
+    tail = wl.n - pb.Nc * wl.C
+    assert tail < 12
+    q = b.bits_to_bf16(wlm.gen_q_block(wl, 12, 4, 0, 0))
+    with pytest.raises(b.KveError) as e:
+        st.decode_attn_block(0, q, causal=True)
+    assert e.value.rc == -4
+    # as many query tokens as the tail has rows is the limit case and is served
+    T = tail
+    q = wlm.gen_q_block(wl, T, 4, 0, 0)
     out = st.decode_attn_block(0, b.bits_to_bf16(q), causal=True)
     torch.cuda.synchronize()
     assert st.poll_status() == 0
-    # oracle per token: gated chunks beyond the token's own position do not exist for it either, so the
-    # comparison is restricted to the tokens whose prefix still covers all gated chunks
-    tail = wl.n - pb.Nc * wl.C
     got = wlm.bf16_bits_to_f32(b.bf16_to_bits(out)).astype(np.float64)
-    for t in range(12 - tail, 12):
-        n_t = wl.n - (11 - t)
+    for t in range(T):
+        n_t = wl.n - (T - 1 - t)
         for g in range(2):
             qs = np.ascontiguousarray(q[:, t, g::2, :].reshape(wl.S, 128))
             want, _, _, _ = pb.o64.attn(qs, np.ascontiguousarray(pb.K[:, :n_t]), np.ascontiguousarray(pb.V[:, :n_t]), wl.C, pb.Nc,
                                         pb.idx64, pb.cnt64, pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)
             assert np.abs(got[0, t, g::2] - want).max() <= 2e-2
-    # tokens whose position lies inside the gated range: they see every kept chunk and no raw row (finite, no NaN)
-    assert np.isfinite(got).all()
+    # the full-cache form counts all stored tokens as the tail, so 12 tokens are fine there
+    st.decode_attn_block(0, b.bits_to_bf16(wlm.gen_q_block(wl, 12, 4, 0, 0)), dense=True, causal=True)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
 
 
 @pytest.mark.parametrize("n", [2048, 2051])
