@@ -210,7 +210,7 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
     keep = st.keep_cnt[0].float().mean().item()
     q = torch.randn((g.B, T, Hkv * G, 128), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     out = torch.empty_like(q)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = Flusher()
     st.profile(True)
     res = {"what": f"kvE_decode_attn_block: {T} query tokens x {Hkv * G} query heads on {Hkv} KV heads, B={g.B}, n={n}; "
                    "tcgen05 kernel, one launch timed alone, L2 flushed",
@@ -218,7 +218,7 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
     for name, dense, rows in (("gated", False, n - Nc * g.C + keep), ("dense", True, n)):
         ts = []
         for i in range(12):
-            flush.fill_(1)
+            flush()
             st.decode_attn_block(0, q, dense=dense, out=out)
             torch.cuda.synchronize()
             if i >= 2:
@@ -399,14 +399,18 @@ def iters_for(fn, target_s=0.15, lo=10, hi=400):
 
 
 class Flusher:
-    """writes a buffer larger than L2 (126 MB) so that the next launch starts cold"""
+    """Leaves L2 (126 MB) cold AND clean before the next launch: writes a 256 MB buffer (every line of the launch's
+    data is gone), then reads another 256 MB buffer (the dirty lines of the write are written back now, not under the
+    timed kernel's first reads, where they would be billed to it as extra DRAM traffic)."""
 
     def __init__(self):
         import torch
-        self.buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        self.wbuf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        self.rbuf = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda")
 
     def __call__(self):
-        self.buf.fill_(1)
+        self.wbuf.fill_(1)
+        self.rbuf.max()
 
 
 def copy_us(total_bytes, flush):

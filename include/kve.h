@@ -126,12 +126,14 @@ int kvE_append(kvE_store* st, int layer, const void* k_new, const void* v_new, i
  * replay appends the next n_new tokens (k_new, v_new: DEVICE bf16 [S][n_new][d], read at replay time).  This is the decode
  * loop between two gate triggers of Sec. 3.3 without a host round trip per token.
  *   n_reserve: how many further tokens such appends (replays included) may add before the next kvE_set_len or
- *   kvE_append; attention launches issued after this call are sized for that much growth, so they stay valid
- *   when replayed along.  The handle's own length advances by n_new per call, not per replay: after replaying,
- *   give it the true length with kvE_set_len(layer, n) before summarising or gating the chunks that have
- *   completed meanwhile (attention keeps reading them as raw rows until then, which is exact).
- *   Device side: a sequence without room for n_new more tokens is left alone, and an attention launch replayed past the
- *   growth it was sized for drops nothing silently: both set KVE_ERR_CAPACITY in the status word. */
+ *   kvE_append.  kvE_decode_attn / kvE_decode_attn_dense cut their work into pieces on the device from the length
+ *   they find there, so a replayed launch follows the cache however far it grows; kvE_decode_attn_block launches
+ *   issued after this call are sized for n_reserve more tokens, and one replayed past that sets KVE_ERR_CAPACITY in
+ *   the status word instead of dropping rows.  The handle's own length advances by n_new per call, not per replay:
+ *   after replaying, give it the true length with kvE_set_len(layer, n) before summarising or gating the chunks
+ *   that have completed meanwhile (attention keeps reading them as raw rows until then, which is exact).
+ *   Device side: a sequence without room for n_new more tokens is left alone and KVE_ERR_CAPACITY is set in the
+ *   status word. */
 int kvE_append_next(kvE_store* st, int layer, const void* k_new, const void* v_new, int n_new, int n_reserve,
                     void* stream);
 
@@ -219,15 +221,15 @@ int kvE_decode_attn_block(kvE_store* st, int layer, const void* q, int n_query_t
  * running: a robot-control loop that handed the whole GPU to its framework's memory pool at
  * start-up and may not stall on, or fail in, an allocation between two control ticks; a plug-in that
  * is given device pointers by a host application and has no right to allocate on that device.  For
- * them the split-K partial results and tickets of the attention kernel live in a device array that
+ * them the partial results and tickets of the attention kernel live in a device array that
  * is part of the library image itself (KVE_STATIC_SCRATCH_BYTES, about 2.1 MiB, held by every GPU that
  * loads the library until the process exits) instead of the handle's workspace, and this call
  * performs no cudaMalloc / cudaFree and calls no allocating routine.
  *   - same arguments, result and errors as kvE_decode_attn (gated attention of `layer`, mode from
  *     cfg.attend); q, out: DEVICE bf16 [S][d]; lse: DEVICE fp32 [S] or NULL.
- *   - limits: S <= KVE_STATIC_MAX_SEQUENCES and S * splits <= KVE_STATIC_MAX_PARTIALS, where splits
- *     (1..32) is what the library picks for the layer's current length; beyond that the call
- *     returns KVE_ERR_CAPACITY without launching (text via kvE_last_cuda_error).
+ *   - limits: S <= KVE_STATIC_MAX_SEQUENCES and S + CTAs <= KVE_STATIC_MAX_PARTIALS, where CTAs (at most two
+ *     per SM: 296 on a B200) is the size of the launch the library picks for the layer's current state;
+ *     beyond that the call returns KVE_ERR_CAPACITY without launching (text via kvE_last_cuda_error).
  *   - the first call on each device looks up the array's device address (that device must be
  *     current); make that first call outside any stream capture.
  *   - one array per device, shared by every handle and stream: the call clears the tickets it

@@ -27,8 +27,8 @@ struct kvE_store {
   int device = -1;       // the device that was current at kvE_create: owner of every buffer; calls check it
   int S, max_chunks;
   // workspace carve-up (byte offsets)
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, ws_needed;
-  int max_splits;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, ws_needed;
+  int attn_grid_max;     // most CTAs an attention launch uses (two per SM of the handle's device): sizes the partial records
   // block-of-queries attention: tensor maps over the page pools and the summary store (encoded at
   // create when cfg.max_query_tokens > 0), rows per page box, split cap the workspace was sized for
   alignas(64) unsigned char block_maps[4 * ATTN_BLOCK_MAP_BYTES];
@@ -57,7 +57,8 @@ int kve::sm_count() {
 
 namespace {
 
-constexpr int MAX_SPLITS = 32;
+constexpr int MAX_SPLITS = 32;            // block-of-queries attention: most splits per sequence
+constexpr size_t ATTN_GRID_LIMIT = 1024;  // most CTAs of one kvE_decode_attn launch the workspace is sized for (>= 2 per SM)
 constexpr size_t ALIGN = 256;
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 constexpr size_t align_const(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
@@ -81,8 +82,13 @@ int check_config(const kvE_config* c) {
 }
 
 struct Carve {
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, total;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, total;
 };
+// most CTAs of one attention launch: two resident per SM (148 SMs assumed where no device can be asked)
+int attn_grid_cap() {
+  int dev = 0;
+  return 2 * (cudaGetDevice(&dev) == cudaSuccess ? sm_count() : 148);
+}
 // most splits per sequence the block-of-queries attention uses: one CTA per SM, one wave
 int block_split_cap(long long S) {
   long long c = sm_count() / S;
@@ -94,7 +100,8 @@ Carve carve(const kvE_config& c) {
   Carve k;
   size_t o = 0;
   k.off_P = o;        o = align_up(o + S * max_chunks * 4 * (size_t)c.d_g * sizeof(float));
-  k.off_partials = o; o = align_up(o + S * MAX_SPLITS * ATTN_PARTIAL_FLOATS * sizeof(float));
+  // attention partial records: the one of (sequence s, CTA c) at s + c, at most ATTN_GRID_LIMIT CTAs
+  k.off_partials = o; o = align_up(o + (S + ATTN_GRID_LIMIT) * ATTN_PARTIAL_FLOATS * sizeof(float));
   k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
   k.off_stage = o;    o = align_up(o + 4 * S * 128 * 2);   // k_new, v_new, q, out of kvE_decode_step_host
   k.off_reclaim = o;  o = align_up(o + (2 * S + 1) * sizeof(int32_t));   // per-sequence counts and offsets of kvE_reclaim_pages
@@ -104,6 +111,10 @@ Carve carve(const kvE_config& c) {
     const size_t rows = ((size_t)c.max_query_tokens * (c.Hq / c.Hkv) + 15) / 16 * 16;
     o = align_up(o + S * block_split_cap((long long)S) * rows * ATTN_PARTIAL_FLOATS * sizeof(float));
   }
+  // what kvE_compact leaves for attention: the kept summary rows, compacted per sequence
+  const size_t sum_bytes = (size_t)c.n_layers * S * max_chunks * 128 * 2;
+  k.off_kept_k = o;   o = align_up(o + sum_bytes);
+  k.off_kept_v = o;   o = align_up(o + sum_bytes);
   k.total = o;
   return k;
 }
@@ -163,41 +174,64 @@ bool wrong_device(const kvE_store* st) {
   return cudaGetDevice(&dev) != cudaSuccess || dev != st->device;
 }
 
-// rows per split and grid width for `n_rows_upper` logical rows per sequence
-AttnPlan plan_attention(const kvE_store* st, long long n_rows_upper) {
-  const long long one_wave = sm_count() * 2LL;     // two CTAs per SM: everything resident at once, fewest merges
-  long long splits = one_wave / st->S;
-  const long long max_useful = (n_rows_upper + 2 * ATTN_TILE_ROWS - 1) / (2 * ATTN_TILE_ROWS);   // >= 128 rows per split
-  if (splits > max_useful) splits = max_useful;
-  if (splits > MAX_SPLITS) splits = MAX_SPLITS;
-  if (splits < 1) splits = 1;
-  long long rows = (n_rows_upper + splits - 1) / splits;
-  rows = (rows + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS * ATTN_TILE_ROWS;
-  if (rows < ATTN_TILE_ROWS) rows = ATTN_TILE_ROWS;
-  AttnPlan p;
-  p.rows_per_split = (int)rows;
-  p.max_splits = (int)((n_rows_upper + rows - 1) / rows);
-  if (p.max_splits < 1) p.max_splits = 1;
-  return p;
+// How an attention launch is cut up.  Every sequence is cut into k equal parts and CTA c of G takes the contiguous
+// run of parts [c S k / G, (c + 1) S k / G), which it streams as one piece (no break between parts of one sequence).
+// G is one resident wave at most (two CTAs per SM).  k is chosen by a small cost model in units of 64-row tiles: the
+// busiest CTA's tiles, plus two tiles' worth of time for the exchange through global memory that is needed as soon as
+// a sequence is shared between CTAs (k > 1).  Small k keeps whole sequences together; large k evens out the bytes per
+// CTA when S is not a multiple of the wave.
+struct AttnCut { int k, grid; };
+AttnCut attention_cut(const kvE_store* st, AttnMode mode, const LayerState& ls) {
+  const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
+  long long tail, lead;
+  if (mode == ATTN_DENSE) { tail = n_upper; lead = 0; }
+  else {
+    tail = n_upper - (long long)ls.n_compacted * st->cfg.C;
+    lead = (long long)ls.n_compacted * (mode == ATTN_RAW ? st->cfg.C : 1) / 2;      // about half of the chunks are kept
+  }
+  long long tiles = (tail + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS + (lead + ATTN_TILE_ROWS - 1) / ATTN_TILE_ROWS;
+  if (tiles < 1) tiles = 1;
+  const long long G = st->attn_grid_max, S = st->S;
+  const long long k_max = tiles < MAX_SPLITS ? tiles : MAX_SPLITS;
+  AttnCut cut{1, 1};
+  double best = 1e30;
+  for (long long k = 1; k <= k_max; ++k) {
+    if (S * k * (G + 1) >= (1LL << 32)) break;                          // the kernel cuts the parts up in 32-bit arithmetic
+    const long long parts = S * k, grid = parts < G ? parts : G;
+    const long long rounds = (parts + grid - 1) / grid;                 // parts of the busiest CTA
+    const double cost = (double)rounds * (double)tiles / (double)k + (k > 1 ? 2.0 : 0.0);
+    if (cost < best - 0.25 || (cost <= best + 1e-9 && k > 1)) {         // ties go to the finer cut (evener bytes)
+      best = cost < best ? cost : best;
+      cut.k = (int)k;
+      cut.grid = (int)grid;
+    }
+  }
+  return cut;
+}
+
+struct KeptRows { void *k, *v; };      // kept summary rows of a layer, compacted by kvE_compact
+KeptRows kept_rows(const kvE_store* st, int layer) {
+  char* ws = static_cast<char*>(st->buf.workspace);
+  const size_t rows = (size_t)layer * st->S * st->max_chunks;
+  return KeptRows{ws + st->off_kept_k + rows * 256, ws + st->off_kept_v + rows * 256};
+}
+
+int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* out, float* lse, float scale,
+                  float* partials, int32_t* counters, cudaStream_t stream) {
+  const LayerState& ls = st->layers[layer];
+  const KeptRows kr = kept_rows(st, layer);
+  const AttnCut cut = attention_cut(st, mode, ls);
+  Prof prof(st, mode == ATTN_DENSE ? KVE_K_ATTN_DENSE : KVE_K_ATTN, stream);
+  cudaError_t e = launch_attn(view(st, layer), mode, ls.n_compacted, cut.k, cut.grid, q, out, lse, scale, kr.k, kr.v, partials,
+                              counters, stream);
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
 }
 
 int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* out, float* lse, float scale,
                   cudaStream_t stream) {
-  const LayerState& ls = st->layers[layer];
-  const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
-  long long rows_upper;
-  if (mode == ATTN_DENSE) rows_upper = n_upper;
-  else {
-    const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;
-    rows_upper = (long long)ls.n_compacted * per + (n_upper - (long long)ls.n_compacted * st->cfg.C);
-  }
-  AttnPlan plan = plan_attention(st, rows_upper);
   char* ws = static_cast<char*>(st->buf.workspace);
-  Prof prof(st, mode == ATTN_DENSE ? KVE_K_ATTN_DENSE : KVE_K_ATTN, stream);
-  cudaError_t e = launch_attn(view(st, layer), mode, ls.n_compacted, ls.n_tokens, plan, q, out, lse, scale,
-                              reinterpret_cast<float*>(ws + st->off_partials),
-                              reinterpret_cast<int32_t*>(ws + st->off_counters), stream);
-  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+  return run_attention(st, layer, mode, q, out, lse, scale, reinterpret_cast<float*>(ws + st->off_partials),
+                       reinterpret_cast<int32_t*>(ws + st->off_counters), stream);
 }
 
 }  // namespace
@@ -232,7 +266,10 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   st->S = cfg->B * cfg->Hkv;
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
   st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
-  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_ticket = k.off_ticket; st->off_block = k.off_block; st->ws_needed = k.total;
+  st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_ticket = k.off_ticket; st->off_block = k.off_block;
+  st->off_kept_k = k.off_kept_k; st->off_kept_v = k.off_kept_v; st->ws_needed = k.total;
+  st->attn_grid_max = attn_grid_cap();
+  if ((size_t)st->attn_grid_max > ATTN_GRID_LIMIT) st->attn_grid_max = (int)ATTN_GRID_LIMIT;
   if (cfg->max_query_tokens > 0) {
     st->block_hp = attn_block_hp(cfg->C);
     st->block_split_cap = block_split_cap(st->S);
@@ -245,9 +282,8 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
     }
     st->block_ready = true;
   }
-  st->max_splits = MAX_SPLITS;
   st->layers.assign(cfg->n_layers, LayerState());
-  cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.total - k.off_partials);
+  cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.off_kept_k - k.off_partials);
   if (e == cudaSuccess) e = cudaMemset(buf->status_word, 0, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(buf->seq_len, 0, sizeof(int32_t) * (size_t)cfg->n_layers * cfg->B);
   if (e == cudaSuccess) e = cudaMemset(buf->keep_cnt, 0, sizeof(int32_t) * (size_t)cfg->n_layers * st->S);
@@ -353,6 +389,7 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   if (chunk_begin <= ls.n_summarised && chunk_end > ls.n_summarised) ls.n_summarised = chunk_end;
+  if (ls.n_compacted > chunk_begin) ls.n_compacted = chunk_begin;   // the compacted copies of these summaries are stale
   return KVE_OK;
 }
 
@@ -392,7 +429,8 @@ int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
-  cudaError_t e = launch_compact(view(st, layer), ls.n_gated, tau, static_cast<cudaStream_t>(stream));
+  const KeptRows kr = kept_rows(st, layer);
+  cudaError_t e = launch_compact(view(st, layer), ls.n_gated, tau, kr.k, kr.v, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_compacted = ls.n_gated;
   ls.tau = tau;
@@ -406,7 +444,8 @@ int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream) {
   LayerState& ls = st->layers[layer];
   if (ls.n_gated > 2048) return KVE_ERR_GEOMETRY;      // the kernel stages one sequence's scores per warp
   Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
-  cudaError_t e = launch_compact_topk(view(st, layer), ls.n_gated, k, static_cast<cudaStream_t>(stream));
+  const KeptRows kr = kept_rows(st, layer);
+  cudaError_t e = launch_compact_topk(view(st, layer), ls.n_gated, k, kr.k, kr.v, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_compacted = ls.n_gated;
   ls.by_topk = true;
@@ -632,16 +671,13 @@ extern "C" int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, v
   if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   const LayerState& ls = st->layers[layer];
-  const long long per = (mode == ATTN_RAW) ? st->cfg.C : 1;
-  const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
-  const long long rows_upper = (long long)ls.n_compacted * per + (n_upper - (long long)ls.n_compacted * st->cfg.C);
-  const AttnPlan plan = plan_attention(st, rows_upper);
-  const long long records = (long long)st->S * plan.max_splits;
+  // the kernel needs S + G partial records for a launch of G CTAs
+  const int grid = attention_cut(st, mode, ls).grid;
+  const long long records = (long long)st->S + grid;
   if (st->S > STATIC_MAX_SEQ || records > STATIC_MAX_REC) {
-    st->cuda_error = "kvE_decode_attn_static: " + std::to_string(st->S) + " sequences x " +
-                     std::to_string(plan.max_splits) + " splits exceed the built-in scratch (" +
-                     std::to_string(STATIC_MAX_SEQ) + " sequences, " + std::to_string(STATIC_MAX_REC) +
-                     " partial records); use kvE_decode_attn";
+    st->cuda_error = "kvE_decode_attn_static: " + std::to_string(st->S) + " sequences on " + std::to_string(grid) +
+                     " CTAs exceed the built-in scratch (" + std::to_string(STATIC_MAX_SEQ) + " sequences, " +
+                     std::to_string(STATIC_MAX_REC) + " partial records); use kvE_decode_attn";
     return KVE_ERR_CAPACITY;
   }
   unsigned char* scratch = nullptr;
@@ -653,6 +689,5 @@ extern "C" int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, v
   // the array keeps whatever the last call left: the tickets must start at zero
   e = cudaMemsetAsync(counters, 0, sizeof(int32_t) * (size_t)st->S, s);
   if (e != cudaSuccess) return cuda_fail(st, e);
-  e = launch_attn(view(st, layer), mode, ls.n_compacted, ls.n_tokens, plan, q, out, lse, scale, partials, counters, s);
-  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+  return run_attention(st, layer, mode, q, out, lse, scale, partials, counters, s);
 }

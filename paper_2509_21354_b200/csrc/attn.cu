@@ -1,19 +1,30 @@
-// Split-K flash-decode over the retained set (Sec. 3.3, softmax of Eq. 1):
-//   out = softmax(q K'^T * scale) V',  rows of K', V' = [kept chunks, oldest first] ++ [raw tail]
+// Flash-decode over the retained set (Sec. 3.3, softmax of Eq. 1):
+//   out = softmax(q K'^T * scale) V',  rows of K', V' = [raw tail] ++ [kept chunks, oldest first]
 // and, with mode = DENSE, Eq. 1 over every stored token (the full-cache baseline).
 //
-// HBM-bound: every retained K and V row (256 bytes each) is read exactly once.
-//  * grid = (splits, sequences); a CTA owns a contiguous range of a sequence's logical rows
-//    (raw tail first, kept chunks after it).
-//  * one producer warp turns logical rows into addresses (summary store / page table), merges
-//    rows that are contiguous in memory into runs with a ballot, and issues one bulk copy
-//    (TMA engine, global -> shared, mbarrier byte counting) per run into a 3-stage ring of
-//    64-row K and V tiles.
-//  * eight consumer warps each take 8 rows of a tile: q.k partial sums per lane (4 head dims per
-//    lane), a butterfly transpose-reduce that leaves one row's logit per group of four lanes, online softmax
-//    with warp shuffles, then p.V with each lane owning 4 output dims.
-//  * per-CTA (m, l, acc) partials go to the workspace; the last CTA of a sequence to finish (atomic
-//    ticket, nobody spins) merges them by log-sum-exp and writes the bf16 output.
+// HBM-bound: every retained K and V row (256 bytes each) is read exactly once, so the kernel is built
+// to keep every SM streaming from its first microsecond to its last:
+//  * A sequence's rows form 64-row tiles (raw tail first, kept chunks after it).  The host picks k,
+//    the number of equal parts every sequence is cut into, so that the S k parts divide evenly over
+//    the CTAs of one resident wave (two per SM); CTA c takes parts [c S k / G, (c + 1) S k / G): a
+//    contiguous run that may span several sequences.  Its pipeline runs across sequence boundaries
+//    without draining, every CTA moves nearly the same number of bytes whatever S is, and where a
+//    part begins follows from the launch arguments, the stored length and one keep count, so the
+//    first copies leave two dependent loads after the kernel starts.
+//  * Warp 8 (producer) turns tiles into addresses (page table; kept summary rows sit compacted in
+//    one contiguous run per sequence), merges rows that are contiguous in memory into runs with a
+//    ballot, and issues one bulk copy (TMA engine, global -> shared, mbarrier byte counting) per run
+//    into a 3-stage ring of 64-row K and V tiles.  The query row of a sequence travels with the
+//    first tile of that sequence.
+//  * Warps 0-7 (consumers) each take 8 rows of a tile: q.k partial sums per lane (4 head dims per
+//    lane), a butterfly transpose-reduce that leaves one row's logit per group of four lanes, online
+//    softmax with warp shuffles, then p.V with each lane owning 4 output dims.  When a CTA's run
+//    leaves a sequence, the consumers drop their (m, l, acc) into a double-buffered exchange area
+//    and carry on with the next sequence.
+//  * Warp 9 (merger) folds the eight consumer states of a finished sequence (or part of one), and
+//    either writes the output (this CTA had the whole sequence) or a partial record plus an atomic
+//    ticket; the CTA that draws a sequence's last ticket merges its records by log-sum-exp.  Nobody
+//    spins on another CTA.
 // Every mbarrier wait is bounded; on give-up the status word gets KVE_ERR_TIMEOUT.
 #include "common.cuh"
 #include "kernels.h"
@@ -24,55 +35,75 @@ constexpr int AT_TILE = ATTN_TILE_ROWS;       // rows per stage
 constexpr int AT_STAGES = 3;
 constexpr int AT_CWARPS = 8;                  // consumer warps
 constexpr int AT_SUB = AT_TILE / AT_CWARPS;   // 8 rows per consumer warp per tile
-constexpr int AT_THREADS = (AT_CWARPS + 1) * 32;
+constexpr int AT_PRODUCER = AT_CWARPS;        // warp ids
+constexpr int AT_THREADS = (AT_CWARPS + 2) * 32;
 constexpr int AT_STAGE_ELEMS = AT_TILE * D;   // bf16 elements of one K (or V) tile
-constexpr int AT_SMEM_BYTES = 2 * AT_STAGES * AT_STAGE_ELEMS * 2 + AT_CWARPS * ATTN_PARTIAL_FLOATS * 4 + 2 * AT_STAGES * 8 + 16;
 static_assert(AT_SUB == 8, "the transpose-reduce below is written for 8 rows per warp");
+
+// shared-memory carve-up (bytes)
+constexpr int AT_OFF_K = 0;
+constexpr int AT_OFF_V = AT_OFF_K + AT_STAGES * AT_STAGE_ELEMS * 2;
+constexpr int AT_OFF_Q = AT_OFF_V + AT_STAGES * AT_STAGE_ELEMS * 2;                 // [stages][128] bf16
+constexpr int AT_OFF_COMB = AT_OFF_Q + AT_STAGES * ROW_BYTES;                       // [2][consumer warps][132] fp32
+constexpr int AT_OFF_INFO = AT_OFF_COMB + 2 * AT_CWARPS * ATTN_PARTIAL_FLOATS * 4;  // [stages] int4
+constexpr int AT_OFF_FINFO = AT_OFF_INFO + AT_STAGES * 16;                          // [2] int4
+constexpr int AT_OFF_BAR = AT_OFF_FINFO + 2 * 16;                                   // full[3], empty[3], ffull[2], fempty[2]
+constexpr int AT_SMEM_BYTES = AT_OFF_BAR + (2 * AT_STAGES + 4) * 8;
+static_assert(AT_OFF_COMB % 16 == 0 && AT_OFF_INFO % 16 == 0 && AT_OFF_BAR % 8 == 0, "alignment of the carve-up");
 
 int attn_smem_bytes() { return AT_SMEM_BYTES; }
 
+// tile flags handed from the producer to the consumers
+constexpr int TF_NEW = 1;      // first tile of a (sequence, list) in this CTA: fresh softmax state, query row in the stage
+constexpr int TF_FLUSH = 2;    // last tile of a (sequence, list) in this CTA: hand the state to the merger afterwards
+constexpr int TF_END = 4;      // no tile: the CTA's work is done
+
 struct AttnArgs {
   LayerView v;
-  int mode, n_chunks, rows_per_split, max_splits;
+  int mode, n_chunks;
+  int k;                       // parts per sequence
   const uint16_t* q;
   uint16_t* out;
   float* lse;
   float scale;
-  float* partials;     // [S][max_splits][132]
-  int32_t* counters;   // [S], zero between launches
+  const uint16_t* kkept;       // [S][max_chunks][128] kept summary rows, compacted (SUMMARY mode)
+  const uint16_t* vkept;
+  float* partials;             // [S + G][132]: the record of (sequence s, CTA c) sits at s + c
+  int32_t* counters;           // [S], zero between launches
 };
 
-// address of logical row L of sequence s (K and V); falls back to a safe row and flags the status
-// word when an index is out of range
-// The CTA walks a sequence's rows in the order [raw tail ; kept chunks]: the raw tail's addresses need
-// only the page table, so the first tiles can be requested while the keep list is still on its way
-// (softmax does not care about the order of its rows).
-__device__ __forceinline__ void row_address(const AttnArgs& a, int s, int L, int n_tail, int raw0,
-                                            const uint16_t*& kp, const uint16_t*& vp) {
+// what every role derives from the launch arguments and the stored length
+struct AttnGeo {
+  int n_tail, raw0, TT, per;   // tail rows / tiles per sequence; rows a kept chunk contributes
+  uint32_t I, P;               // parts in the launch (S k); CTAs that get any (min(G, I): none of them is empty)
+};
+
+// CTA c of P takes parts [c I / P, (c + 1) I / P); CTAs c >= P take none.  32-bit arithmetic (64-bit division
+// would sit on the path to the first copy): the host keeps I * G below 2^32.
+__device__ __forceinline__ uint32_t piece_begin(uint32_t c, uint32_t I, uint32_t P) { return c >= P ? I : (c * I) / P; }
+// the CTA that holds part x
+__device__ __forceinline__ uint32_t piece_of(uint32_t x, uint32_t I, uint32_t P) { return ((x + 1u) * P - 1u) / I; }
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Pulls what the producer will look up for sequence s into L2 (fire and forget: the keep count, the page ids
+// of the raw tail, the head of the kept-chunk list), so that the dependent look-ups that follow cost an L2 hit each.
+__device__ __forceinline__ void prefetch_sequence_metadata(const AttnArgs& a, int s, int lane) {
   const LayerView& v = a.v;
+  if (s < 0 || s >= v.S) return;
   const long long sb = (long long)s * v.max_chunks;
-  int chunk, r;
-  if (L < n_tail) {
-    const int p = raw0 + L;
-    chunk = p / v.C;
-    r = p - chunk * v.C;
-  } else if (a.mode == ATTN_SUMMARY) {
-    int t = v.keep_idx[sb + (L - n_tail)];
-    if (t < 0 || t >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); t = 0; }
-    kp = v.ksum_bf16 + (sb + t) * D;
-    vp = v.vsum_bf16 + (sb + t) * D;
-    return;
-  } else {            // RAW: row r of the ((L - n_tail) / C)-th kept chunk
-    const int ci = (L - n_tail) / v.C;
-    r = (L - n_tail) - ci * v.C;
-    chunk = v.keep_idx[sb + ci];
-    if (chunk < 0 || chunk >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); chunk = 0; }
-  }
-  long long page = v.page_table[sb + chunk];
-  if (page < 0 || page >= v.n_pages) { set_status(v.status, ERR_CAPACITY); page = 0; }
-  const long long off = (page * v.C + r) * D;
-  kp = v.k_pages + off;
-  vp = v.v_pages + off;
+  const int first_tail_chunk = (a.mode == ATTN_DENSE) ? 0 : a.n_chunks;
+  if (lane == 0) prefetch_l2(v.keep_cnt + s);
+  // page ids of the tail: 32 entries per 128-byte line; up to 8 lines (256 chunks) ahead
+  if (lane < 8 && first_tail_chunk + lane * 32 < v.max_chunks) prefetch_l2(v.page_table + sb + first_tail_chunk + lane * 32);
+  if (a.mode == ATTN_RAW && lane == 8) prefetch_l2(v.keep_idx + sb);
+}
+
+// rows the kept chunks of sequence s contribute
+__device__ __forceinline__ int lead_rows_of(const AttnArgs& a, const AttnGeo& g, int s) {
+  if (a.mode == ATTN_DENSE || a.n_chunks <= 0) return 0;
+  const int M = min(max(a.v.keep_cnt[s], 0), a.n_chunks);
+  return M * g.per;
 }
 
 #define KVE_TR_ROUND(OFF, CNT)                                                        \
@@ -85,81 +116,161 @@ __device__ __forceinline__ void row_address(const AttnArgs& a, int s, int L, int
     }                                                                                 \
   }
 
+// one tile of the CTA's work as the producer sees it
+struct TileDesc {
+  int s, list, j, rows, flags;      // list 0: raw tail, 1: kept chunks; j: tile index inside the sequence's list
+};
+
 __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
-  uint16_t* Ks = reinterpret_cast<uint16_t*>(smem);
-  uint16_t* Vs = Ks + AT_STAGES * AT_STAGE_ELEMS;
-  float* comb = reinterpret_cast<float*>(Vs + AT_STAGES * AT_STAGE_ELEMS);          // [AT_CWARPS][132]
-  uint64_t* full = reinterpret_cast<uint64_t*>(comb + AT_CWARPS * ATTN_PARTIAL_FLOATS);   // 16-byte aligned
+  uint16_t* Ks = reinterpret_cast<uint16_t*>(smem + AT_OFF_K);
+  uint16_t* Vs = reinterpret_cast<uint16_t*>(smem + AT_OFF_V);
+  uint16_t* Qs = reinterpret_cast<uint16_t*>(smem + AT_OFF_Q);
+  float* comb = reinterpret_cast<float*>(smem + AT_OFF_COMB);
+  int4* info = reinterpret_cast<int4*>(smem + AT_OFF_INFO);
+  int4* finfo = reinterpret_cast<int4*>(smem + AT_OFF_FINFO);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + AT_OFF_BAR);
   uint64_t* empty = full + AT_STAGES;
+  uint64_t* ffull = empty + AT_STAGES;
+  uint64_t* fempty = ffull + 2;
 
   pdl_launch_dependents();
   const LayerView& v = a.v;
-  const int s = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  pdl_wait();      // lengths, keep lists and summaries come from earlier kernels
-
-  int n = v.seq_len[s / v.H];
-  n = min(max(n, 0), v.max_tokens);
-  const int M = (a.mode == ATTN_DENSE) ? 0 : min(max(v.keep_cnt[s], 0), a.n_chunks);
-  const int raw0 = (a.mode == ATTN_DENSE) ? 0 : a.n_chunks * v.C;
-  const int n_lead = (a.mode == ATTN_RAW) ? M * v.C : M;
-  const int n_tail = max(0, n - raw0);
-  const int n_rows = n_tail + n_lead;
-  int n_splits = max(1, (n_rows + a.rows_per_split - 1) / a.rows_per_split);
-  // the sequence has outgrown what this launch was sized for (a replayed launch): rows beyond the grid
-  // are dropped, which the status word reports; the splits that exist still merge, so the ticket
-  // counter returns to zero and a later, correctly sized launch starts clean
-  if (n_splits > (int)gridDim.x) {
-    if (split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
-    n_splits = (int)gridDim.x;
+  if (warp == AT_PRODUCER) {
+    // where this CTA starts follows from the launch arguments alone: warm L2 with what the first look-ups need
+    // while the barriers are set up and the predecessor drains (prefetches return nothing, so they may run early)
+    const uint32_t I = (uint32_t)v.S * (uint32_t)a.k, P = min(gridDim.x, I);
+    if (blockIdx.x < P) prefetch_sequence_metadata(a, (int)(piece_begin(blockIdx.x, I, P) / (uint32_t)a.k), lane);
+    if (lane == 31) prefetch_l2(v.seq_len);
   }
-  if (split >= n_splits) return;
-  const int r_begin = split * a.rows_per_split;
-  const int r_end = min(n_rows, r_begin + a.rows_per_split);
-  const int n_tiles = (max(r_end - r_begin, 0) + AT_TILE - 1) / AT_TILE;
-
   if (threadIdx.x == 0) {
     for (int i = 0; i < AT_STAGES; ++i) {
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], AT_CWARPS);
     }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ffull[i], AT_CWARPS);
+      mbar_init(&fempty[i], 1);
+    }
     mbar_fence_init();
   }
   __syncthreads();
+  pdl_wait();      // lengths, keep lists, summaries and the new token come from earlier kernels
 
-  if (warp == AT_CWARPS) {
+  // ---- geometry (every thread) ---------------------------------------------------------------------------
+  AttnGeo g;
+  {
+    int n = v.seq_len[0];
+    n = min(max(n, 0), v.max_tokens);
+    g.raw0 = (a.mode == ATTN_DENSE) ? 0 : a.n_chunks * v.C;
+    g.n_tail = max(0, n - g.raw0);
+    g.TT = (g.n_tail + AT_TILE - 1) / AT_TILE;
+    g.per = (a.mode == ATTN_RAW) ? v.C : 1;
+    g.I = (uint32_t)v.S * (uint32_t)a.k;
+    g.P = min(gridDim.x, g.I);
+  }
+  const uint32_t c = blockIdx.x, uk = (uint32_t)a.k;
+  const uint32_t i0 = piece_begin(c, g.I, g.P), i1 = piece_begin(c + 1, g.I, g.P);      // this CTA's parts
+
+  if (warp == AT_PRODUCER) {
     // ================= producer warp =================
-    // Row addresses need up to two dependent global loads (keep list, page table).  They are resolved
-    // AT_STAGES tiles ahead of the copies, each tile in a slot of its own, so the look-ups of several
-    // tiles are in flight together and never sit between a freed stage and its refill.
+    // walks the CTA's parts in order, sequence by sequence; within a sequence the tiles [j_lo, j_hi) that
+    // its parts in this CTA cover (part p of a sequence with T tiles: tiles [p T / k, (p + 1) T / k))
+    const int s_first = (int)(i0 / uk), s_last = (int)((i1 - 1u) / uk);      // meaningful when i0 < i1
+    int s = s_first, j = 0, j_hi = 0, lt_rows = 0, tiles = 0;
+    bool fresh = true;                      // the next tile is the first one of sequence s in this CTA
+    auto enter_sequence = [&]() {
+      if (s < s_last) prefetch_sequence_metadata(a, s + 1, lane);      // the next one's look-ups will hit L2
+      lt_rows = lead_rows_of(a, g, s);
+      tiles = g.TT + (lt_rows + AT_TILE - 1) / AT_TILE;
+      // part p of the sequence's tiles: [p tiles / k, (p + 1) tiles / k); p <= 32 and tiles < 2^20, so 32 bits do
+      const uint32_t p_lo = (s == s_first) ? i0 - (uint32_t)s * uk : 0u;
+      const uint32_t p_hi = (s == s_last) ? i1 - (uint32_t)s * uk : uk;
+      j = (int)((p_lo * (uint32_t)tiles) / uk);
+      j_hi = (int)((p_hi * (uint32_t)tiles) / uk);
+      fresh = true;
+    };
+    bool done = i0 >= i1;
+    if (!done) enter_sequence();
+    auto next_tile = [&](TileDesc& t) {
+      if (done) {
+        t.s = -1; t.list = 0; t.j = 0; t.rows = 0; t.flags = TF_END;
+        return;
+      }
+      t.s = s;
+      if (j >= j_hi) {
+        // parts without a tile (fewer tiles than parts, or a sequence without a retained row): an empty tile keeps
+        // the bookkeeping uniform - the merger still gets this CTA's (empty) share of the sequence
+        t.list = 0; t.j = 0; t.rows = 0;
+        t.flags = TF_NEW | TF_FLUSH;
+      } else {
+        t.list = j >= g.TT ? 1 : 0;
+        t.j = t.list ? j - g.TT : j;
+        t.rows = min(AT_TILE, (t.list ? lt_rows : g.n_tail) - t.j * AT_TILE);
+        t.flags = (fresh ? TF_NEW : 0) | (j + 1 >= j_hi ? TF_FLUSH : 0);
+        fresh = false;
+        ++j;
+      }
+      if (t.flags & TF_FLUSH) {
+        if (s == s_last) done = true;
+        else { ++s; enter_sequence(); }
+      }
+    };
+    // addresses of the tile's rows: lane l resolves rows l and l + 32
     struct TileAddr { const uint16_t *k[AT_TILE / 32], *v[AT_TILE / 32]; };
-    auto resolve = [&](int i, TileAddr& t) {
-      const int row0 = r_begin + i * AT_TILE;
-      const int rows_in_tile = (i < n_tiles) ? min(AT_TILE, r_end - row0) : 0;
+    auto resolve = [&](const TileDesc& t, TileAddr& ta) {
+#pragma unroll
+      for (int half = 0; half < AT_TILE / 32; ++half) ta.k[half] = ta.v[half] = nullptr;
+      if (t.flags & TF_END) return;
+      const long long sb = (long long)t.s * v.max_chunks;
 #pragma unroll
       for (int half = 0; half < AT_TILE / 32; ++half) {
         const int rl = half * 32 + lane;
-        t.k[half] = t.v[half] = nullptr;
-        if (rl < rows_in_tile) row_address(a, s, row0 + rl, n_tail, raw0, t.k[half], t.v[half]);
+        if (rl >= t.rows) continue;
+        const int L = t.j * AT_TILE + rl;              // row inside the sequence's list
+        int chunk, r;
+        if (t.list == 0) {
+          const int p = g.raw0 + L;
+          chunk = p / v.C;
+          r = p - chunk * v.C;
+        } else if (a.mode == ATTN_SUMMARY) {
+          ta.k[half] = a.kkept + (sb + L) * D;
+          ta.v[half] = a.vkept + (sb + L) * D;
+          continue;
+        } else {                                       // RAW: row r of the (L / C)-th kept chunk
+          const int ci = L / v.C;
+          r = L - ci * v.C;
+          chunk = v.keep_idx[sb + ci];
+          if (chunk < 0 || chunk >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); chunk = 0; }
+        }
+        long long page = v.page_table[sb + chunk];
+        if (page < 0 || page >= v.n_pages) { set_status(v.status, ERR_CAPACITY); page = 0; }
+        const long long off = (page * v.C + r) * D;
+        ta.k[half] = v.k_pages + off;
+        ta.v[half] = v.v_pages + off;
       }
     };
-    // waits for the stage, issues the copies of tile i from its resolved addresses; false on a timed-out wait
-    auto issue = [&](int i, const TileAddr& t) -> bool {
+    // waits for the stage, publishes the tile's description, issues its copies; false on a timed-out wait
+    auto issue = [&](int i, const TileDesc& t, const TileAddr& ta) -> bool {
       const int stage = i % AT_STAGES, round = i / AT_STAGES;
       if (round > 0 && !mbar_wait_bounded(&empty[stage], (round - 1) & 1)) {
         if (lane == 0) set_status(v.status, ERR_TIMEOUT);
         return false;
       }
-      const int row0 = r_begin + i * AT_TILE;
-      const int rows_in_tile = min(AT_TILE, r_end - row0);
-      if (lane == 0) mbar_arrive_expect_tx(&full[stage], (uint32_t)rows_in_tile * 2u * ROW_BYTES);
+      if (lane == 0) {
+        info[stage] = make_int4(t.s, t.rows, t.flags, t.list);
+        const bool with_q = (t.flags & TF_NEW) != 0;
+        const uint32_t bytes = (uint32_t)t.rows * 2u * ROW_BYTES + (with_q ? (uint32_t)ROW_BYTES : 0u);
+        mbar_arrive_expect_tx(&full[stage], bytes);      // release: the description is visible to whoever sees the phase
+        if (with_q) bulk_g2s(Qs + stage * D, a.q + (long long)t.s * D, ROW_BYTES, &full[stage]);
+      }
       __syncwarp();
 #pragma unroll
       for (int half = 0; half < AT_TILE / 32; ++half) {
         const int rl = half * 32 + lane;
-        const bool valid = rl < rows_in_tile;
-        const uint16_t *kp = t.k[half], *vp = t.v[half];
+        const bool valid = rl < t.rows;
+        const uint16_t *kp = ta.k[half], *vp = ta.v[half];
         const unsigned long long ka = (unsigned long long)kp, va = (unsigned long long)vp;
         const unsigned long long kprev = __shfl_up_sync(0xffffffffu, ka, 1);
         const unsigned long long vprev = __shfl_up_sync(0xffffffffu, va, 1);
@@ -177,34 +288,48 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       }
       return true;
     };
-    static_assert(AT_STAGES == 3, "three slots of look-ahead");
-    TileAddr t0, t1, t2;
-    resolve(0, t0);
-    resolve(1, t1);
-    resolve(2, t2);
-    for (int i = 0; i < n_tiles; i += AT_STAGES) {
-      if (!issue(i, t0)) break;
-      resolve(i + 3, t0);
-      if (i + 1 < n_tiles) { if (!issue(i + 1, t1)) break; resolve(i + 4, t1); }
-      if (i + 2 < n_tiles) { if (!issue(i + 2, t2)) break; resolve(i + 5, t2); }
+    // The first tiles go out as soon as each is resolved; from then on the addresses of tile i + 1 are
+    // looked up before the wait for its stage, i.e. while the consumers still work on the tiles in flight.
+    // The END description takes a stage of its own (no copies): that is how the consumers learn that they are done.
+    TileDesc d;
+    TileAddr t;
+    for (int i = 0;; ++i) {
+      next_tile(d);
+      resolve(d, t);
+      if (!issue(i, d, t) || (d.flags & TF_END)) break;
     }
-  } else {
+  } else if (warp < AT_CWARPS) {
     // ================= consumer warps =================
-    float qf[4];
-    {
-      const uint2 qw = *reinterpret_cast<const uint2*>(a.q + (long long)s * D + lane * 4);
-      qf[0] = bf16lo(qw.x); qf[1] = bf16hi(qw.x); qf[2] = bf16lo(qw.y); qf[3] = bf16hi(qw.y);
-    }
     const float sl2 = a.scale * 1.44269504088896340736f;   // logits kept in log2 units
+    float qf[4] = {0.f, 0.f, 0.f, 0.f};
     float m = -INFINITY, l = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int i = 0; i < n_tiles; ++i) {
+    int n_flush = 0;
+    for (int i = 0;; ++i) {
       const int stage = i % AT_STAGES, round = i / AT_STAGES;
       if (!mbar_wait_bounded(&full[stage], round & 1)) {
         if (lane == 0) set_status(v.status, ERR_TIMEOUT);
         break;
       }
-      const int rows_in_tile = min(AT_TILE, r_end - (r_begin + i * AT_TILE));
-      const int nvalid = min(max(rows_in_tile - warp * AT_SUB, 0), AT_SUB);
+      const int4 ti = info[stage];                 // (sequence, rows, flags, list)
+      if (ti.z & TF_END) {
+        // tell the merger that nothing more comes
+        const int fb = n_flush & 1;
+        if (n_flush >= 2 && !mbar_wait_bounded(&fempty[fb], ((n_flush >> 1) - 1) & 1)) {
+          if (lane == 0) set_status(v.status, ERR_TIMEOUT);
+          break;
+        }
+        if (warp == 0 && lane == 0) finfo[fb] = make_int4(-1, 0, 0, 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ffull[fb]);
+        break;
+      }
+      if (ti.z & TF_NEW) {
+        const uint2 qw = *reinterpret_cast<const uint2*>(Qs + stage * D + lane * 4);
+        qf[0] = bf16lo(qw.x); qf[1] = bf16hi(qw.x); qf[2] = bf16lo(qw.y); qf[3] = bf16hi(qw.y);
+        m = -INFINITY; l = 0.f;
+        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+      }
+      const int nvalid = min(max(ti.y - warp * AT_SUB, 0), AT_SUB);
       if (nvalid > 0) {
         const uint16_t* kt = Ks + stage * AT_STAGE_ELEMS + (warp * AT_SUB) * D + lane * 4;
         const uint16_t* vt = Vs + stage * AT_STAGE_ELEMS + (warp * AT_SUB) * D + lane * 4;
@@ -244,69 +369,102 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);
+      if (ti.z & TF_FLUSH) {
+        // hand (m, l, acc) of this (sequence, list) to the merger; the exchange area is double-buffered
+        const int fb = n_flush & 1;
+        if (n_flush >= 2 && !mbar_wait_bounded(&fempty[fb], ((n_flush >> 1) - 1) & 1)) {
+          if (lane == 0) set_status(v.status, ERR_TIMEOUT);
+          break;
+        }
+        float* cw = comb + (fb * AT_CWARPS + warp) * ATTN_PARTIAL_FLOATS;
+        *reinterpret_cast<float4*>(cw + lane * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        if (lane == 0) { cw[128] = m; cw[129] = l; }
+        if (warp == 0 && lane == 0) finfo[fb] = make_int4(ti.x, ti.w, 0, 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ffull[fb]);      // release
+        ++n_flush;
+      }
     }
-    float* cw = comb + warp * ATTN_PARTIAL_FLOATS;
-    *reinterpret_cast<float4*>(cw + lane * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    if (lane == 0) { cw[128] = m; cw[129] = l; }
-  }
-  __syncthreads();
-  if (warp != 0) return;
-
-  // ---- warp 0: merge the consumer warps of this CTA ------------------------------------------------
-  float mC = -INFINITY;
+  } else {
+    // ================= merger warp =================
+    for (int f = 0;; ++f) {
+      const int fb = f & 1;
+      if (!mbar_wait_bounded(&ffull[fb], (f >> 1) & 1)) {
+        if (lane == 0) set_status(v.status, ERR_TIMEOUT);
+        break;
+      }
+      const int4 fi = finfo[fb];                   // (sequence, -, -, -); sequence < 0: no more work
+      const int s = fi.x;
+      if (s < 0) break;
+      // ---- the eight consumer states -> one ----
+      const float* cb = comb + fb * AT_CWARPS * ATTN_PARTIAL_FLOATS;
+      float mC = -INFINITY;
 #pragma unroll
-  for (int w = 0; w < AT_CWARPS; ++w) mC = fmaxf(mC, comb[w * ATTN_PARTIAL_FLOATS + 128]);
-  float lC = 0.f, accC[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int w = 0; w < AT_CWARPS; ++w) mC = fmaxf(mC, cb[w * ATTN_PARTIAL_FLOATS + 128]);
+      float lC = 0.f, accC[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int w = 0; w < AT_CWARPS; ++w) {
-    const float mw = comb[w * ATTN_PARTIAL_FLOATS + 128];
-    const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - mC);
-    lC = fmaf(comb[w * ATTN_PARTIAL_FLOATS + 129], sc, lC);
-    const float4 av = *reinterpret_cast<const float4*>(comb + w * ATTN_PARTIAL_FLOATS + lane * 4);
-    accC[0] = fmaf(av.x, sc, accC[0]); accC[1] = fmaf(av.y, sc, accC[1]);
-    accC[2] = fmaf(av.z, sc, accC[2]); accC[3] = fmaf(av.w, sc, accC[3]);
-  }
+      for (int w = 0; w < AT_CWARPS; ++w) {
+        const float mw = cb[w * ATTN_PARTIAL_FLOATS + 128];
+        const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - mC);
+        lC = fmaf(cb[w * ATTN_PARTIAL_FLOATS + 129], sc, lC);
+        const float4 av = *reinterpret_cast<const float4*>(cb + w * ATTN_PARTIAL_FLOATS + lane * 4);
+        accC[0] = fmaf(av.x, sc, accC[0]); accC[1] = fmaf(av.y, sc, accC[1]);
+        accC[2] = fmaf(av.z, sc, accC[2]); accC[3] = fmaf(av.w, sc, accC[3]);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&fempty[fb]);     // the exchange buffer may be refilled
 
-  if (n_splits > 1) {
-    float* mine = a.partials + ((long long)s * a.max_splits + split) * ATTN_PARTIAL_FLOATS;
-    *reinterpret_cast<float4*>(mine + lane * 4) = make_float4(accC[0], accC[1], accC[2], accC[3]);
-    if (lane == 0) { mine[128] = mC; mine[129] = lC; }
-    __threadfence();
-    __syncwarp();
-    int ticket = 0;
-    if (lane == 0) ticket = atomicAdd(a.counters + s, 1);
-    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (ticket != n_splits - 1) return;      // somebody else finishes later and merges
-    __threadfence();
-    const float* base = a.partials + (long long)s * a.max_splits * ATTN_PARTIAL_FLOATS;
-    mC = -INFINITY;
-    for (int sp = 0; sp < n_splits; ++sp) mC = fmaxf(mC, __ldcg(base + sp * ATTN_PARTIAL_FLOATS + 128));
-    lC = 0.f;
-    accC[0] = accC[1] = accC[2] = accC[3] = 0.f;
-    for (int sp = 0; sp < n_splits; ++sp) {
-      const float* ps = base + sp * ATTN_PARTIAL_FLOATS;
-      const float mw = __ldcg(ps + 128);
-      const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - mC);
-      lC = fmaf(__ldcg(ps + 129), sc, lC);
-      const float4 av = __ldcg(reinterpret_cast<const float4*>(ps + lane * 4));
-      accC[0] = fmaf(av.x, sc, accC[0]); accC[1] = fmaf(av.y, sc, accC[1]);
-      accC[2] = fmaf(av.z, sc, accC[2]); accC[3] = fmaf(av.w, sc, accC[3]);
+      // ---- which CTAs hold parts of sequence s ----
+      const uint32_t c0 = piece_of((uint32_t)s * uk, g.I, g.P), c1 = piece_of((uint32_t)(s + 1) * uk - 1u, g.I, g.P);
+      const int n_parts = (int)(c1 - c0 + 1u);
+      if (n_parts > 1) {
+        float* mine = a.partials + (long long)(s + c) * ATTN_PARTIAL_FLOATS;
+        *reinterpret_cast<float4*>(mine + lane * 4) = make_float4(accC[0], accC[1], accC[2], accC[3]);
+        if (lane == 0) { mine[128] = mC; mine[129] = lC; }
+        __threadfence();
+        __syncwarp();
+        int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(a.counters + s, 1);
+        ticket = __shfl_sync(0xffffffffu, ticket, 0);
+        if (ticket != n_parts - 1) continue;       // somebody else finishes later and merges
+        __threadfence();
+        // records of sequence s: CTAs c0 .. c1, at s + c0 .. s + c1; lanes fetch the (m, l) pairs side by side
+        const float* base = a.partials + (long long)(s + c0) * ATTN_PARTIAL_FLOATS;
+        mC = -INFINITY;
+        for (int p = lane; p < n_parts; p += 32) mC = fmaxf(mC, __ldcg(base + (long long)p * ATTN_PARTIAL_FLOATS + 128));
+        mC = warp_max(mC);
+        lC = 0.f;
+        for (int p = lane; p < n_parts; p += 32) {
+          const float mw = __ldcg(base + (long long)p * ATTN_PARTIAL_FLOATS + 128);
+          const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - mC);
+          lC = fmaf(__ldcg(base + (long long)p * ATTN_PARTIAL_FLOATS + 129), sc, lC);
+        }
+        lC = warp_sum(lC);
+        accC[0] = accC[1] = accC[2] = accC[3] = 0.f;
+#pragma unroll 4
+        for (int p = 0; p < n_parts; ++p) {
+          const float* ps = base + (long long)p * ATTN_PARTIAL_FLOATS;
+          const float mw = __ldcg(ps + 128);
+          const float4 av = __ldcg(reinterpret_cast<const float4*>(ps + lane * 4));
+          const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - mC);
+          accC[0] = fmaf(av.x, sc, accC[0]); accC[1] = fmaf(av.y, sc, accC[1]);
+          accC[2] = fmaf(av.z, sc, accC[2]); accC[3] = fmaf(av.w, sc, accC[3]);
+        }
+        if (lane == 0) a.counters[s] = 0;          // leave the ticket counter clean for the next launch
+      }
+      const float inv = (lC > 0.f) ? (1.f / lC) : 0.f;
+      uint2 o;
+      o.x = pack_bf16x2(accC[0] * inv, accC[1] * inv);
+      o.y = pack_bf16x2(accC[2] * inv, accC[3] * inv);
+      *reinterpret_cast<uint2*>(a.out + (long long)s * D + lane * 4) = o;
+      if (a.lse && lane == 0) a.lse[s] = (lC > 0.f) ? (mC + log2f(lC)) * 0.69314718055994530942f : -INFINITY;
     }
-    if (lane == 0) a.counters[s] = 0;        // leave the ticket counter clean for the next launch
   }
-
-  const float inv = (lC > 0.f) ? (1.f / lC) : 0.f;
-  uint2 o;
-  o.x = pack_bf16x2(accC[0] * inv, accC[1] * inv);
-  o.y = pack_bf16x2(accC[2] * inv, accC[3] * inv);
-  *reinterpret_cast<uint2*>(a.out + (long long)s * D + lane * 4) = o;
-  if (a.lse && lane == 0) a.lse[s] = (lC > 0.f) ? (mC + log2f(lC)) * 0.69314718055994530942f : -INFINITY;
 }
 
-cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_tokens_upper, AttnPlan plan,
-                        const void* q, void* out, float* lse, float scale, float* partials, int32_t* counters,
+cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int parts_per_seq, int grid, const void* q, void* out,
+                        float* lse, float scale, const void* kkept, const void* vkept, float* partials, int32_t* counters,
                         cudaStream_t st) {
-  (void)n_tokens_upper;
   if (v.S <= 0) return cudaSuccess;
   static DeviceFlags opted;
   {
@@ -314,12 +472,11 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_t
     if (e != cudaSuccess) return e;
   }
   AttnArgs a;
-  a.v = v; a.mode = (int)mode; a.n_chunks = n_chunks;
-  a.rows_per_split = plan.rows_per_split; a.max_splits = plan.max_splits;
+  a.v = v; a.mode = (int)mode; a.n_chunks = n_chunks; a.k = parts_per_seq < 1 ? 1 : parts_per_seq;
   a.q = static_cast<const uint16_t*>(q); a.out = static_cast<uint16_t*>(out); a.lse = lse; a.scale = scale;
+  a.kkept = static_cast<const uint16_t*>(kkept); a.vkept = static_cast<const uint16_t*>(vkept);
   a.partials = partials; a.counters = counters;
-  dim3 grid((unsigned)plan.max_splits, (unsigned)v.S);
-  return launch_pdl(kve_decode_attn_kernel, grid, dim3(AT_THREADS), AT_SMEM_BYTES, st, a);
+  return launch_pdl(kve_decode_attn_kernel, dim3((unsigned)(grid < 1 ? 1 : grid)), dim3(AT_THREADS), AT_SMEM_BYTES, st, a);
 }
 
 }  // namespace kve

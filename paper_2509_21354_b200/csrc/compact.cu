@@ -28,8 +28,56 @@ __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_kernel(LayerVi
   if (lane == 0) v.keep_cnt[s] = base;
 }
 
-cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStream_t st) {
-  return launch_pdl(kve_compact_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), 0, st, v, n_chunks, tau);
+// ---- what attention wants from a fresh keep list ---------------------------------------------------------
+// The kept chunks' summary rows, copied into one contiguous run per sequence ("compacted chunk tokens",
+// Sec. 3.3): attention then fetches a sequence's kept rows with one bulk copy per 64 rows instead of one
+// per row, on every decode step until the next trigger.  One warp moves 8 kept rows: lanes 0-15 the K
+// row, lanes 16-31 the V row, 16 bytes each, all 8 loads in flight.
+constexpr int GATHER_ROWS = 8;
+
+__global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_keep_gather_kernel(LayerView v, int n_chunks, int groups,
+                                                                            uint4* __restrict__ kkept, uint4* __restrict__ vkept) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long unit = (long long)blockIdx.x * COMPACT_WARPS + warp;
+  const int s = (int)(unit / groups), gi = (int)(unit - (long long)s * groups);
+  if (s >= v.S) return;
+  const int M = min(max(v.keep_cnt[s], 0), n_chunks);
+  const int i0 = gi * GATHER_ROWS;
+  if (i0 >= M) return;
+  const long long sb = (long long)s * v.max_chunks;
+  const int is_v = lane >> 4, l16 = lane & 15;
+  const uint4* src = reinterpret_cast<const uint4*>(is_v ? v.vsum_bf16 : v.ksum_bf16);
+  uint4* dst = is_v ? vkept : kkept;
+  int t[GATHER_ROWS];
+#pragma unroll
+  for (int r = 0; r < GATHER_ROWS; ++r) {
+    t[r] = (i0 + r < M) ? v.keep_idx[sb + i0 + r] : -1;
+    if (t[r] >= n_chunks) { set_status(v.status, ERR_CAPACITY); t[r] = -1; }
+  }
+  uint4 w[GATHER_ROWS];
+#pragma unroll
+  for (int r = 0; r < GATHER_ROWS; ++r)
+    if (t[r] >= 0) w[r] = __ldg(src + (sb + t[r]) * 16 + l16);
+#pragma unroll
+  for (int r = 0; r < GATHER_ROWS; ++r)
+    if (t[r] >= 0) dst[(sb + i0 + r) * 16 + l16] = w[r];
+}
+
+// after either retention rule: the kept rows, compacted
+static cudaError_t launch_keep_gather(const LayerView& v, int n_chunks, void* kkept, void* vkept, cudaStream_t st) {
+  if (n_chunks <= 0) return cudaSuccess;
+  const int groups = (n_chunks + GATHER_ROWS - 1) / GATHER_ROWS;
+  const long long units = (long long)v.S * groups;
+  return launch_pdl(kve_keep_gather_kernel, dim3((unsigned)((units + COMPACT_WARPS - 1) / COMPACT_WARPS)), dim3(COMPACT_WARPS * 32), 0, st,
+                    v, n_chunks, groups, static_cast<uint4*>(kkept), static_cast<uint4*>(vkept));
+}
+
+cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, void* kkept, void* vkept, cudaStream_t st) {
+  cudaError_t e = launch_pdl(kve_compact_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), 0, st, v,
+                             n_chunks, tau);
+  return e == cudaSuccess ? launch_keep_gather(v, n_chunks, kkept, vkept, st) : e;
 }
 
 // ---- kvE_compact_topk kernel: keep the k highest-scoring chunks of every sequence --------------------------
@@ -72,11 +120,12 @@ __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_topk_kernel(La
   if (lane == 0) v.keep_cnt[s] = base;
 }
 
-cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, cudaStream_t st) {
+cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, void* kkept, void* vkept, cudaStream_t st) {
   if (n_chunks > TOPK_MAX_CHUNKS) return cudaErrorInvalidValue;
   const size_t smem = sizeof(float) * (size_t)COMPACT_WARPS * (n_chunks > 0 ? n_chunks : 1);
-  return launch_pdl(kve_compact_topk_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), smem, st, v,
-                    n_chunks, k);
+  cudaError_t e = launch_pdl(kve_compact_topk_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), smem, st,
+                             v, n_chunks, k);
+  return e == cudaSuccess ? launch_keep_gather(v, n_chunks, kkept, vkept, st) : e;
 }
 
 // ---- kvE_reclaim_pages kernels (Sec. 3.3, memory ratio n / (W + M)): pages of gated chunks go back to the caller ----

@@ -54,7 +54,7 @@ struct MlpWeights {
 
 enum AttnMode { ATTN_SUMMARY = 0, ATTN_RAW = 1, ATTN_DENSE = 2 };
 
-// attention split geometry chosen on the host
+// split geometry of the block-of-queries attention, chosen on the host
 struct AttnPlan {
   int rows_per_split;   // multiple of the kernel's tile height
   int max_splits;       // grid.x: upper bound of splits any sequence can need
@@ -72,12 +72,16 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
                              const float* b_hh, int d_g, float* P, cudaStream_t st);
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
                             int d_g, float* P, bool reset_state, cudaStream_t st);
-cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, cudaStream_t st);
-cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, cudaStream_t st);
+// both also leave the kept chunks' summary rows compacted in kkept / vkept [S][max_chunks][128] bf16, which is
+// what attention reads until the next keep list
+cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, void* kkept, void* vkept, cudaStream_t st);
+cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, void* kkept, void* vkept, cudaStream_t st);
 cudaError_t launch_reclaim(const LayerView& v, int t0, int t1, float tau, int mode, int32_t* scratch, int32_t* free_list,
                            long long capacity, int32_t* free_count, cudaStream_t st);
-cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int n_tokens_upper, AttnPlan plan,
-                        const void* q, void* out, float* lse, float scale, float* partials, int32_t* counters,
+// parts_per_seq: equal parts every sequence is cut into; grid: CTAs that share the S * parts_per_seq parts;
+// partials: S + grid records of ATTN_PARTIAL_FLOATS
+cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int parts_per_seq, int grid, const void* q, void* out,
+                        float* lse, float scale, const void* kkept, const void* vkept, float* partials, int32_t* counters,
                         cudaStream_t st);
 int attn_smem_bytes();
 

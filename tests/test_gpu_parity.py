@@ -269,7 +269,7 @@ def test_set_len_below_the_compacted_range_drops_the_keep_list():
         out = fn(0, b.bits_to_bf16(q))
         torch.cuda.synchronize()
         assert st.poll_status() == 0
-        want, _, _ = pb.oracle_dense(q, "f64", pb.K[:, :-1], pb.V[:, :-1])
+        want, _, _ = pb.oracle_dense(q, "f64", np.ascontiguousarray(pb.K[:, :-1]), np.ascontiguousarray(pb.V[:, :-1]))
         hz.check_output(b.bf16_to_bits(out), want, "attention after roll-back")
     # gating and compacting again brings the gated path back
     st.append(0, b.bits_to_bf16(pb.K[:, -1:]), b.bits_to_bf16(pb.V[:, -1:]))
@@ -670,24 +670,35 @@ def test_decode_loop_advances_under_a_cuda_graph():
     st.gate(0, pb.Nc, nc, lw)
     torch.cuda.synchronize()
     assert st.poll_status() == 0
-    # a replay beyond the reserved growth is reported, not silently truncated
+    # a single-query attention launch is cut into pieces on the device from the length it finds there, so a replay far
+    # beyond the growth that was announced (n_reserve = 0) still attends to every row
     wl2 = wlm.CFG1.small(B=1, H=2, n=300, C=64, W=64, seed=44, n_append=400)
     st2 = make_store(wl2)
     pb2 = hz.Problem(wl2)
     load_kv(st2, 0, pb2.K, pb2.V)
     run_gpu_pipeline(st2, pb2, 0, None, b.LstmWeights(pb2.lstm))
     z = torch.zeros((st2.S, 128), dtype=torch.bfloat16, device="cuda")
+    q2 = wlm.gen_q(wl2, 0, 9)
+    q2d, out2 = b.bits_to_bf16(q2), torch.empty_like(z)
     g2 = torch.cuda.CUDAGraph()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         with torch.cuda.graph(g2, stream=side):
             st2.append_next(0, z, z, n_reserve=0)
-            st2.decode_attn(0, z, torch.empty_like(z))
+            st2.decode_attn(0, q2d, out2)
     torch.cuda.current_stream().wait_stream(side)
-    for _ in range(200):                                           # far past the tile the launch was sized for
+    for _ in range(200):
         g2.replay()
     torch.cuda.synchronize()
-    assert st2.poll_status() == -3
+    assert st2.poll_status() == 0 and int(st2.seq_len[0, 0]) == wl2.n + 200
+    pad = np.zeros((st2.S, 200, 128), np.uint16)
+    want, _, _, _ = pb2.oracle_attn(q2, "summary", "f64", np.concatenate([pb2.K, pad], axis=1), np.concatenate([pb2.V, pad], axis=1), pb2.Nc)
+    hz.check_output(b.bf16_to_bits(out2), want, "replayed 200 tokens past the announced growth")
+    # the cache is full after 400 appended tokens: further replays are refused on the device, nothing is overwritten
+    for _ in range(201):
+        g2.replay()
+    torch.cuda.synchronize()
+    assert st2.poll_status() == -3 and int(st2.seq_len[0, 0]) == wl2.n + 400
 
 
 @pytest.mark.parametrize("seed", list(range(12)) + [104])      # 104: nothing has left the window yet
