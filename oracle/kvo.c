@@ -40,6 +40,7 @@ typedef KVO_REAL real;
 #define KVO_AGG_MLP 1
 #define KVO_AGG_IDENTITY 2
 #define KVO_AGG_MAX 3
+#define KVO_AGG_TOKEN_MLP 4
 #define KVO_ATTEND_SUMMARY 0
 #define KVO_ATTEND_RAW 1
 
@@ -112,6 +113,8 @@ static void mlp2(const real* m, int d, int d_sum, const float* W1, const float* 
  *             MLP : Kbar = MLP_K(mean), Vbar = MLP_V(mean)  (2 layers, hidden d_sum, erf-GELU)
  *             IDENTITY (C == 1 only): Kbar = k
  *             MAX : Kbar = element-wise maximum of the chunk's keys ("pooling", Sec. 3.1), Vbar likewise
+ *             TOKEN_MLP: Eq. 2 taken literally, the MLP acting on every element of the set {k_j}:
+ *                   y_j = MLP_K(k_j) for each of the C tokens, Kbar = (1/C) sum_j y_j  (mean-pool of the outputs)
  * outputs     ksum, vsum [S][stride][d] real at row t; *_b16 the same values rounded to bf16
  * returns 0, or -1 on a bad argument
  */
@@ -123,15 +126,20 @@ int kvo_summarize(const uint16_t* K, const uint16_t* V, int S, int n, int d, int
   if (S < 0 || n < 0 || d <= 0 || C <= 0 || t0 < 0 || t1 < t0 || (long)t1 * C > n || t1 > stride)
     return -1;
   if (agg == KVO_AGG_IDENTITY && C != 1) return -1;
-  if (agg == KVO_AGG_MLP && (d_sum <= 0 || !W1K || !b1K || !W2K || !b2K || !W1V || !b1V || !W2V || !b2V))
+  if ((agg == KVO_AGG_MLP || agg == KVO_AGG_TOKEN_MLP) &&
+      (d_sum <= 0 || !W1K || !b1K || !W2K || !b2K || !W1V || !b1V || !W2V || !b2V))
     return -1;
-  if (agg != KVO_AGG_MEAN && agg != KVO_AGG_MLP && agg != KVO_AGG_IDENTITY && agg != KVO_AGG_MAX) return -1;
+  if (agg != KVO_AGG_MEAN && agg != KVO_AGG_MLP && agg != KVO_AGG_IDENTITY && agg != KVO_AGG_MAX &&
+      agg != KVO_AGG_TOKEN_MLP)
+    return -1;
 #pragma omp parallel for schedule(static)
   for (int s = 0; s < S; ++s) {
     real* mk = (real*)malloc(sizeof(real) * (size_t)d);
     real* mv = (real*)malloc(sizeof(real) * (size_t)d);
     real* yk = (real*)malloc(sizeof(real) * (size_t)d);
     real* yv = (real*)malloc(sizeof(real) * (size_t)d);
+    real* tk = (real*)malloc(sizeof(real) * (size_t)d);
+    real* tv = (real*)malloc(sizeof(real) * (size_t)d);
     real* hid = (real*)malloc(sizeof(real) * (size_t)(d_sum > 0 ? d_sum : 1));
     for (int t = t0; t < t1; ++t) {
       for (int x = 0; x < d; ++x) {
@@ -162,6 +170,28 @@ int kvo_summarize(const uint16_t* K, const uint16_t* V, int S, int n, int d, int
         ok = yk;
         ov = yv;
       }
+      if (agg == KVO_AGG_TOKEN_MLP) {      /* the MLP on each token, then the mean of the C outputs */
+        for (int x = 0; x < d; ++x) yk[x] = yv[x] = 0;
+        for (int j = 0; j < C; ++j) {
+          size_t row = ((size_t)s * n + (size_t)t * C + j) * d;
+          for (int x = 0; x < d; ++x) {      /* the token itself (mk, mv reused as the MLP input) */
+            mk[x] = bf16_to_real(K[row + x]);
+            mv[x] = bf16_to_real(V[row + x]);
+          }
+          mlp2(mk, d, d_sum, W1K, b1K, W2K, b2K, hid, tk);
+          mlp2(mv, d, d_sum, W1V, b1V, W2V, b2V, hid, tv);
+          for (int x = 0; x < d; ++x) {
+            yk[x] += tk[x];
+            yv[x] += tv[x];
+          }
+        }
+        for (int x = 0; x < d; ++x) {
+          yk[x] = yk[x] / (real)C;
+          yv[x] = yv[x] / (real)C;
+        }
+        ok = yk;
+        ov = yv;
+      }
       size_t o = ((size_t)s * stride + t) * d;
       for (int x = 0; x < d; ++x) {
         ksum[o + x] = ok[x];
@@ -170,7 +200,7 @@ int kvo_summarize(const uint16_t* K, const uint16_t* V, int S, int n, int d, int
         vsum_b16[o + x] = real_to_bf16(ov[x]);
       }
     }
-    free(mk); free(mv); free(yk); free(yv); free(hid);
+    free(mk); free(mv); free(yk); free(yv); free(tk); free(tv); free(hid);
   }
   return 0;
 }

@@ -11,7 +11,7 @@ import numpy as np
 
 from . import build as _build
 
-AGG_MEAN, AGG_MLP, AGG_IDENTITY, AGG_MAX = 0, 1, 2, 3
+AGG_MEAN, AGG_MLP, AGG_IDENTITY, AGG_MAX, AGG_TOKEN_MLP = 0, 1, 2, 3, 4
 ATTEND_SUMMARY, ATTEND_RAW = 0, 1
 
 _u16p = C.POINTER(C.c_uint16)
@@ -64,7 +64,7 @@ class Oracle:
                        ksum_b16=np.zeros((S, stride, d), np.uint16), vsum_b16=np.zeros((S, stride, d), np.uint16))
         w = {}
         d_sum = 0
-        if agg == AGG_MLP:
+        if agg in (AGG_MLP, AGG_TOKEN_MLP):
             d_sum = mlp["W1K"].shape[0]
             for k in ("W1K", "b1K", "W2K", "b2K", "W1V", "b1V", "W2V", "b2V"):
                 w[k] = np.ascontiguousarray(mlp[k], np.float32)

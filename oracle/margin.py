@@ -13,7 +13,8 @@ from paper_2509_21354_b200 import workloads as wlm
 
 from . import kvo
 
-AGG_CODE = {"mean": kvo.AGG_MEAN, "mlp": kvo.AGG_MLP, "identity": kvo.AGG_IDENTITY, "max": kvo.AGG_MAX}
+AGG_CODE = {"mean": kvo.AGG_MEAN, "mlp": kvo.AGG_MLP, "identity": kvo.AGG_IDENTITY, "max": kvo.AGG_MAX,
+            "token_mlp": kvo.AGG_TOKEN_MLP}
 
 
 def centred_b_s(o: kvo.Oracle, wl: wlm.Workload, K, V, mlp, lstm, keep=0.5, n_chunks=None):

@@ -31,6 +31,22 @@
 
 namespace kve {
 
+// Optional per-CTA time stamps (build with -DKVE_ATTN_STAMPS, see attn_stamps.py): where a launch's time goes.
+// Slots: 0 kernel entry, 1 after the wait for the predecessor, 2 first copy issued, 3 first tile landed,
+// 4 last tile consumed, 5 merger warp done, 6 producer warp done.  Compiled out of the product library.
+#ifdef KVE_ATTN_STAMPS
+constexpr int STAMP_CTAS = 2048, STAMP_SLOTS = 8;
+__device__ unsigned long long g_attn_stamps[STAMP_CTAS * STAMP_SLOTS];
+__device__ __forceinline__ void stamp(int slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  if (blockIdx.x < STAMP_CTAS) g_attn_stamps[blockIdx.x * STAMP_SLOTS + slot] = t;
+}
+#define KVE_STAMP(cond, slot) do { if (cond) stamp(slot); } while (0)
+#else
+#define KVE_STAMP(cond, slot) do { } while (0)
+#endif
+
 constexpr int AT_TILE = ATTN_TILE_ROWS;       // rows per stage
 constexpr int AT_STAGES = 3;
 constexpr int AT_CWARPS = 8;                  // consumer warps
@@ -137,6 +153,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   pdl_launch_dependents();
   const LayerView& v = a.v;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  KVE_STAMP(threadIdx.x == 0, 0);
   if (warp == AT_PRODUCER) {
     // where this CTA starts follows from the launch arguments alone: warm L2 with what the first look-ups need
     // while the barriers are set up and the predecessor drains (prefetches return nothing, so they may run early)
@@ -157,6 +174,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   }
   __syncthreads();
   pdl_wait();      // lengths, keep lists, summaries and the new token come from earlier kernels
+  KVE_STAMP(threadIdx.x == 0, 1);
 
   // ---- geometry (every thread) ---------------------------------------------------------------------------
   AttnGeo g;
@@ -297,7 +315,9 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       next_tile(d);
       resolve(d, t);
       if (!issue(i, d, t) || (d.flags & TF_END)) break;
+      KVE_STAMP(i == 0 && lane == 0, 2);
     }
+    KVE_STAMP(lane == 0, 6);
   } else if (warp < AT_CWARPS) {
     // ================= consumer warps =================
     const float sl2 = a.scale * 1.44269504088896340736f;   // logits kept in log2 units
@@ -311,7 +331,9 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
         break;
       }
       const int4 ti = info[stage];                 // (sequence, rows, flags, list)
+      KVE_STAMP(i == 0 && warp == 0 && lane == 0, 3);
       if (ti.z & TF_END) {
+        KVE_STAMP(warp == 0 && lane == 0, 4);
         // tell the merger that nothing more comes
         const int fb = n_flush & 1;
         if (n_flush >= 2 && !mbar_wait_bounded(&fempty[fb], ((n_flush >> 1) - 1) & 1)) {
@@ -459,6 +481,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       *reinterpret_cast<uint2*>(a.out + (long long)s * D + lane * 4) = o;
       if (a.lse && lane == 0) a.lse[s] = (lC > 0.f) ? (mC + log2f(lC)) * 0.69314718055994530942f : -INFINITY;
     }
+    KVE_STAMP(lane == 0, 5);
   }
 }
 
@@ -480,3 +503,16 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int par
 }
 
 }  // namespace kve
+
+#ifdef KVE_ATTN_STAMPS
+// instrumented build only: copy the stamps of the last launch to the host / clear them
+extern "C" int kve_attn_stamps_read(unsigned long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, kve::g_attn_stamps, sizeof(unsigned long long) * n);
+}
+extern "C" int kve_attn_stamps_clear() {
+  void* p = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&p, kve::g_attn_stamps);
+  if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(kve::g_attn_stamps));
+  return (int)e;
+}
+#endif

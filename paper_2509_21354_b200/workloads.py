@@ -44,7 +44,7 @@ class Workload:
     C: int                 # chunk size
     W: int                 # recent window kept raw
     d_g: int               # LSTM hidden size
-    agg: str = "mean"      # "mean" | "mlp" | "identity"
+    agg: str = "mean"      # "mean" | "mlp" | "identity" | "max" | "token_mlp"
     d_sum: int = 0         # MLP hidden size (agg == "mlp")
     n_layers: int = 1
     tau: float = 0.5
@@ -166,7 +166,7 @@ def gen_new_tokens(wl: Workload, layer: int = 0, step: int = 0, n_new: int = 1):
 def gen_mlp_weights(wl: Workload, layer: int = 0):
     """Aggregator weights, N(0, 1/fan_in) entries rounded to bf16-representable float32; small N(0, BIAS_STD^2) biases
     so that a dropped bias term shows up in parity."""
-    if wl.agg != "mlp":
+    if wl.agg not in ("mlp", "token_mlp"):
         return None
     rng = _rng(wl.seed, _TAG_MLP, layer)
     d, ds = wl.d, wl.d_sum

@@ -213,6 +213,50 @@ def test_summary_mlp_matches_torch_modules(o64):
     assert np.array_equal(r["ksum_b16"], np.vectorize(o64.bf16_rne, otypes=[np.uint16])(r["ksum"]))
 
 
+def test_summary_token_mlp_hand_worked(o64, o32):
+    """Eq. 2 with the MLP on every token, then the mean: differs from mean-then-MLP on the same numbers."""
+    g = read_golden("token_mlp_2x2.txt")
+    K = bits(np.array([[[1, 3], [1, -1]]], np.float32))
+    V = np.zeros((1, 2, 2), np.uint16)
+    mlp = dict(W1K=np.array([[1, 0], [0, -1]], np.float32), b1K=np.zeros(2, np.float32),
+               W2K=np.array([[1, 1], [2, 0]], np.float32), b2K=np.array([0.5, 0], np.float32),
+               W1V=np.array([[3, 1], [1, 2]], np.float32), b1V=np.zeros(2, np.float32),
+               W2V=np.array([[5, 7], [1, 1]], np.float32), b2V=np.array([0.25, -0.75], np.float32))
+    for o, tol in ((o64, 1e-14), (o32, 3e-7)):
+        r = o.summarize(K, V, 2, 0, 1, kvo.AGG_TOKEN_MLP, mlp)
+        assert np.allclose(r["ksum"][0, 0], g["kbar"], atol=tol)
+        assert np.allclose(r["vsum"][0, 0], g["vbar"], atol=tol)
+    other = read_golden("mlp_2x2.txt")
+    assert abs(g["kbar"][0] - other["kbar"][0]) > 0.5          # the two readings of Eq. 2 give different numbers here
+
+
+def test_summary_token_mlp_matches_torch_modules_and_special_cases(o64):
+    wl = wlm.Workload("t", B=1, H=2, n=24, C=4, W=8, d_g=8, agg="token_mlp", d_sum=6, d=8)
+    K, V = wlm.gen_kv(wl)
+    mlp = wlm.gen_mlp_weights(wl)
+    r = o64.summarize(K, V, wl.C, 0, 4, kvo.AGG_TOKEN_MLP, mlp)
+    gelu = torch.nn.GELU(approximate="none")
+    for side, X, got in (("K", K, r["ksum"]), ("V", V, r["vsum"])):
+        x = torch.from_numpy(widen(X))[:, :16].reshape(2, 4, 4, 8)                     # [S, chunk, token, d]
+        W1, b1, W2, b2 = (torch.from_numpy(mlp[k + side]).double() for k in ("W1", "b1", "W2", "b2"))
+        per_token = torch.nn.functional.linear(gelu(torch.nn.functional.linear(x, W1, b1)), W2, b2)
+        assert np.allclose(got, per_token.mean(dim=2).numpy(), atol=1e-14)
+        # the last layer is affine and the mean is linear: pooling the activations first gives the same vector
+        pooled = gelu(torch.nn.functional.linear(x, W1, b1)).mean(dim=2)
+        assert np.allclose(got, torch.nn.functional.linear(pooled, W2, b2).numpy(), atol=1e-13)
+    # chunks of one token: nothing to pool, so both readings of Eq. 2 coincide
+    a = o64.summarize(K, V, 1, 0, 24, kvo.AGG_TOKEN_MLP, mlp)
+    b_ = o64.summarize(K, V, 1, 0, 24, kvo.AGG_MLP, mlp)
+    assert np.allclose(a["ksum"], b_["ksum"], atol=1e-15) and np.allclose(a["vsum"], b_["vsum"], atol=1e-15)
+    # a chunk of identical tokens: the mean of equal outputs is that output = the MLP of the (equal) mean
+    Kc = np.repeat(K[:, :1], 4, axis=1)
+    Vc = np.repeat(V[:, :1], 4, axis=1)
+    a = o64.summarize(Kc, Vc, 4, 0, 1, kvo.AGG_TOKEN_MLP, mlp)
+    b_ = o64.summarize(Kc, Vc, 4, 0, 1, kvo.AGG_MLP, mlp)
+    assert np.allclose(a["ksum"], b_["ksum"], atol=1e-14) and np.allclose(a["vsum"], b_["vsum"], atol=1e-14)
+    assert np.array_equal(r["ksum_b16"], np.vectorize(o64.bf16_rne, otypes=[np.uint16])(r["ksum"]))
+
+
 # ---------------------------------------------------------------- Eq. 3: LSTM gate
 def small_gate_problem(seed=21, S=3, Nc=6, d=4, d_g=5):
     rng = np.random.default_rng(seed)
