@@ -555,6 +555,45 @@ def trigger_leg(wl, attend, seed, steady_ms, n_triggers=24):
             "trigger_share_of_amortised_step": trig / (wl.C * steady_ms + trig)}
 
 
+def token_mlp_leg(wl, peaks, peak_kind, flush, seed):
+    """Eq. 2 taken literally (KVE_AGG_TOKEN_MLP): the aggregator MLP on EVERY stale token, outputs mean-pooled, on the
+    workload's geometry.  The first layer is a tcgen05 contraction [tokens, 128] x [128, d_sum]; the kernel is bound by
+    the activation arithmetic of its epilogue (erf GELU: about 21 FP32-pipe instructions and 2 special-function ops per
+    activation, plus the pooling shuffles), so its roofline is the FP32 issue rate: SMs x 128 lanes x clock / 21."""
+    import torch
+    d_sum = 256
+    g = wl.small(agg="token_mlp", d_sum=d_sum)
+    rig = Rig(g, "summary", seed)
+    st = rig.st
+    st.profile(True)
+    ts = []
+    for _ in range(6):
+        flush()
+        st.summarize_chunks(0, 0, rig.Nc, rig.aw)
+        ts.append(st.profile_read()["chunk_mlp"])
+    st.profile(False)
+    us = float(np.median(ts[1:]))
+    assert st.poll_status() == 0
+    tokens = g.S * rig.Nc * g.C
+    flops = 2 * tokens * 2 * 128 * d_sum + 2 * g.S * rig.Nc * 2 * d_sum * 128
+    acts = 2 * tokens * d_sum
+    kv_bytes = tokens * 512
+    sm_mhz = peaks.get("sm_max_mhz", 1965.0)
+    alu_peak = 148 * 128 * sm_mhz * 1e6 / 21.0          # activations per second if the FP32 pipe did nothing else
+    tensor_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    res = {"what": f"kvE_summarize_chunks with the per-token MLP aggregator (d_sum {d_sum}) over all {rig.Nc} stale chunks of "
+                   f"{g.S} sequences ({tokens} tokens per side), both kernels, L2 flushed",
+           "us": us, "stale_kv_bytes": kv_bytes, "GB/s": kv_bytes / us / 1e3, "frac_of_hbm_peak": kv_bytes / us / 1e3 / peaks["hbm_gbs"],
+           "flops": flops, "TFLOP/s": flops / us / 1e6, "frac_of_bf16_peak": flops / us / 1e6 / tensor_peak,
+           "activations": acts, "Gact/s": acts / us / 1e3,
+           "roofline": {"bound": "alu", "achieved": acts / us / 1e3, "peak": alu_peak / 1e9, "unit": "Gact/s",
+                        "frac": acts / us / 1e3 / (alu_peak / 1e9),
+                        "peak_kind": "derived: 148 SMs x 128 FP32 lanes x max SM clock / 21 instructions per activation"},
+           "peak_kind": f"of {peak_kind}"}
+    st.close()
+    return res
+
+
 SWEEP_GEOMETRIES = [  # (B, n, C): every corner of the grid, then a diagonal through its middle
     (1, 2048, 32), (1, 2048, 256), (1, 32768, 32), (1, 32768, 256),
     (64, 2048, 32), (64, 2048, 256), (64, 32768, 32), (64, 32768, 256),
@@ -796,6 +835,8 @@ def run_ours(args, rank, world, local_rank):
     res["per_config"] = per
     if "sweep" in legs:
         res["sweep"] = sweep_leg(peaks, peak_kind, flush, seed + 200)
+    if "token_mlp" in legs:
+        res["token_mlp_aggregator"] = token_mlp_leg(wlm.CFG2.small(n_layers=1), peaks, peak_kind, flush, seed + 300)
     if "query_block" in legs:
         res["query_block_attention"] = query_block_leg(wl, hbm, tensor_peak, peak_kind, seed + 17)
     if "tick_graph" in legs and args.tick_layers > 0:
@@ -898,7 +939,7 @@ def run_reference(args, rank):
             "gpu_launches": 0, "wall_s": wall}
 
 
-ALL_LEGS = "per_config,sweep,trigger,query_block,tick_graph,cpu"
+ALL_LEGS = "per_config,sweep,trigger,token_mlp,query_block,tick_graph,cpu"
 
 
 def main():
@@ -911,8 +952,8 @@ def main():
                     help="the configuration the headline step is timed on (default: the largest single-GPU one)")
     ap.add_argument("--attend", default="summary", choices=["summary", "raw"])
     ap.add_argument("--legs", default=ALL_LEGS,
-                    help="comma-separated extra legs of the single-GPU report (per_config, sweep, trigger, query_block, "
-                         "tick_graph, cpu); empty string: the headline only")
+                    help="comma-separated extra legs of the single-GPU report (per_config, sweep, trigger, token_mlp, "
+                         "query_block, tick_graph, cpu); empty string: the headline only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-timed-s", type=float, default=0.25,
                     help="the K-step loop is repeated until at least this much device time has been timed")

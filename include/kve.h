@@ -43,7 +43,9 @@ typedef enum {
   KVE_ERR_TIMEOUT = -6    /* a bounded device-side wait ran out (reported through status_word) */
 } kvE_status;
 
-enum { KVE_AGG_MEAN = 0, KVE_AGG_MLP = 1, KVE_AGG_IDENTITY = 2, KVE_AGG_MAX = 3 };   /* Eq. 2 aggregator; MAX = max-pool (Sec. 3.1) */
+/* Eq. 2 aggregator.  MEAN: chunk mean; MLP: 2-layer GELU MLP on the chunk mean; IDENTITY: C == 1; MAX: max-pool
+ * (Sec. 3.1); TOKEN_MLP: Eq. 2 taken literally, the MLP on every token of the chunk, the C outputs mean-pooled. */
+enum { KVE_AGG_MEAN = 0, KVE_AGG_MLP = 1, KVE_AGG_IDENTITY = 2, KVE_AGG_MAX = 3, KVE_AGG_TOKEN_MLP = 4 };
 enum { KVE_ATTEND_SUMMARY = 0, KVE_ATTEND_RAW = 1 };                /* what a kept chunk contributes */
 
 /* Geometry, fixed at kvE_create. */
@@ -57,7 +59,8 @@ typedef struct {
   int32_t max_tokens;  /* capacity of one sequence */
   int32_t n_layers;    /* independent layers sharing the handle */
   int32_t agg;         /* KVE_AGG_* ; IDENTITY needs C == 1; MAX: element-wise maximum of the chunk */
-  int32_t d_sum;       /* MLP hidden size (KVE_AGG_MLP), multiple of 8, <= 1024 */
+  int32_t d_sum;       /* MLP hidden size: KVE_AGG_MLP: multiple of 8, <= 1024; KVE_AGG_TOKEN_MLP: 128 or 256, and C
+                          must be 32, 64, 128 or a multiple of 128 */
   int32_t d_g;         /* LSTM hidden size: 64, 128 or 256 */
   int32_t attend;      /* KVE_ATTEND_* */
   int32_t max_query_tokens; /* most query tokens per kvE_decode_attn_block call; 0: that entry point is not used.
@@ -87,7 +90,8 @@ typedef struct {
   int32_t* status_word; /* one int32, zeroed by kvE_create; first device-side error sticks */
 } kvE_buffers;
 
-/* Aggregator MLP_K / MLP_V of Eq. 2 (KVE_AGG_MLP): y = W2 gelu(W1 m + b1) + b2, m the chunk mean.
+/* Aggregator MLP_K / MLP_V of Eq. 2 (KVE_AGG_MLP: y = W2 gelu(W1 m + b1) + b2, m the chunk mean; KVE_AGG_TOKEN_MLP:
+ * the same MLP applied to every token of the chunk, the outputs averaged).
  * DEVICE pointers; W1 [d_sum][d], W2 [d][d_sum] bf16; b1 [d_sum], b2 [d] fp32. */
 typedef struct {
   const void *W1K, *W2K, *W1V, *W2V;
@@ -152,7 +156,7 @@ int kvE_set_len(kvE_store* st, int layer, int n, void* stream);
 int kvE_set_attend(kvE_store* st, int attend);
 
 /* Eq. 2: summaries of chunks [chunk_begin, chunk_end) of every sequence of `layer`;
- * chunk_end <= floor((n - W) / C).  w is NULL unless agg == KVE_AGG_MLP. */
+ * chunk_end <= floor((n - W) / C).  w is NULL unless agg is KVE_AGG_MLP or KVE_AGG_TOKEN_MLP. */
 int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_end,
                          const kvE_agg_weights* w, void* stream);
 

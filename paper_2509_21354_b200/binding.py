@@ -16,7 +16,7 @@ import torch
 
 from . import build as _build
 
-AGG = {"mean": 0, "mlp": 1, "identity": 2, "max": 3}
+AGG = {"mean": 0, "mlp": 1, "identity": 2, "max": 3, "token_mlp": 4}
 ATTEND = {"summary": 0, "raw": 1}
 STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_CAPACITY",
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}

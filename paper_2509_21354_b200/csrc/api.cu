@@ -67,7 +67,9 @@ int check_config(const kvE_config* c) {
   if (!c) return KVE_ERR_ARG;
   if (c->B <= 0 || c->Hq <= 0 || c->Hkv <= 0 || c->C <= 0 || c->W < 0 || c->max_tokens <= 0 || c->n_layers <= 0)
     return KVE_ERR_ARG;
-  if (c->agg != KVE_AGG_MEAN && c->agg != KVE_AGG_MLP && c->agg != KVE_AGG_IDENTITY && c->agg != KVE_AGG_MAX) return KVE_ERR_ARG;
+  if (c->agg != KVE_AGG_MEAN && c->agg != KVE_AGG_MLP && c->agg != KVE_AGG_IDENTITY && c->agg != KVE_AGG_MAX &&
+      c->agg != KVE_AGG_TOKEN_MLP)
+    return KVE_ERR_ARG;
   if (c->attend != KVE_ATTEND_SUMMARY && c->attend != KVE_ATTEND_RAW) return KVE_ERR_ARG;
   if (c->d != 128 || c->Hq % c->Hkv != 0 || c->C > 1024) return KVE_ERR_GEOMETRY;
   if (c->max_query_tokens < 0) return KVE_ERR_ARG;
@@ -76,6 +78,7 @@ int check_config(const kvE_config* c) {
     return KVE_ERR_GEOMETRY;
   if (c->agg == KVE_AGG_IDENTITY && c->C != 1) return KVE_ERR_GEOMETRY;
   if (c->agg == KVE_AGG_MLP && (c->d_sum <= 0 || c->d_sum % 8 != 0 || c->d_sum > 1024)) return KVE_ERR_GEOMETRY;
+  if (c->agg == KVE_AGG_TOKEN_MLP && !token_mlp_supported(c->C, c->d_sum)) return KVE_ERR_GEOMETRY;
   if (c->d_g != 64 && c->d_g != 128 && c->d_g != 256) return KVE_ERR_GEOMETRY;
   if ((long long)c->B * c->Hkv > 65535) return KVE_ERR_GEOMETRY;
   return KVE_OK;
@@ -99,7 +102,11 @@ Carve carve(const kvE_config& c) {
   const size_t max_chunks = ((size_t)c.max_tokens + c.C - 1) / c.C;
   Carve k;
   size_t o = 0;
-  k.off_P = o;        o = align_up(o + S * max_chunks * 4 * (size_t)c.d_g * sizeof(float));
+  // gate projection P [S max_chunks][4 d_g]; the per-token MLP aggregator, which runs before the gate, borrows it
+  // for its pooled activations [2][S max_chunks][d_sum]
+  size_t p_floats = S * max_chunks * 4 * (size_t)c.d_g;
+  if (c.agg == KVE_AGG_TOKEN_MLP && 2 * S * max_chunks * (size_t)c.d_sum > p_floats) p_floats = 2 * S * max_chunks * (size_t)c.d_sum;
+  k.off_P = o;        o = align_up(o + p_floats * sizeof(float));
   // attention partial records: the one of (sequence s, CTA c) at s + c, at most ATTN_GRID_LIMIT CTAs
   k.off_partials = o; o = align_up(o + (S + ATTN_GRID_LIMIT) * ATTN_PARTIAL_FLOATS * sizeof(float));
   k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
@@ -368,16 +375,25 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
   if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
   if (chunk_end > stale_chunks(st->cfg, ls.n_tokens)) return KVE_ERR_STATE;   // the window is never summarised
+  const bool token_mlp = st->cfg.agg == KVE_AGG_TOKEN_MLP;
   const bool mlp = st->cfg.agg == KVE_AGG_MLP;
-  if (mlp && (!w || !w->W1K || !w->W2K || !w->W1V || !w->W2V || !w->b1K || !w->b2K || !w->b1V || !w->b2V))
+  if ((mlp || token_mlp) && (!w || !w->W1K || !w->W2K || !w->W1V || !w->W2V || !w->b1K || !w->b2K || !w->b1V || !w->b2V))
     return KVE_ERR_ARG;
   if (chunk_end == chunk_begin) return KVE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const LayerView v = view(st, layer);
-  cudaError_t e;
-  {
+  cudaError_t e = cudaSuccess;
+  if (!token_mlp) {
     Prof prof(st, KVE_K_CHUNK_MEAN, s);
     e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, st->cfg.agg == KVE_AGG_MAX, s);
+  } else {
+    Prof prof(st, KVE_K_CHUNK_MLP, s);
+    MlpWeights mw;
+    mw.W1K = static_cast<const uint16_t*>(w->W1K); mw.W2K = static_cast<const uint16_t*>(w->W2K);
+    mw.W1V = static_cast<const uint16_t*>(w->W1V); mw.W2V = static_cast<const uint16_t*>(w->W2V);
+    mw.b1K = w->b1K; mw.b2K = w->b2K; mw.b1V = w->b1V; mw.b2V = w->b2V;
+    e = launch_chunk_token_mlp(v, chunk_begin, chunk_end, mw, st->cfg.d_sum,
+                               reinterpret_cast<float*>(static_cast<char*>(st->buf.workspace) + st->off_P), s);
   }
   if (e == cudaSuccess && mlp) {
     Prof prof(st, KVE_K_CHUNK_MLP, s);

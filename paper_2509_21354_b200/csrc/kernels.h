@@ -68,6 +68,9 @@ cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void
                                cudaStream_t st);
 cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st);
 cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st);
+// per-token MLP aggregator: hid = scratch of 2 * S * (t1 - t0) * d_sum floats
+bool token_mlp_supported(int C, int d_sum);
+cudaError_t launch_chunk_token_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, float* hid, cudaStream_t st);
 cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t* W_ih, const float* b_ih,
                              const float* b_hh, int d_g, float* P, cudaStream_t st);
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,

@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.cuh"
+#include "gelu.cuh"
 
 namespace kve {
 
@@ -239,20 +240,6 @@ __device__ __forceinline__ void store_split8(const float (&x)[8], unsigned char*
   for (int pl = 0; pl < 3; ++pl)
     *reinterpret_cast<uint4*>(dst + pl * plane_stride) = make_uint4(w[0][pl], w[1][pl], w[2][pl], w[3][pl]);
 }
-
-// erf by the rational-times-exponential formula 7.1.26 of Abramowitz & Stegun (absolute error below
-// 1.5e-7, i.e. at the level of fp32 rounding of the activations), odd extension for x < 0
-__device__ __forceinline__ float erf_as(float x) {
-  const float ax = fabsf(x);
-  const float t = __fdividef(1.f, fmaf(0.3275911f, ax, 1.f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float y = 1.f - poly * t * __expf(-ax * ax);
-  return copysignf(y, x);
-}
-__device__ __forceinline__ float gelu_tc(float x) { return 0.5f * x * (1.f + erf_as(x * 0.70710678118654752440f)); }
 
 __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerView v, int t0, int n_range, long long n_units,
                                                                          MlpWeights w, int d_sum) {

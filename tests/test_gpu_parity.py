@@ -580,6 +580,38 @@ def test_max_pool_aggregator_full_pipeline(C):
     full_check(wl, "summary")
 
 
+@pytest.mark.parametrize("C,d_sum", [(32, 128), (64, 256), (128, 256), (256, 128)])
+def test_token_mlp_aggregator_full_pipeline(C, d_sum):
+    """Eq. 2 taken literally (the MLP on every token, outputs mean-pooled): tiles of several chunks (C < 128), of one
+    chunk, and chunks of two tiles (C = 256); ragged tail; the whole path behind it against the oracle."""
+    wl = wlm.CFG2.small(B=2, H=3, n=C * 9 + 5, C=C, W=2 * C, agg="token_mlp", d_sum=d_sum, seed=60 + C)
+    st, pb, aw, lw = full_check(wl, "summary")
+    assert pb.Nc == 7
+
+
+def test_token_mlp_aggregator_incremental_ranges_and_unsupported_geometry():
+    b = _binding()
+    wl = wlm.CFG2.small(B=1, H=5, n=64 * 11, C=64, W=128, agg="token_mlp", d_sum=256, seed=71)
+    pb = hz.Problem(wl)
+    st = make_store(wl)
+    load_kv(st, 0, pb.K, pb.V)
+    aw, lw = b.AggWeights(pb.mlp), b.LstmWeights(pb.lstm)
+    for lo, hi in ((0, 3), (3, 4), (4, pb.Nc)):          # an odd number of chunks per call: half-filled tiles
+        st.summarize_chunks(0, lo, hi, aw)
+    st.gate(0, 0, pb.Nc, lw)
+    st.compact(0, pb.tau)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    check_summaries(st, pb)
+    check_gate_and_keep(st, pb)
+    with pytest.raises(b.KveError) as e:                  # chunk sizes the tensor-core tiling does not cover are refused at create
+        b.Store(B=1, H=1, C_=48, W=48, max_tokens=480, d_g=64, agg="token_mlp", d_sum=256)
+    assert e.value.rc == -2
+    with pytest.raises(b.KveError) as e:
+        b.Store(B=1, H=1, C_=64, W=64, max_tokens=640, d_g=64, agg="token_mlp", d_sum=192)
+    assert e.value.rc == -2
+
+
 def test_decode_tick_replays_from_a_cuda_graph():
     """append + gated attention of two layers captured once and replayed: the calls neither synchronise nor
     allocate, so the replay must reproduce the eager outputs bit for bit (and the oracle's within tolerance)."""
