@@ -155,6 +155,12 @@ int kvE_set_len(kvE_store* st, int layer, int n, void* stream);
  * KVE_RECLAIM_GATED are gone for KVE_ATTEND_RAW (reading them flags KVE_ERR_CAPACITY). */
 int kvE_set_attend(kvE_store* st, int attend);
 
+/* Precision of the recurrent product W_hh h of Eq. 3 for all later kvE_gate calls on this handle.  W_hh is bf16 and
+ * the state h is fp32; the tensor cores take h as a sum of bf16 planes.  planes == 2 (default): h = hi + lo to
+ * 2^-17 |h| (16 of its 24 significant bits), the faster form; planes == 3: h = p0 + p1 + p2 exactly, every product
+ * exact, the sum differing from a plain fp32 loop only in summation order.  Host-side only. */
+int kvE_set_gate_planes(kvE_store* st, int planes);
+
 /* Eq. 2: summaries of chunks [chunk_begin, chunk_end) of every sequence of `layer`;
  * chunk_end <= floor((n - W) / C).  w is NULL unless agg is KVE_AGG_MLP or KVE_AGG_TOKEN_MLP. */
 int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_end,
@@ -282,6 +288,14 @@ int kvE_profile_read(kvE_store* st, float* us /* [KVE_K_COUNT] */);
 
 /* Text of the last CUDA runtime error seen by this handle's calls ("" if none). */
 const char* kvE_last_cuda_error(const kvE_store* st);
+
+/* ---- self-test (not part of the paper's path) ----------------------------------------------------------------------
+ * Makes a bounded device-side wait run out on purpose, without a fault: a small kernel waits on a barrier that nothing
+ * ever completes, with a limit of a few thousand polls (which == 0: the wait the copy pipelines and tensor-core
+ * commits use) or two milliseconds (which == 1: the wait between the CTAs of a cluster in the gate recurrence).  The
+ * kernel returns by itself, the status word reads KVE_ERR_TIMEOUT at the next kvE_poll_status, and the handle stays
+ * usable.  A way to check, on the installed driver and GPU, that the failure path every kernel relies on works. */
+int kvE_selftest_timeout(kvE_store* st, int which, void* stream);
 
 #ifdef __cplusplus
 }

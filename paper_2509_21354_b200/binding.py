@@ -21,10 +21,10 @@ ATTEND = {"summary": 0, "raw": 1}
 STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_CAPACITY",
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
-EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_set_attend", "kvE_append", "kvE_append_next", "kvE_set_len",
+EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_set_attend", "kvE_set_gate_planes", "kvE_append", "kvE_append_next", "kvE_set_len",
            "kvE_summarize_chunks", "kvE_gate", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense", "kvE_decode_attn_block",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
-           "kvE_profile", "kvE_profile_read"]
+           "kvE_profile", "kvE_profile_read", "kvE_selftest_timeout"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense", "attn_block"]
 
 
@@ -78,6 +78,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_append.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p]
     lib.kvE_set_len.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
     lib.kvE_set_attend.argtypes = [C.c_void_p, C.c_int]
+    lib.kvE_set_gate_planes.argtypes = [C.c_void_p, C.c_int]
     lib.kvE_append_next.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
     lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
     lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
@@ -97,6 +98,7 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_layer_state.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_int)] * 4
     lib.kvE_profile.argtypes = [C.c_void_p, C.c_int]
     lib.kvE_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
+    lib.kvE_selftest_timeout.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.kvE_last_cuda_error.restype = C.c_char_p
     lib.kvE_last_cuda_error.argtypes = [C.c_void_p]
     for name in EXPORTS:
@@ -247,6 +249,10 @@ class Store:
         """"summary" | "raw": what a kept chunk contributes to attention from now on"""
         _check("kvE_set_attend", self.lib.kvE_set_attend(self.handle, ATTEND[attend]))
 
+    def set_gate_planes(self, planes: int):
+        """2 (default) or 3 (exact products) bf16 planes of the LSTM state in the recurrent product"""
+        _check("kvE_set_gate_planes", self.lib.kvE_set_gate_planes(self.handle, int(planes)))
+
     def summarize_chunks(self, layer, chunk_begin, chunk_end, agg_weights=None, stream=None):
         kvE_summarize_chunks(self, layer, chunk_begin, chunk_end, agg_weights, stream)
 
@@ -289,6 +295,10 @@ class Store:
 
     def poll_status(self) -> int:
         return kvE_poll_status(self)
+
+    def selftest_timeout(self, which: int, stream=None):
+        """launches the kernel whose bounded wait runs out (which: 0 = CTA-scope wait, 1 = cluster-scope wait)"""
+        _check("kvE_selftest_timeout", self.lib.kvE_selftest_timeout(self.handle, int(which), _stream(stream)), self.handle)
 
     def layer_state(self, layer=0) -> dict:
         return kvE_layer_state(self, layer)

@@ -24,6 +24,7 @@ struct LayerState {
 struct kvE_store {
   kvE_config cfg;
   kvE_buffers buf;
+  int gate_planes = 2;   // bf16 planes of h in the recurrent product (kvE_set_gate_planes)
   int device = -1;       // the device that was current at kvE_create: owner of every buffer; calls check it
   int S, max_chunks;
   // workspace carve-up (byte offsets)
@@ -369,6 +370,12 @@ int kvE_set_attend(kvE_store* st, int attend) {
   return KVE_OK;
 }
 
+int kvE_set_gate_planes(kvE_store* st, int planes) {
+  if (!st || (planes != 2 && planes != 3)) return KVE_ERR_ARG;
+  st->gate_planes = planes;
+  return KVE_OK;
+}
+
 int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE_agg_weights* w,
                          void* stream) {
   if (bad_layer(st, layer) || chunk_begin < 0 || chunk_end < chunk_begin) return KVE_ERR_ARG;
@@ -432,7 +439,7 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE
   if (e == cudaSuccess) {
     Prof prof(st, KVE_K_GATE_RNN, s);
     e = launch_gate_rnn(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_hh), w->w_s, w->b_s, st->cfg.d_g,
-                        P, chunk_begin == 0, s);
+                        P, chunk_begin == 0, st->gate_planes, s);
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_gated = chunk_end;
@@ -641,6 +648,13 @@ int kvE_profile_read(kvE_store* st, float* us) {
 }
 
 const char* kvE_last_cuda_error(const kvE_store* st) { return st ? st->cuda_error.c_str() : ""; }
+
+int kvE_selftest_timeout(kvE_store* st, int which, void* stream) {
+  if (!st || (which != 0 && which != 1)) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
+  cudaError_t e = launch_selftest_timeout(which, st->buf.status_word, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+}
 
 }  // extern "C"
 

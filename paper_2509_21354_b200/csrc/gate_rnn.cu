@@ -11,7 +11,7 @@
 //    fragments for the whole kernel (128 registers per thread at d_g = 256, CL = 4).
 //  * Per step the CTA computes its rows of W_hh h for all its sequences with warp-level tensor-core
 //    MMAs (m16n8k16, bf16 x bf16 -> fp32).  W_hh is bf16 by definition; the fp32 state h enters as
-//    RNN_PLANES = 2 bf16 planes (h = hi + lo up to 2^-17 |h|: 16 of its 24 significant bits; a third
+//    PL = 2 bf16 planes by default (h = hi + lo up to 2^-17 |h|: 16 of its 24 significant bits; a third
 //    plane makes the products exact, moves the scores by 1e-7 - far below what the fast
 //    exponentials of the cell update contribute, 5e-5 - and costs a third more MMAs: 119 vs 99 us
 //    on 256 sequences x 56 chunks).  Each plane has its own accumulators (as many independent MMA
@@ -38,17 +38,17 @@ namespace kve {
 // NG independent groups of 8 sequences per cluster.  A group is one pipeline (own h buffers, barriers,
 // staging and cell state); a warp works through the groups one after the other within a step, so
 // while group A's new h is on its way between the CTAs the warp is busy with group B.
-template <int DG, int CL, int NG>
+template <int DG, int CL, int NG, int PL>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve_gate_rnn_kernel(RnnArgs a) {
   constexpr int HU = DG / CL;            // hidden units owned by this CTA
   constexpr int UW = HU / RNN_WARPS;     // hidden units per warp
   constexpr int MP = UW / 8;             // pairs of m16 tiles per warp (a pair = 8 units x 4 gates)
   constexpr int KT = DG / 16;            // k tiles
   constexpr int NS = 8;                  // sequences per group: the n of the m16n8k16 MMA
-  constexpr int KBLK = RNN_PLANES * NS * 8;                     // bf16 elements of one k-block: [plane][sequence][8 units]
+  constexpr int KBLK = PL * NS * 8;                     // bf16 elements of one k-block: [plane][sequence][8 units]
   constexpr int HS_BUF = (DG / 8) * KBLK;                       // bf16 elements per h buffer: [k-block][plane][sequence][8]
   constexpr int STG_WARP = MP * KBLK;                           // bf16 elements of one warp's staging area (its k-blocks)
-  constexpr uint32_t H_BYTES = RNN_PLANES * NS * (DG - HU) * 2; // bytes of h planes a CTA receives from its peers per step and group
+  constexpr uint32_t H_BYTES = PL * NS * (DG - HU) * 2; // bytes of h planes a CTA receives from its peers per step and group
   constexpr int OFF_STAGE = NG * 2 * HS_BUF * 2;
   constexpr int OFF_BARS = OFF_STAGE + NG * RNN_WARPS * STG_WARP * 2;
   static_assert(UW % 8 == 0 && MP >= 1, "8 warps x 8k hidden units per CTA");
@@ -96,11 +96,11 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       const float2 hv = *reinterpret_cast<const float2*>(a.lstm_h + (long long)s * DG + k2 * 2);
       h0 = hv.x; h1 = hv.y;
     }
-    uint32_t p0[3], p1[3];      // the leading RNN_PLANES pieces are used
+    uint32_t p0[3], p1[3];      // the leading PL pieces are used
     split3(h0, p0);
     split3(h1, p1);
 #pragma unroll
-    for (int pl = 0; pl < RNN_PLANES; ++pl)
+    for (int pl = 0; pl < PL; ++pl)
       *reinterpret_cast<uint32_t*>(hs + gi * 2 * HS_BUF + (k2 >> 2) * KBLK + (pl * NS + j) * 8 + (k2 & 3) * 2) = p0[pl] | (p1[pl] << 16);
   }
   float c[NG][MP][2], hlast[NG][MP][2];
@@ -155,9 +155,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       }
 
       // ---- W_hh h_{t-1} on the tensor cores: one accumulator set per plane ---------------------------
-      float acc[RNN_PLANES][2 * MP][4];
+      float acc[PL][2 * MP][4];
 #pragma unroll
-      for (int pl = 0; pl < RNN_PLANES; ++pl)
+      for (int pl = 0; pl < PL; ++pl)
 #pragma unroll
         for (int mt = 0; mt < 2 * MP; ++mt)
 #pragma unroll
@@ -165,21 +165,21 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       // B fragments: one ldmatrix.x4 brings the 8 sequences x 32 k-values of a plane (two k tiles);
       // lane l addresses row (l & 7) of the 8 x 8 block (l >> 3).  Loaded one k-tile pair ahead.
       const uint32_t hb_lane = smem_u32(hs_g + buf * HS_BUF + (lane >> 3) * KBLK + (lane & 7) * 8);
-      uint32_t bf[2][RNN_PLANES][4];
+      uint32_t bf[2][PL][4];
 #pragma unroll
-      for (int pl = 0; pl < RNN_PLANES; ++pl) ldmatrix_x4(bf[0][pl], hb_lane + (uint32_t)(pl * NS * 8 * 2));
+      for (int pl = 0; pl < PL; ++pl) ldmatrix_x4(bf[0][pl], hb_lane + (uint32_t)(pl * NS * 8 * 2));
 #pragma unroll
       for (int kp = 0; kp < KT / 2; ++kp) {
         const int cur = kp & 1;
         if (kp + 1 < KT / 2) {
 #pragma unroll
-          for (int pl = 0; pl < RNN_PLANES; ++pl)
+          for (int pl = 0; pl < PL; ++pl)
             ldmatrix_x4(bf[cur ^ 1][pl], hb_lane + (uint32_t)(((kp + 1) * 4 * KBLK + pl * NS * 8) * 2));
         }
 #pragma unroll
         for (int half = 0; half < 2; ++half)
 #pragma unroll
-          for (int pl = 0; pl < RNN_PLANES; ++pl)
+          for (int pl = 0; pl < PL; ++pl)
 #pragma unroll
             for (int mt = 0; mt < 2 * MP; ++mt)
               mma_bf16_16816(acc[pl][mt], A[mt][2 * kp + half], bf[cur][pl][2 * half], bf[cur][pl][2 * half + 1]);
@@ -214,9 +214,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
 #pragma unroll
           for (int q = 0; q < 4; ++q) {   // q: 0 = i, 1 = f (tile 2p, rows g / g+8), 2 = g, 3 = o (tile 2p+1)
             const int mt = 2 * p + (q >> 1), ai = (q & 1) * 2 + e;
-            float sum = acc[RNN_PLANES - 1][mt][ai];      // smallest plane first
+            float sum = acc[PL - 1][mt][ai];      // smallest plane first
 #pragma unroll
-            for (int pl = RNN_PLANES - 2; pl >= 0; --pl) sum += acc[pl][mt][ai];
+            for (int pl = PL - 2; pl >= 0; --pl) sum += acc[pl][mt][ai];
             pre[q] = sum + pin[gi][p][q][e];
           }
           const float ig = fast_sigmoid(pre[0]);
@@ -237,7 +237,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
             split3(hv, pl3);
             const int j = tig * 2 + e;
 #pragma unroll
-            for (int pl = 0; pl < RNN_PLANES; ++pl) my_stage[p * KBLK + (pl * NS + j) * 8 + g] = (uint16_t)pl3[pl];
+            for (int pl = 0; pl < PL; ++pl) my_stage[p * KBLK + (pl * NS + j) * 8 + g] = (uint16_t)pl3[pl];
           }
         }
       }
@@ -315,34 +315,38 @@ __global__ void __launch_bounds__(256) kve_gate_score_kernel(const float* __rest
   }
 }
 
-template <int DG, int CL, int NG>
+template <int DG, int CL, int NG, int PL>
 static cudaError_t launch_rnn_t(const RnnArgs& a, cudaStream_t st) {
   constexpr int NS = 8 * NG;      // sequences per cluster
-  constexpr int smem = 2 * RNN_PLANES * NS * DG * 2 + RNN_PLANES * NS * (DG / CL) * 2 + NG * 2 * 8;
+  constexpr int smem = 2 * PL * NS * DG * 2 + PL * NS * (DG / CL) * 2 + NG * 2 * 8;
   static DeviceFlags opted;
   {
-    cudaError_t e = smem_opt_in(opted, kve_gate_rnn_kernel<DG, CL, NG>, smem);
+    cudaError_t e = smem_opt_in(opted, kve_gate_rnn_kernel<DG, CL, NG, PL>, smem);
     if (e != cudaSuccess) return e;
   }
   const int clusters = (a.S + NS - 1) / NS;
-  return launch_pdl(kve_gate_rnn_kernel<DG, CL, NG>, dim3(clusters * CL), dim3(RNN_THREADS), smem, st, a);
+  return launch_pdl(kve_gate_rnn_kernel<DG, CL, NG, PL>, dim3(clusters * CL), dim3(RNN_THREADS), smem, st, a);
+}
+
+template <int PL>
+static cudaError_t launch_rnn_planes(const RnnArgs& a, int d_g, cudaStream_t st) {
+  // two 8-sequence groups per cluster once one group per cluster would need more than one wave of clusters
+  switch (d_g) {
+    case 256: return (a.S > 8 * (sm_count() / 4)) ? launch_rnn_t<256, 4, 2, PL>(a, st) : launch_rnn_t<256, 4, 1, PL>(a, st);
+    case 128: return launch_rnn_t<128, 1, 1, PL>(a, st);
+    case 64:  return (a.S > 8 * sm_count()) ? launch_rnn_t<64, 1, 2, PL>(a, st) : launch_rnn_t<64, 1, 1, PL>(a, st);
+    default:  return cudaErrorInvalidValue;
+  }
 }
 
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
-                            int d_g, float* P, bool reset_state, cudaStream_t st) {
+                            int d_g, float* P, bool reset_state, int planes, cudaStream_t st) {
   if (t1 <= t0 || v.S <= 0) return cudaSuccess;
   RnnArgs a;
   a.P = P; a.W_hh = W_hh; a.w_s = w_s; a.b_s = b_s;
   a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c; a.status = v.status;
   a.S = v.S; a.max_chunks = v.max_chunks; a.t0 = t0; a.n_range = t1 - t0; a.reset = reset_state ? 1 : 0;
-  // two 8-sequence groups per cluster once one group per cluster would need more than one wave of clusters
-  cudaError_t e;
-  switch (d_g) {
-    case 256: e = (v.S > 8 * (sm_count() / 4)) ? launch_rnn_t<256, 4, 2>(a, st) : launch_rnn_t<256, 4, 1>(a, st); break;
-    case 128: e = launch_rnn_t<128, 1, 1>(a, st); break;
-    case 64:  e = (v.S > 8 * sm_count()) ? launch_rnn_t<64, 1, 2>(a, st) : launch_rnn_t<64, 1, 1>(a, st); break;
-    default:  return cudaErrorInvalidValue;
-  }
+  const cudaError_t e = planes == 3 ? launch_rnn_planes<3>(a, d_g, st) : launch_rnn_planes<2>(a, d_g, st);
   if (e != cudaSuccess) return e;
   const long long n_rows = (long long)v.S * a.n_range;
   return launch_pdl(kve_gate_score_kernel, dim3((unsigned)((n_rows + 7) / 8)), dim3(256), 0, st, (const float*)P, w_s, b_s, v.scores, n_rows,

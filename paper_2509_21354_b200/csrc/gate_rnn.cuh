@@ -9,7 +9,6 @@ namespace kve {
 
 constexpr int RNN_WARPS = 8;
 constexpr int RNN_THREADS = RNN_WARPS * 32;
-constexpr int RNN_PLANES = 2;      // bf16 planes of h that enter the recurrent product (3 = exact)
 
 struct RnnArgs {
   float* P;                // [S * n_range][4 d_g]; columns [0, d_g) of row (s, t) receive h_t once P_t is consumed
@@ -62,8 +61,9 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
       : "memory");
   return ok != 0;
 }
-// bounded: gives up one second after the quick polls ran out, then false
-__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_t parity) {
+// bounded: gives up `deadline_ns` (one second unless told otherwise) after the quick polls ran out, then false
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_t parity,
+                                                          unsigned long long deadline_ns = 1000000000ull) {
   for (int i = 0; i < 4096; ++i)
     if (mbar_try_wait_cluster(bar, parity)) return true;
   unsigned long long t_start, t_now;
@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_
     if (mbar_try_wait_cluster(bar, parity)) return true;
     __nanosleep(128);
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_now));
-  } while (t_now - t_start < 1000000000ull);
+  } while (t_now - t_start < deadline_ns);
   return false;
 }
 __device__ __forceinline__ void cluster_sync_all() {

@@ -73,8 +73,9 @@ bool token_mlp_supported(int C, int d_sum);
 cudaError_t launch_chunk_token_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, float* hid, cudaStream_t st);
 cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t* W_ih, const float* b_ih,
                              const float* b_hh, int d_g, float* P, cudaStream_t st);
+// planes: bf16 planes of the fp32 state h that enter the recurrent product (2, or 3 = exact products)
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
-                            int d_g, float* P, bool reset_state, cudaStream_t st);
+                            int d_g, float* P, bool reset_state, int planes, cudaStream_t st);
 // both also leave the kept chunks' summary rows compacted in kkept / vkept [S][max_chunks][128] bf16, which is
 // what attention reads until the next keep list
 cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, void* kkept, void* vkept, cudaStream_t st);
@@ -87,6 +88,7 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int par
                         float* lse, float scale, const void* kkept, const void* vkept, float* partials, int32_t* counters,
                         cudaStream_t st);
 int attn_smem_bytes();
+cudaError_t launch_selftest_timeout(int which, int32_t* status, cudaStream_t st);
 
 // block-of-queries attention (grouped query heads x query tokens), tensor-map fed
 constexpr int ATTN_BLOCK_MAX_ROWS = 128;       // query rows (tokens x heads per KV head) per KV sequence
