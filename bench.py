@@ -43,7 +43,10 @@ METRIC = "gated_decode_attention_steps_per_sec"
 UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 SCALE = 1.0 / math.sqrt(128.0)
-KERNELS_PER_STEP = 9   # set_len, append, chunk mean, chunk MLP, gate projection, gate recurrence, score head, compact, attention
+def kernels_per_step(wl, Nc):
+    """kernel launches of one from-scratch step: set_len, append, chunk mean [+ chunk MLP], gate projection,
+    recurrence, score head, keep list, kept-row gather, attention"""
+    return 9 + (1 if wl.agg == "mlp" else 0)
 
 
 def load_peaks():
@@ -793,7 +796,7 @@ def run_ours(args, rank, world, local_rank):
                    "loops_ms": loops, "timed_s_total": sum(loops) / 1e3},
         "e2e": {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * S * 256,
                 "d2h_bytes_per_step": S * 256, "matches_device_path": same},
-        "gpu_launches": KERNELS_PER_STEP * args.steps * repeats,
+        "gpu_launches": kernels_per_step(wl, rig.Nc) * args.steps * repeats,
         "clocks": clk.summary(),
         "roofline": roofline,
         "roofline_largest_hbm_kernel": roofline_hbm,

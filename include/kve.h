@@ -176,6 +176,12 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
  * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw. */
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream);
 
+/* Sec. 3.3, the whole aggregation-and-gating step of `layer` from scratch in one call: summaries of every chunk
+ * outside the window (Eq. 2), the gate over all of them starting from h = c = 0 (Eq. 3), the keep list for `tau`
+ * (Sec. 3.2): kvE_summarize_chunks(0, Nc) + kvE_gate(0, Nc) + kvE_compact(tau), Nc = floor((n - W) / C).
+ * aw is NULL unless the aggregator has an MLP. */
+int kvE_refresh(kvE_store* st, int layer, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, void* stream);
+
 /* The gating-strategy variant the paper names for its ablations (Sec. 5): keep the k highest-scoring gated
  * chunks of every sequence instead of thresholding.  Equal scores: the older chunk ranks first, so the
  * list is unique.  Writes keep_idx / keep_cnt like kvE_compact (ascending ids; k <= 0 keeps nothing,
@@ -253,7 +259,7 @@ int kvE_decode_attn_static(kvE_store* st, int layer, const void* q, void* out, f
 
 /* One whole decode step of `layer` from HOST memory: copies k_new, v_new, q (bf16 [S][d] each,
  * ideally pinned) to the device, appends the token, brings summaries, gate and keep list up to
- * date for every chunk that has left the window (from scratch if `from_scratch` != 0), runs
+ * date for every chunk that has left the window (from scratch, through kvE_refresh, if `from_scratch` != 0), runs
  * kvE_decode_attn and copies out (bf16 [S][d]) back to host memory.  Staging uses the tail of the
  * workspace.  Waits for the stream before returning. */
 int kvE_decode_step_host(kvE_store* st, int layer, const void* k_new_host, const void* v_new_host,

@@ -37,6 +37,7 @@ struct kvE_store {
   int block_hp = 0, block_split_cap = 1;
   std::vector<LayerState> layers;
   std::string cuda_error;
+
   // optional per-kernel timing: one (start, stop) event pair per kernel id
   bool profiling = false;
   cudaEvent_t ev[2 * KVE_K_COUNT] = {};
@@ -242,6 +243,11 @@ int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* 
                        reinterpret_cast<int32_t*>(ws + st->off_counters), stream);
 }
 
+void release_host_objects(kvE_store* st) {
+  if (st->ev_made)
+    for (cudaEvent_t e : st->ev) cudaEventDestroy(e);
+}
+
 }  // namespace
 
 extern "C" {
@@ -297,6 +303,7 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   if (e == cudaSuccess) e = cudaMemset(buf->keep_cnt, 0, sizeof(int32_t) * (size_t)cfg->n_layers * st->S);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
+    release_host_objects(st);
     delete st;
     return KVE_ERR_CUDA;
   }
@@ -305,8 +312,7 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
 }
 
 int kvE_destroy(kvE_store* st) {
-  if (st && st->ev_made)
-    for (cudaEvent_t e : st->ev) cudaEventDestroy(e);
+  if (st) release_host_objects(st);
   delete st;
   return KVE_OK;
 }
@@ -461,6 +467,15 @@ int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   return KVE_OK;
 }
 
+int kvE_refresh(kvE_store* st, int layer, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, void* stream) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  const int nc = stale_chunks(st->cfg, st->layers[layer].n_tokens);
+  int rc = kvE_summarize_chunks(st, layer, 0, nc, aw, stream);
+  if (rc == KVE_OK) rc = kvE_gate(st, layer, 0, nc, lw, stream);
+  if (rc == KVE_OK) rc = kvE_compact(st, layer, tau, stream);
+  return rc;
+}
+
 int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream) {
   if (bad_layer(st, layer)) return KVE_ERR_ARG;
   if (wrong_device(st)) return KVE_ERR_STATE;
@@ -565,17 +580,21 @@ static int decode_step_host(kvE_store* st, int layer, const void* k_new_host, co
   if (rc != KVE_OK) return rc;
   LayerState& ls = st->layers[layer];
   const int nc = stale_chunks(st->cfg, ls.n_tokens);
-  const int s0 = from_scratch ? 0 : ls.n_summarised;
+  if (from_scratch) {
+    rc = kvE_refresh(st, layer, aw, lw, tau, stream);
+    if (rc != KVE_OK) return rc;
+  }
+  const int s0 = ls.n_summarised;
   if (nc > s0) {
     rc = kvE_summarize_chunks(st, layer, s0, nc, aw, stream);
     if (rc != KVE_OK) return rc;
   }
-  const int g0 = from_scratch ? 0 : ls.n_gated;
-  if (nc > g0 || from_scratch) {
+  const int g0 = ls.n_gated;
+  if (nc > g0) {
     rc = kvE_gate(st, layer, g0, nc, lw, stream);
     if (rc != KVE_OK) return rc;
   }
-  if (ls.n_compacted != ls.n_gated || from_scratch) {
+  if (ls.n_compacted != ls.n_gated) {
     rc = kvE_compact(st, layer, tau, stream);
     if (rc != KVE_OK) return rc;
   }

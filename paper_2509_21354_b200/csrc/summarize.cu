@@ -84,16 +84,33 @@ __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerVi
   }
 }
 
+// CTAs of the mean kernel that are resident per SM (registers decide), looked up once per device
+template <bool POOL_MAX>
+static int mean_ctas_per_sm() {
+  static std::atomic<int> cached[MAX_DEVICES];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 4;
+  int n = cached[dev].load(std::memory_order_acquire);
+  if (n > 0) return n;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kve_chunk_mean_kernel<POOL_MAX>, MEAN_WARPS * 32, 0) != cudaSuccess || n <= 0) n = 4;
+  cached[dev].store(n, std::memory_order_release);
+  return n;
+}
+
+// The grid is exactly one resident wave and every warp strides over the units, so all SMs carry the same share.
+// That only holds if the CTAs land on an empty GPU: the kernel is therefore launched WITHOUT the programmatic edge the
+// other kernels use.  (Launched early, beside the tail of its predecessor, its CTAs spread unevenly over the SMs
+// and the static striding turns that into a tail: measured +25 % on 4 GB of stale KV.)
 cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st) {
   const int n_range = t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
   long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
-  if (blocks > sm_count() * 8LL) blocks = sm_count() * 8LL;      // 64 resident warps per SM, every CTA resident from the start
-  if (pool_max)
-    return launch_pdl(kve_chunk_mean_kernel<true>, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units, 1);
-  return launch_pdl(kve_chunk_mean_kernel<false>, dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st, v, t0, n_range, n_units,
-                    final_output ? 1 : 0);
+  const long long wave = (long long)sm_count() * (pool_max ? mean_ctas_per_sm<true>() : mean_ctas_per_sm<false>());
+  if (blocks > wave) blocks = wave;
+  if (pool_max) kve_chunk_mean_kernel<true><<<dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st>>>(v, t0, n_range, n_units, 1);
+  else kve_chunk_mean_kernel<false><<<dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st>>>(v, t0, n_range, n_units, final_output ? 1 : 0);
+  return cudaGetLastError();
 }
 
 // ---- aggregator MLP (Eq. 2 read as mean -> d_sum -> d, exact-erf GELU), fp32 FMA ------------------

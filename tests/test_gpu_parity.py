@@ -278,6 +278,43 @@ def test_set_len_below_the_compacted_range_drops_the_keep_list():
     check_attention(st, pb, "summary")
 
 
+@pytest.mark.parametrize("agg", ["mlp", "mean", "token_mlp"])
+def test_refresh_equals_the_stepwise_calls(agg):
+    """kvE_refresh = summaries of all stale chunks + gate from scratch + keep list in one call: against the oracle, and
+    bit for bit against the three calls issued one after the other; also replayed from a CUDA graph."""
+    b = _binding()
+    wl = wlm.CFG2.small(B=2, H=6, n=64 * 75 + 9, C=64, W=128, agg=agg, d_sum=256 if agg != "mean" else 0, seed=91)
+    pb = hz.Problem(wl)
+    assert pb.Nc == 73
+    st = make_store(wl)
+    load_kv(st, 0, pb.K, pb.V)
+    aw = b.AggWeights(pb.mlp) if pb.mlp is not None else None
+    lw = b.LstmWeights(pb.lstm)
+    for rep in range(2):                                     # twice: the second run finds the first one's state
+        st.refresh(0, aw, lw, pb.tau)
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        assert st.layer_state(0) == dict(n_tokens=wl.n, n_summarised=pb.Nc, n_gated=pb.Nc, n_compacted=pb.Nc)
+        check_summaries(st, pb)
+        check_gate_and_keep(st, pb)
+        check_attention(st, pb, "summary", step=rep)
+    got = [x.clone() for x in (st.scores[0], st.keep_idx[0], st.lstm_h[0], st.lstm_c[0], st.ksum_bf16[0])]
+    run_gpu_pipeline(st, pb, 0, aw, lw)
+    for a_, b_ in zip(got, (st.scores[0], st.keep_idx[0], st.lstm_h[0], st.lstm_c[0], st.ksum_bf16[0])):
+        assert torch.equal(a_, b_)
+    # inside a CUDA graph
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            st.refresh(0, aw, lw, pb.tau)
+    torch.cuda.current_stream().wait_stream(side)
+    st.scores.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0 and torch.equal(st.scores[0], got[0])
+
+
 def test_layers_are_independent():
     b = _binding()
     wl = wlm.CFG1.small(n=1024, B=2, H=4, n_layers=3)
