@@ -237,11 +237,11 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
     return res
 
 
-def graph_tick_leg(wl, n_layers, seed, replays=20, mem_cap=40e9):
+def graph_tick_leg(wl, n_layers, seed, replays=20, mem_cap=40e9, fused=True):
     """The decode loop of a whole model between two gate triggers: per token, for each of n_layers layers
     append the new token at the device-held length (kvE_append_next) and run the gated attention; all
     layers captured once in a CUDA graph, every replay advancing by one token.  Compared with the
-    same calls issued one by one."""
+    same calls issued one by one.  fused: kvE_decode_step (append + attention in one launch) instead of the two calls."""
     import torch
     from paper_2509_21354_b200 import binding as b
     g = wl.small(agg="mean", d_sum=0)                      # the aggregator only feeds the keep list here
@@ -278,8 +278,11 @@ def graph_tick_leg(wl, n_layers, seed, replays=20, mem_cap=40e9):
 
     def tick():                                            # every call / replay appends the NEXT token of every layer
         for L in range(n_layers):
-            st.append_next(L, k_new[L], v_new[L], n_reserve=2 * budget)
-            st.decode_attn(L, q[L], out[L])
+            if fused:
+                st.decode_step(L, k_new[L], v_new[L], q[L], out[L], n_reserve=2 * budget)
+            else:
+                st.append_next(L, k_new[L], v_new[L], n_reserve=2 * budget)
+                st.decode_attn(L, q[L], out[L])
 
     tick()
     torch.cuda.synchronize()
@@ -296,10 +299,11 @@ def graph_tick_leg(wl, n_layers, seed, replays=20, mem_cap=40e9):
     graph.replay()
     torch.cuda.synchronize()
     same = bool(torch.equal(out, eager_out))
-    res = {"what": f"decode loop over {n_layers} layers between two gate triggers (per layer and token: kvE_append_next at the "
-                   "device-held length, gated attention), captured once in a CUDA graph and replayed - every replay "
-                   "appends the next token - vs the same calls issued one by one",
-           "n_layers": n_layers, "graph_first_tick_equals_eager": same}
+    calls = "kvE_decode_step: append at the device-held length + gated attention in one launch" if fused else \
+        "kvE_append_next at the device-held length, then kvE_decode_attn"
+    res = {"what": f"decode loop over {n_layers} layers between two gate triggers (per layer and token: {calls}), captured once "
+                   "in a CUDA graph and replayed - every replay appends the next token - vs the same calls issued one by one",
+           "n_layers": n_layers, "launches_per_layer_and_token": 1 if fused else 2, "graph_first_tick_equals_eager": same}
     for name, fn in (("eager", tick), ("graph", graph.replay)):
         rewind()
         for _ in range(3):
@@ -368,7 +372,13 @@ class Rig:
         st.decode_attn(0, self.q, self.out)
 
     def step_steady(self):
-        """the step between two gate triggers (token n0 + 1: no chunk leaves the window, the keep list stands)"""
+        """the step between two gate triggers (token n0 + 1: no chunk leaves the window, the keep list stands):
+        roll back, then append + gated attention in one launch (kvE_decode_step)"""
+        st = self.st
+        st.set_len(0, self.n0)
+        st.decode_step(0, self.k_new, self.v_new, self.q, self.out)
+
+    def step_steady_two_launches(self):
         st = self.st
         st.set_len(0, self.n0)
         st.append(0, self.k3, self.v3)
@@ -675,14 +685,19 @@ def sweep_leg(peaks, peak_kind, flush, seed, mem_cap=120e9):
 def action_step_leg(seed):
     """cfg3 in its stated form: one control step = 7 action tokens appended autoregressively, each through all 32
     layers (append at the device-held length + gated attention per layer and token), the 32-layer tick captured in a
-    CUDA graph and replayed 7 times."""
+    CUDA graph and replayed 7 times; with kvE_decode_step (one launch per layer and token) and, for comparison, with the two
+    separate calls."""
     wl = wlm.CFG3
+    two = graph_tick_leg(wl, wl.n_layers, seed, replays=wl.n_append, fused=False)
     r = graph_tick_leg(wl, wl.n_layers, seed, replays=wl.n_append)
     ms = r["graph"]["ms_per_tick"] * wl.n_append
     return {"what": f"{wl.n_append} action tokens x {r['n_layers']} layers, graph-replayed (B={wl.B}, H={wl.H}, n={wl.n})",
             "ms_per_action_step": ms, "action_steps_per_s": 1e3 / ms, "attention_calls_per_action_step": wl.n_append * r["n_layers"],
             "us_per_layer_and_token": r["graph"]["us_per_layer"], "eager_ms_per_action_step": r["eager"]["ms_per_tick"] * wl.n_append,
-            "kv_bytes_per_token": r["kv_bytes_per_tick"], "GB/s": r["GB/s_graph"], "graph_first_tick_equals_eager": r["graph_first_tick_equals_eager"]}
+            "kv_bytes_per_token": r["kv_bytes_per_tick"], "GB/s": r["GB/s_graph"], "graph_first_tick_equals_eager": r["graph_first_tick_equals_eager"],
+            "launches_per_layer_and_token": 1,
+            "with_two_launches_per_layer_and_token": {"ms_per_action_step": two["graph"]["ms_per_tick"] * wl.n_append,
+                                                      "us_per_layer_and_token": two["graph"]["us_per_layer"]}}
 
 
 def run_ours(args, rank, world, local_rank):
@@ -720,8 +735,11 @@ def run_ours(args, rank, world, local_rank):
     assert st.poll_status() == 0
     rig.step_full()                      # back to the state and output of a full step
     torch.cuda.synchronize()
-    steady = {"what": "append + gated attention only (summaries, gate and keep list reused: the state between two triggers)",
-              "value": world * args.steps / (ms_steady * 1e-3), "unit": UNIT, "ms_per_step": ms_steady / args.steps}
+    ms_two = float(np.median(max_over_ranks(time_loop(rig.step_steady_two_launches, args.steps, min(repeats, 3), barrier), world)))
+    steady = {"what": "append + gated attention only (summaries, gate and keep list reused: the state between two triggers), "
+                      "through kvE_decode_step (one launch)",
+              "value": world * args.steps / (ms_steady * 1e-3), "unit": UNIT, "ms_per_step": ms_steady / args.steps,
+              "ms_per_step_with_separate_append_and_attention": ms_two / args.steps}
 
     # ---- end to end: the same step through kvE_decode_step_host, host buffers, copies timed ----
     hk, hv, hq = (t.cpu().pin_memory() for t in (rig.k_new, rig.v_new, rig.q))

@@ -210,6 +210,17 @@ int kvE_reclaim_pages(kvE_store* st, int layer, int chunk_begin, int chunk_end, 
 int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale,
                     void* stream);
 
+/* One decode step of `layer` between two gate triggers in ONE launch: append the step's token to every sequence
+ * (k_new, v_new: DEVICE bf16 [S][d]) and attend over [kept chunks ; raw tail] with it included (Sec. 3.2 "temporal
+ * order" + Sec. 3.3 + Eq. 1).  Same result as kvE_append_next(n_new = 1) followed by kvE_decode_attn.  The token goes
+ * to the position the DEVICE holds (seq_len), which the call advances by one, so the call can be captured in a CUDA
+ * graph and every replay handles the next token (the buffers are read at replay time); n_reserve as in
+ * kvE_append_next.  The handle's own length advances by one per call, not per replay: give it the true length with
+ * kvE_set_len before the next summarise / gate.  A full cache sets KVE_ERR_CAPACITY in the status word and attends
+ * over what is stored.  q, out: DEVICE bf16 [S][d]; lse: DEVICE fp32 [S] or NULL. */
+int kvE_decode_step(kvE_store* st, int layer, const void* k_new, const void* v_new, const void* q, void* out, float* lse,
+                    float scale, int n_reserve, void* stream);
+
 /* Eq. 1 over all n stored tokens of `layer` (the full-cache baseline of Sec. 3.3). */
 int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse,
                           float scale, void* stream);

@@ -22,7 +22,7 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_set_attend", "kvE_set_gate_planes", "kvE_append", "kvE_append_next", "kvE_set_len",
-           "kvE_summarize_chunks", "kvE_gate", "kvE_refresh", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_attn_dense", "kvE_decode_attn_block",
+           "kvE_summarize_chunks", "kvE_gate", "kvE_refresh", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_step", "kvE_decode_attn_dense", "kvE_decode_attn_block",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read", "kvE_selftest_timeout"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense", "attn_block"]
@@ -87,6 +87,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_compact_topk.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
     lib.kvE_decode_attn.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
     lib.kvE_decode_attn_dense.argtypes = lib.kvE_decode_attn.argtypes
+    lib.kvE_decode_step.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                    C.c_int, C.c_void_p]
     lib.kvE_decode_attn_static.argtypes = lib.kvE_decode_attn.argtypes
     lib.kvE_decode_attn_block.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                           C.c_float, C.c_void_p]
@@ -274,6 +276,17 @@ class Store:
 
     def decode_attn(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn(self, layer, q, out, lse, scale, stream)
+
+    def decode_step(self, layer, k_new, v_new, q, out=None, lse=None, scale=None, n_reserve=0, stream=None):
+        """append one token per sequence (k_new, v_new: bf16 [S, 128]) at the device-held length and attend, one launch"""
+        for t in (k_new, v_new, q):
+            assert t.dtype == torch.bfloat16 and tuple(t.shape) == (self.S, 128)
+        if out is None:
+            out = torch.empty_like(q)
+        scale = 1.0 / np.sqrt(128.0) if scale is None else scale
+        _check("kvE_decode_step", self.lib.kvE_decode_step(self.handle, layer, _p(k_new), _p(v_new), _p(q), _p(out), _p(lse),
+                                                           C.c_float(scale), int(n_reserve), _stream(stream)), self.handle)
+        return out
 
     def decode_attn_dense(self, layer, q, out=None, lse=None, scale=None, stream=None):
         return kvE_decode_attn_dense(self, layer, q, out, lse, scale, stream)

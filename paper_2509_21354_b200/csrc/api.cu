@@ -226,13 +226,14 @@ KeptRows kept_rows(const kvE_store* st, int layer) {
 }
 
 int run_attention(kvE_store* st, int layer, AttnMode mode, const void* q, void* out, float* lse, float scale,
-                  float* partials, int32_t* counters, cudaStream_t stream) {
+                  float* partials, int32_t* counters, cudaStream_t stream, const void* k_new = nullptr, const void* v_new = nullptr) {
   const LayerState& ls = st->layers[layer];
   const KeptRows kr = kept_rows(st, layer);
   const AttnCut cut = attention_cut(st, mode, ls);
+  int32_t* ticket = reinterpret_cast<int32_t*>(static_cast<char*>(st->buf.workspace) + st->off_ticket);
   Prof prof(st, mode == ATTN_DENSE ? KVE_K_ATTN_DENSE : KVE_K_ATTN, stream);
   cudaError_t e = launch_attn(view(st, layer), mode, ls.n_compacted, cut.k, cut.grid, q, out, lse, scale, kr.k, kr.v, partials,
-                              counters, stream);
+                              counters, k_new, v_new, ticket, stream);
   return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
 }
 
@@ -516,6 +517,24 @@ int kvE_decode_attn(kvE_store* st, int layer, const void* q, void* out, float* l
   if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;      // grouped query heads go through kvE_decode_attn_block
   const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
   return run_attention(st, layer, mode, q, out, lse, scale, static_cast<cudaStream_t>(stream));
+}
+
+int kvE_decode_step(kvE_store* st, int layer, const void* k_new, const void* v_new, const void* q, void* out, float* lse,
+                    float scale, int n_reserve, void* stream) {
+  if (bad_layer(st, layer) || !k_new || !v_new || !q || !out || n_reserve < 0) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
+  if (st->cfg.Hq != st->cfg.Hkv) return KVE_ERR_GEOMETRY;
+  LayerState& ls = st->layers[layer];
+  if ((long long)ls.n_tokens + 1 > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
+  // the launch is sized for the cache with the new token (and the announced growth) in it
+  long long upper = (long long)ls.n_tokens + 1 + n_reserve;
+  if (upper > st->cfg.max_tokens) upper = st->cfg.max_tokens;
+  if (upper > ls.reserve_upper) ls.reserve_upper = (int)upper;
+  ls.n_tokens += 1;
+  const AttnMode mode = st->cfg.attend == KVE_ATTEND_RAW ? ATTN_RAW : ATTN_SUMMARY;
+  char* ws = static_cast<char*>(st->buf.workspace);
+  return run_attention(st, layer, mode, q, out, lse, scale, reinterpret_cast<float*>(ws + st->off_partials),
+                       reinterpret_cast<int32_t*>(ws + st->off_counters), static_cast<cudaStream_t>(stream), k_new, v_new);
 }
 
 int kvE_decode_attn_dense(kvE_store* st, int layer, const void* q, void* out, float* lse, float scale, void* stream) {

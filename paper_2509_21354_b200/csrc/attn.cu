@@ -25,6 +25,9 @@
 //    either writes the output (this CTA had the whole sequence) or a partial record plus an atomic
 //    ticket; the CTA that draws a sequence's last ticket merges its records by log-sum-exp.  Nobody
 //    spins on another CTA.
+//  * Fused append (kvE_decode_step): the step's new token need not be in its page yet.  Its row is streamed from the
+//    caller's buffer as the last row of the raw tail, the CTA that streams it also stores it in the page, and the last
+//    CTA to finish advances the stored length: one launch per decode step and layer instead of two.
 // Every mbarrier wait is bounded; on give-up the status word gets KVE_ERR_TIMEOUT.
 #include "common.cuh"
 #include "kernels.h"
@@ -86,11 +89,17 @@ struct AttnArgs {
   const uint16_t* vkept;
   float* partials;             // [S + G][132]: the record of (sequence s, CTA c) sits at s + c
   int32_t* counters;           // [S], zero between launches
+  // fused append (kvE_decode_step): one new token per sequence, placed at the length the device holds
+  const uint16_t* k_new;       // [S][128] or null
+  const uint16_t* v_new;
+  int32_t* ticket;             // last CTA to finish publishes the new length
 };
 
 // what every role derives from the launch arguments and the stored length
 struct AttnGeo {
   int n_tail, raw0, TT, per;   // tail rows / tiles per sequence; rows a kept chunk contributes
+  int n;                       // tokens attended to (the new one included when one is being appended)
+  bool appending;              // the last tail row of every sequence is the new token, taken from k_new / v_new
   uint32_t I, P;               // parts in the launch (S k); CTAs that get any (min(G, I): none of them is empty)
 };
 
@@ -181,6 +190,10 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   {
     int n = v.seq_len[0];
     n = min(max(n, 0), v.max_tokens);
+    g.appending = a.k_new != nullptr && n < v.max_tokens;
+    if (a.k_new != nullptr && !g.appending && blockIdx.x == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);   // cache full
+    if (g.appending) n += 1;
+    g.n = n;
     g.raw0 = (a.mode == ATTN_DENSE) ? 0 : a.n_chunks * v.C;
     g.n_tail = max(0, n - g.raw0);
     g.TT = (g.n_tail + AT_TILE - 1) / AT_TILE;
@@ -249,6 +262,11 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
         const int L = t.j * AT_TILE + rl;              // row inside the sequence's list
         int chunk, r;
         if (t.list == 0) {
+          if (g.appending && L == g.n_tail - 1) {      // the token being appended: straight from the caller's buffers
+            ta.k[half] = a.k_new + (long long)t.s * D;
+            ta.v[half] = a.v_new + (long long)t.s * D;
+            continue;
+          }
           const int p = g.raw0 + L;
           chunk = p / v.C;
           r = p - chunk * v.C;
@@ -309,11 +327,27 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
     // The first tiles go out as soon as each is resolved; from then on the addresses of tile i + 1 are
     // looked up before the wait for its stage, i.e. while the consumers still work on the tiles in flight.
     // The END description takes a stage of its own (no copies): that is how the consumers learn that they are done.
+    // fused append: whoever streams a sequence's last tail tile also stores the new token's row in its page
+    // (lanes 0-15 the K row, 16-31 the V row, 16 bytes each)
+    auto store_new_token = [&](const TileDesc& td) {
+      if (!g.appending || (td.flags & TF_END) || td.list != 0 || td.rows == 0 || td.j * AT_TILE + td.rows != g.n_tail) return;
+      const int pos = g.n - 1, chunk = pos / v.C, r = pos - chunk * v.C;
+      const long long page = v.page_table[(long long)td.s * v.max_chunks + chunk];
+      if (page < 0 || page >= v.n_pages) {
+        if (lane == 0) set_status(v.status, ERR_CAPACITY);
+        return;
+      }
+      const int is_v = lane >> 4, l16 = lane & 15;
+      const uint4* src = reinterpret_cast<const uint4*>((is_v ? a.v_new : a.k_new) + (long long)td.s * D) + l16;
+      uint4* dst = reinterpret_cast<uint4*>((is_v ? v.v_pages : v.k_pages) + (page * v.C + r) * D) + l16;
+      *dst = __ldg(src);
+    };
     TileDesc d;
     TileAddr t;
     for (int i = 0;; ++i) {
       next_tile(d);
       resolve(d, t);
+      store_new_token(d);
       if (!issue(i, d, t) || (d.flags & TF_END)) break;
       KVE_STAMP(i == 0 && lane == 0, 2);
     }
@@ -481,13 +515,27 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       *reinterpret_cast<uint2*>(a.out + (long long)s * D + lane * 4) = o;
       if (a.lse && lane == 0) a.lse[s] = (lC > 0.f) ? (mC + log2f(lC)) * 0.69314718055994530942f : -INFINITY;
     }
+    // fused append: every CTA read the old length when it started; the last one to get here publishes the new one
+    if (g.appending) {
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) {
+        __threadfence();
+        last = atomicAdd(a.ticket, 1) == (int)gridDim.x - 1;
+      }
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        for (int b = lane; b < v.B; b += 32) v.seq_len[b] = g.n;
+        if (lane == 0) *a.ticket = 0;      // clean for the next launch
+      }
+    }
     KVE_STAMP(lane == 0, 5);
   }
 }
 
 cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int parts_per_seq, int grid, const void* q, void* out,
                         float* lse, float scale, const void* kkept, const void* vkept, float* partials, int32_t* counters,
-                        cudaStream_t st) {
+                        const void* k_new, const void* v_new, int32_t* ticket, cudaStream_t st) {
   if (v.S <= 0) return cudaSuccess;
   static DeviceFlags opted;
   {
@@ -499,6 +547,7 @@ cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int par
   a.q = static_cast<const uint16_t*>(q); a.out = static_cast<uint16_t*>(out); a.lse = lse; a.scale = scale;
   a.kkept = static_cast<const uint16_t*>(kkept); a.vkept = static_cast<const uint16_t*>(vkept);
   a.partials = partials; a.counters = counters;
+  a.k_new = static_cast<const uint16_t*>(k_new); a.v_new = static_cast<const uint16_t*>(v_new); a.ticket = ticket;
   return launch_pdl(kve_decode_attn_kernel, dim3((unsigned)(grid < 1 ? 1 : grid)), dim3(AT_THREADS), AT_SMEM_BYTES, st, a);
 }
 

@@ -84,9 +84,11 @@ cudaError_t launch_reclaim(const LayerView& v, int t0, int t1, float tau, int mo
                            long long capacity, int32_t* free_count, cudaStream_t st);
 // parts_per_seq: equal parts every sequence is cut into; grid: CTAs that share the S * parts_per_seq parts;
 // partials: S + grid records of ATTN_PARTIAL_FLOATS
+// k_new, v_new ([S][128] bf16) non-null: fused append of one token per sequence at the device-held length; ticket: one
+// int32 (zero between launches) through which the last CTA publishes the new length
 cudaError_t launch_attn(const LayerView& v, AttnMode mode, int n_chunks, int parts_per_seq, int grid, const void* q, void* out,
                         float* lse, float scale, const void* kkept, const void* vkept, float* partials, int32_t* counters,
-                        cudaStream_t st);
+                        const void* k_new, const void* v_new, int32_t* ticket, cudaStream_t st);
 int attn_smem_bytes();
 cudaError_t launch_selftest_timeout(int which, int32_t* status, cudaStream_t st);
 

@@ -11,7 +11,7 @@
 //      128-token slice of a longer chunk).  The token rows are bf16 already, so they are the A operand as
 //      they stand: 16-byte asynchronous copies put a page's rows into the swizzled layout; 8 tcgen05.mma
 //      (M 128, N d_sum, K 16 each) accumulate the pre-activations in tensor memory.
-//    * Two A buffers and two accumulators: while the eight warps read tile i out of tensor memory (a thread
+//    * Two A buffers and two accumulators: while the sixteen warps read tile i out of tensor memory (a thread
 //      owns one token), add b1, apply the erf GELU and sum each column over the tokens of a chunk with a
 //      butterfly of shuffles (lane l ends up with column l), tile i + 1 is gathered and multiplied.
 //    * The pooled activations (1/C) sum_j gelu(...) go to a scratch row per (side, sequence, chunk).
@@ -28,7 +28,7 @@
 namespace kve {
 
 constexpr int TM_M = 128;                                   // tokens per tile
-constexpr int TM_THREADS = 256;
+constexpr int TM_THREADS = 512;                             // 16 warps: four per scheduler hide the latency of the activation chains
 constexpr int TM_MAX_DSUM = 256;
 constexpr int TM_KB_BYTES = TM_M * umma::KBLOCK_ROW_BYTES;  // 16 KB: 128 rows x 64 head dims
 constexpr int TM_SMEM_W1 = 0;                               // 2 K-blocks of [d_sum rows][64]: up to 64 KB
@@ -133,8 +133,8 @@ __global__ void __launch_bounds__(TM_THREADS, 1) kve_token_mlp_pool_kernel(Token
   };
   // Columns [c, c + 32) of this warp's 32 tokens: + b1, GELU, summed over the tokens; lane l adds the sum of
   // column c + l to the running sum of the chunk the warp's tokens belong to.
-  const int lg = warp & 3, half = warp >> 2;
-  const int cols_half = d_sum >> 1;
+  const int lg = warp & 3, quarter = warp >> 2;      // tensor-memory lanes 32 lg .., columns [quarter d_sum / 4, ..)
+  const int cols_q = d_sum >> 2;                     // 32 or 64 columns per warp
   auto epilogue_cols = [&](uint32_t tmem_acc, int c, float* pool_row) {
     float h[32];
     umma::tmem_ld32(tmem_acc + ((uint32_t)(lg * 32) << 16) + (uint32_t)c, h);
@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) kve_token_mlp_pool_kernel(Token
     }
     umma::fence_after_sync();
     const uint32_t acc = tmem_d + (uint32_t)sel * TM_MAX_DSUM;
-    for (int c = half * cols_half; c < half * cols_half + cols_half / 2; c += 32) epilogue_cols(acc, c, pool_row);
+    epilogue_cols(acc, quarter * cols_q, pool_row);
     if (next < n_tiles) {
       cp_async_wait_all();
       umma::fence_smem_to_async();
@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) kve_token_mlp_pool_kernel(Token
       __syncthreads();                                               // also: the other accumulator was drained a tile ago
       if (tid == 0) issue_mma(tmem_d + (uint32_t)(sel ^ 1) * TM_MAX_DSUM, sel ^ 1);
     }
-    for (int c = half * cols_half + cols_half / 2; c < (half + 1) * cols_half; c += 32) epilogue_cols(acc, c, pool_row);
+    if (cols_q > 32) epilogue_cols(acc, quarter * cols_q + 32, pool_row);
     sel ^= 1;
     // the chunk(s) of this item are complete with its last slice: pooled activations out, pool cleared (the barrier at
     // the top of the next round separates the clearing from the next tile's sums)

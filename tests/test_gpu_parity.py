@@ -916,6 +916,64 @@ def test_decode_loop_advances_under_a_cuda_graph():
     assert st2.poll_status() == -3 and int(st2.seq_len[0, 0]) == wl2.n + 400
 
 
+@pytest.mark.parametrize("attend", ["summary", "raw"])
+def test_decode_step_appends_and_attends_in_one_launch(attend):
+    """kvE_decode_step = append one token at the device-held length + gated attention over the cache with it, one launch:
+    against the oracle on the growing cache, byte-exact pages, across a page boundary, and replayed from a CUDA graph."""
+    b = _binding()
+    steps = 40
+    wl = wlm.CFG3.small(B=2, H=4, n_layers=1, n=64 + 2 * 256 + 50, n_append=steps + 2, seed=55)      # 50 rows into a page: crosses at step 14
+    pb = hz.Problem(wl)
+    st = make_store(wl, attend)
+    aw, lw = b.AggWeights(pb.mlp), b.LstmWeights(pb.lstm)
+    load_kv(st, 0, pb.K, pb.V)
+    run_gpu_pipeline(st, pb, 0, aw, lw)
+    S = st.S
+    k_in = torch.zeros((S, 128), dtype=torch.bfloat16, device="cuda")
+    v_in, q_in, out = torch.zeros_like(k_in), torch.zeros_like(k_in), torch.zeros_like(k_in)
+    lse = torch.zeros(S, dtype=torch.float32, device="cuda")
+    K, V = pb.K, pb.V
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    for step in range(steps):
+        kn, vn = wlm.gen_new_tokens(wl, 0, step)
+        q = wlm.gen_q(wl, 0, step)
+        k_in.copy_(b.bits_to_bf16(kn[:, 0])); v_in.copy_(b.bits_to_bf16(vn[:, 0])); q_in.copy_(b.bits_to_bf16(q))
+        if step < 3:                                   # issued directly
+            st.decode_step(0, k_in, v_in, q_in, out, lse=lse, n_reserve=steps)
+        else:
+            if step == 3:                              # then captured once and replayed
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(graph, stream=side):
+                        st.decode_step(0, k_in, v_in, q_in, out, lse=lse, n_reserve=steps)
+                torch.cuda.current_stream().wait_stream(side)
+            graph.replay()
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        K, V = np.concatenate([K, kn], axis=1), np.concatenate([V, vn], axis=1)
+        assert int(st.seq_len[0, 0]) == wl.n + step + 1
+        want, _, want_lse, _ = pb.oracle_attn(q, attend, "f64", K, V, pb.Nc)
+        hz.check_output(b.bf16_to_bits(out), want, f"decode_step {attend}, step {step}")
+        assert np.abs(lse.cpu().numpy() - want_lse).max() <= 1e-3
+    Kd, Vd = pages_to_plain(st, 0, wl.n + steps)
+    assert np.array_equal(Kd, K) and np.array_equal(Vd, V)          # every token landed at its own position
+    # the same tokens through kvE_append_next + kvE_decode_attn on a second handle: same outputs bit for bit
+    st2 = make_store(wl, attend)
+    load_kv(st2, 0, pb.K, pb.V)
+    run_gpu_pipeline(st2, pb, 0, aw, lw)
+    for step in range(steps):
+        kn, vn = wlm.gen_new_tokens(wl, 0, step)
+        st2.append_next(0, b.bits_to_bf16(kn[:, 0]), b.bits_to_bf16(vn[:, 0]), n_reserve=steps)
+        out2 = st2.decode_attn(0, b.bits_to_bf16(wlm.gen_q(wl, 0, step)))
+    torch.cuda.synchronize()
+    assert torch.equal(out2, out)
+    # a full cache: the call is refused on the host once the handle's own count is at the limit
+    st.set_len(0, wl.max_tokens)
+    with pytest.raises(b.KveError) as e:
+        st.decode_step(0, k_in, v_in, q_in, out)
+    assert e.value.rc == -3
+
+
 @pytest.mark.parametrize("seed", list(range(12)) + [104])      # 104: nothing has left the window yet
 def test_whole_path_random_geometries(seed):
     """Seeded random small geometries (chunk size, window, length, gate width, aggregator, keep ratio, append
