@@ -288,8 +288,10 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   if (cfg->max_query_tokens > 0) {
     st->block_hp = attn_block_hp(cfg->C);
     st->block_split_cap = block_split_cap(st->S);
+    // maps over the page pools and over the compacted kept summary rows (all layers) in the workspace
+    char* ws0 = static_cast<char*>(buf->workspace);
     const cudaError_t em = encode_attn_block_maps(st->block_maps, buf->k_pages, buf->v_pages, (long long)buf->n_pages * cfg->C,
-                                                  st->block_hp, buf->ksum_bf16, buf->vsum_bf16,
+                                                  st->block_hp, ws0 + k.off_kept_k, ws0 + k.off_kept_v,
                                                   (long long)cfg->n_layers * st->S * st->max_chunks);
     if (em != cudaSuccess) {
       delete st;
@@ -298,7 +300,9 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
     st->block_ready = true;
   }
   st->layers.assign(cfg->n_layers, LayerState());
-  cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.off_kept_k - k.off_partials);
+  // partial records, tickets ... and the kept-row buffers (a box of the query-block kernel may reach past a sequence's
+  // kept count: what it finds there must be finite)
+  cudaError_t e = cudaMemset(static_cast<char*>(buf->workspace) + k.off_partials, 0, k.total - k.off_partials);
   if (e == cudaSuccess) e = cudaMemset(buf->status_word, 0, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(buf->seq_len, 0, sizeof(int32_t) * (size_t)cfg->n_layers * cfg->B);
   if (e == cudaSuccess) e = cudaMemset(buf->keep_cnt, 0, sizeof(int32_t) * (size_t)cfg->n_layers * st->S);

@@ -45,8 +45,8 @@ cudaError_t encode_attn_block_maps(void* maps, const void* k_pages, const void* 
   CUtensorMap* tm = static_cast<CUtensorMap*>(maps);
   cudaError_t e = encode_rows_map(tm + 0, k_pages, (unsigned long long)page_rows, (unsigned)hp);
   if (e == cudaSuccess) e = encode_rows_map(tm + 1, v_pages, (unsigned long long)page_rows, (unsigned)hp);
-  if (e == cudaSuccess) e = encode_rows_map(tm + 2, ksum, (unsigned long long)sum_rows, 1u);
-  if (e == cudaSuccess) e = encode_rows_map(tm + 3, vsum, (unsigned long long)sum_rows, 1u);
+  if (e == cudaSuccess) e = encode_rows_map(tm + 2, ksum, (unsigned long long)sum_rows, (unsigned)ATTN_BLOCK_SUM_BOX);
+  if (e == cudaSuccess) e = encode_rows_map(tm + 3, vsum, (unsigned long long)sum_rows, (unsigned)ATTN_BLOCK_SUM_BOX);
   return e;
 }
 

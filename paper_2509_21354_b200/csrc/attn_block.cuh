@@ -18,6 +18,7 @@ constexpr int BK_TILE = ATTN_TILE_ROWS;         // 64 rows per stage
 constexpr int BK_KBLOCK_BYTES = BK_TILE * 128;  // one K-block: 64 rows x 64 bf16
 constexpr int BK_TILE_BYTES = 2 * BK_KBLOCK_BYTES;        // K (or V) tile, 16 KB
 constexpr int BK_STAGE_BYTES = 2 * BK_TILE_BYTES;         // K tile then V tile
+constexpr int BK_SUM_BOX = ATTN_BLOCK_SUM_BOX;   // rows per tensor-copy box over the compacted kept summary rows
 constexpr int BK_REC = ATTN_PARTIAL_FLOATS;     // floats per (query row) record: acc[128], m, l, pad
 
 struct BlockArgs {
@@ -27,7 +28,7 @@ struct BlockArgs {
   int rec_rows;             // query-row records per (sequence, split) in `partials`
   int causal;               // query token t sees the cache up to its own position only
   int hp;                   // rows per page box
-  long long sum_row0;       // first row of this layer in the summary tensor maps
+  long long sum_row0;       // first row of this layer in the tensor maps over the compacted kept summary rows
   const uint16_t* q;        // [B][T][Hq][128]
   uint16_t* out;            // [B][T][Hq][128]
   float* lse;               // [B][T][Hq] or null
@@ -92,7 +93,7 @@ __device__ __forceinline__ long long q_row_offset(const BlockArgs& a, int s, int
 // (bounded) on empty[stage] before a stage is reused.
 // What a lane fetches for a tile: up to two boxes (K and V each, both 64-column halves):
 //   page tiles:    lane j < granules: hp rows from global row src[0] to tile row j * hp
-//   summary tiles: lane j: row j (src[0]) and row j + 32 (src[1]), one row each
+//   summary tiles: lane j < ceil(valid / 16): 16 kept summary rows (compacted by kvE_compact) from global row src[0]
 template <int STAGES>
 __device__ __forceinline__ void block_producer(const BlockArgs& a, const BlockGeom& gm, int s, int lane,
                                                const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmKs,
@@ -126,15 +127,8 @@ __device__ __forceinline__ void block_producer(const BlockArgs& a, const BlockGe
         t.src[0] = page_row(chunk, ll - ci * v.C);
       }
     } else {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int l = lane + 32 * h;
-        if (l < valid) {
-          int c = v.keep_idx[sb + (row0 - gm.tail_pad) + l];
-          if (c < 0 || c >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); c = 0; }
-          t.src[h] = (int)(a.sum_row0 + sb + c);
-        }
-      }
+      // kept summary rows sit compacted, one contiguous run per sequence: boxes of BK_SUM_BOX rows, lane j the j-th
+      if (lane * BK_SUM_BOX < valid) t.src[0] = (int)(a.sum_row0 + sb + (row0 - gm.tail_pad) + lane * BK_SUM_BOX);
     }
   };
   auto issue = [&](int i, const TileSrc& t) -> bool {
@@ -147,7 +141,7 @@ __device__ __forceinline__ void block_producer(const BlockArgs& a, const BlockGe
     const int valid = gm.rows_valid(row0);
     const bool pages = row0 < gm.tail_pad || a.mode == ATTN_RAW;
     const uint32_t bytes = pages ? (uint32_t)((valid + a.hp - 1) / a.hp) * a.hp * 2u * ROW_BYTES
-                                 : (uint32_t)valid * 2u * ROW_BYTES;
+                                 : (uint32_t)((valid + BK_SUM_BOX - 1) / BK_SUM_BOX) * BK_SUM_BOX * 2u * ROW_BYTES;
     if (lane == 0) mbar_arrive_expect_tx(&full[stage], bytes);
     __syncwarp();
     const uint32_t kdst = smem_u32(ring + stage * BK_STAGE_BYTES), vdst = kdst + BK_TILE_BYTES;
@@ -159,17 +153,13 @@ __device__ __forceinline__ void block_producer(const BlockArgs& a, const BlockGe
         tma_load_2d(vdst + off, tmV, 0, t.src[0], &full[stage]);
         tma_load_2d(vdst + BK_KBLOCK_BYTES + off, tmV, 64, t.src[0], &full[stage]);
       }
-    } else {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (t.src[h] >= 0) {
-          const uint32_t off = (uint32_t)(lane + 32 * h) * 128u;
-          tma_load_2d(kdst + off, tmKs, 0, t.src[h], &full[stage]);
-          tma_load_2d(kdst + BK_KBLOCK_BYTES + off, tmKs, 64, t.src[h], &full[stage]);
-          tma_load_2d(vdst + off, tmVs, 0, t.src[h], &full[stage]);
-          tma_load_2d(vdst + BK_KBLOCK_BYTES + off, tmVs, 64, t.src[h], &full[stage]);
-        }
-      }
+    } else if (t.src[0] >= 0) {
+      // rows beyond the kept count inside the last box are older kept rows or zeros (finite), masked by the row count
+      const uint32_t off = (uint32_t)(lane * BK_SUM_BOX) * 128u;
+      tma_load_2d(kdst + off, tmKs, 0, t.src[0], &full[stage]);
+      tma_load_2d(kdst + BK_KBLOCK_BYTES + off, tmKs, 64, t.src[0], &full[stage]);
+      tma_load_2d(vdst + off, tmVs, 0, t.src[0], &full[stage]);
+      tma_load_2d(vdst + BK_KBLOCK_BYTES + off, tmVs, 64, t.src[0], &full[stage]);
     }
     return true;
   };

@@ -94,7 +94,8 @@ cudaError_t launch_selftest_timeout(int which, int32_t* status, cudaStream_t st)
 
 // block-of-queries attention (grouped query heads x query tokens), tensor-map fed
 constexpr int ATTN_BLOCK_MAX_ROWS = 128;       // query rows (tokens x heads per KV head) per KV sequence
-constexpr int ATTN_BLOCK_MAP_BYTES = 128;      // one tensor map; a handle keeps four (K pages, V pages, K summaries, V summaries)
+constexpr int ATTN_BLOCK_MAP_BYTES = 128;      // one tensor map; a handle keeps four (K pages, V pages, kept K summaries, kept V summaries)
+constexpr int ATTN_BLOCK_SUM_BOX = 16;         // rows per box of the maps over the compacted kept summary rows
 int attn_block_hp(int C);                      // rows per page box: largest power of two <= 64 dividing C
 cudaError_t encode_attn_block_maps(void* maps, const void* k_pages, const void* v_pages, long long page_rows, int hp,
                                    const void* ksum, const void* vsum, long long sum_rows);
