@@ -185,10 +185,11 @@ bool wrong_device(const kvE_store* st) {
 
 // How an attention launch is cut up.  Every sequence is cut into k equal parts and CTA c of G takes the contiguous
 // run of parts [c S k / G, (c + 1) S k / G), which it streams as one piece (no break between parts of one sequence).
-// G is one resident wave at most (two CTAs per SM).  k is chosen by a small cost model in units of 64-row tiles: the
-// busiest CTA's tiles, plus two tiles' worth of time for the exchange through global memory that is needed as soon as
-// a sequence is shared between CTAs (k > 1).  Small k keeps whole sequences together; large k evens out the bytes per
-// CTA when S is not a multiple of the wave.
+// G is one resident wave at most (two CTAs per SM).  k is chosen by a small cost model in microseconds, fitted to
+// measurements: a CTA takes about 1.4 us per 64-row tile whether it shares its SM or not (its eight consumer warps set
+// that pace; two CTAs per SM are what saturates HBM), so the launch lasts as long as the busiest CTA's tiles, plus its
+// end: about 0.5 us when every CTA owns whole sequences (k = 1), about 3.5 us and growing with the number of records
+// when sequences are shared and the last ones go through global memory (record, fence, ticket, merge).
 struct AttnCut { int k, grid; };
 AttnCut attention_cut(const kvE_store* st, AttnMode mode, const LayerState& ls) {
   const long long n_upper = ls.reserve_upper > ls.n_tokens ? ls.reserve_upper : ls.n_tokens;
@@ -202,20 +203,22 @@ AttnCut attention_cut(const kvE_store* st, AttnMode mode, const LayerState& ls) 
   if (tiles < 1) tiles = 1;
   const long long G = st->attn_grid_max, S = st->S;
   const long long k_max = tiles < MAX_SPLITS ? tiles : MAX_SPLITS;
-  AttnCut cut{1, 1};
-  double best = 1e30;
-  for (long long k = 1; k <= k_max; ++k) {
-    if (S * k * (G + 1) >= (1LL << 32)) break;                          // the kernel cuts the parts up in 32-bit arithmetic
+  auto cost_of = [&](long long k, long long* grid_out) {
     const long long parts = S * k, grid = parts < G ? parts : G;
     const long long rounds = (parts + grid - 1) / grid;                 // parts of the busiest CTA
-    const double cost = (double)rounds * (double)tiles / (double)k + (k > 1 ? 2.0 : 0.0);
-    if (cost < best - 0.25 || (cost <= best + 1e-9 && k > 1)) {         // ties go to the finer cut (evener bytes)
-      best = cost < best ? cost : best;
-      cut.k = (int)k;
-      cut.grid = (int)grid;
-    }
-  }
-  return cut;
+    if (grid_out) *grid_out = grid;
+    return (double)rounds * (double)tiles / (double)k * 1.4 + (k > 1 ? 4.5 + 0.06 * (double)k : 0.5);
+  };
+  // the kernel cuts the parts up in 32-bit arithmetic: S k (G + 1) must stay below 2^32
+  double best = 1e30;
+  for (long long k = 1; k <= k_max && S * k * (G + 1) < (1LL << 32); ++k)
+    if (cost_of(k, nullptr) < best) best = cost_of(k, nullptr);
+  long long k_pick = 1;      // whole sequences only when that is the cheapest; else near-ties go to the finer cut (evener bytes per CTA)
+  for (long long k = 2; k <= k_max && S * k * (G + 1) < (1LL << 32); ++k)
+    if (cost_of(k, nullptr) <= best + 0.3 && cost_of(1, nullptr) > best + 1e-9) k_pick = k;
+  long long grid = 1;
+  cost_of(k_pick, &grid);
+  return AttnCut{(int)k_pick, (int)grid};
 }
 
 struct KeptRows { void *k, *v; };      // kept summary rows of a layer, compacted by kvE_compact
