@@ -173,7 +173,10 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
              const kvE_lstm_weights* w, void* stream);
 
 /* Sec. 3.2 retention rule: keep chunk t iff scores[t] >= tau, over all gated chunks of `layer`;
- * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw. */
+ * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw.  Also copies the kept
+ * chunks' summary rows into one contiguous run per sequence (workspace), which is what attention reads, and records
+ * on the device how many chunks the list covers: kvE_decode_attn / kvE_decode_step read that count from the device,
+ * so one of their launches captured in a CUDA graph keeps serving after later triggers without a new capture. */
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream);
 
 /* Sec. 3.3, the whole aggregation-and-gating step of `layer` from scratch in one call: summaries of every chunk

@@ -28,7 +28,7 @@ struct kvE_store {
   int device = -1;       // the device that was current at kvE_create: owner of every buffer; calls check it
   int S, max_chunks;
   // workspace carve-up (byte offsets)
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, ws_needed;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, off_listed, ws_needed;
   int attn_grid_max;     // most CTAs an attention launch uses (two per SM of the handle's device): sizes the partial records
   // block-of-queries attention: tensor maps over the page pools and the summary store (encoded at
   // create when cfg.max_query_tokens > 0), rows per page box, split cap the workspace was sized for
@@ -87,7 +87,7 @@ int check_config(const kvE_config* c) {
 }
 
 struct Carve {
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, total;
+  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, off_listed, total;
 };
 // most CTAs of one attention launch: two resident per SM (148 SMs assumed where no device can be asked)
 int attn_grid_cap() {
@@ -124,6 +124,7 @@ Carve carve(const kvE_config& c) {
   const size_t sum_bytes = (size_t)c.n_layers * S * max_chunks * 128 * 2;
   k.off_kept_k = o;   o = align_up(o + sum_bytes);
   k.off_kept_v = o;   o = align_up(o + sum_bytes);
+  k.off_listed = o;   o = align_up(o + (size_t)c.n_layers * sizeof(int32_t));      // per layer: chunks the keep list covers
   k.total = o;
   return k;
 }
@@ -169,6 +170,7 @@ LayerView view(const kvE_store* st, int layer) {
   v.lstm_h = b.lstm_h + L * S * c.d_g;
   v.lstm_c = b.lstm_c + L * S * c.d_g;
   v.status = b.status_word;
+  v.n_listed = reinterpret_cast<int32_t*>(static_cast<char*>(b.workspace) + st->off_listed) + layer;
   v.B = c.B; v.H = c.Hkv; v.S = st->S; v.C = c.C; v.max_chunks = st->max_chunks; v.max_tokens = c.max_tokens;
   return v;
 }
@@ -252,6 +254,15 @@ void release_host_objects(kvE_store* st) {
     for (cudaEvent_t e : st->ev) cudaEventDestroy(e);
 }
 
+// the keep list no longer covers chunks from `value` on (their summaries or scores changed): host count and device count
+int lower_listed(kvE_store* st, int layer, int value, cudaStream_t stream) {
+  LayerState& ls = st->layers[layer];
+  if (ls.n_compacted <= value) return KVE_OK;
+  ls.n_compacted = value;
+  cudaError_t e = launch_set_listed(view(st, layer), value, stream);
+  return e == cudaSuccess ? KVE_OK : cuda_fail(st, e);
+}
+
 }  // namespace
 
 extern "C" {
@@ -285,7 +296,7 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
   st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
   st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_ticket = k.off_ticket; st->off_block = k.off_block;
-  st->off_kept_k = k.off_kept_k; st->off_kept_v = k.off_kept_v; st->ws_needed = k.total;
+  st->off_kept_k = k.off_kept_k; st->off_kept_v = k.off_kept_v; st->off_listed = k.off_listed; st->ws_needed = k.total;
   st->attn_grid_max = attn_grid_cap();
   if ((size_t)st->attn_grid_max > ATTN_GRID_LIMIT) st->attn_grid_max = (int)ATTN_GRID_LIMIT;
   if (cfg->max_query_tokens > 0) {
@@ -361,12 +372,13 @@ int kvE_set_len(kvE_store* st, int layer, int n, void* stream) {
   if (bad_layer(st, layer) || n < 0) return KVE_ERR_ARG;
   if (wrong_device(st)) return KVE_ERR_STATE;
   if (n > st->cfg.max_tokens) return KVE_ERR_CAPACITY;
-  cudaError_t e = launch_set_len(view(st, layer), n, static_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return cuda_fail(st, e);
   LayerState& ls = st->layers[layer];
+  const int nc = stale_chunks(st->cfg, n);
+  // a keep list that reaches past the new stale range is dropped, on the device too (-1: leave the device's count alone)
+  cudaError_t e = launch_set_len(view(st, layer), n, ls.n_compacted > nc ? 0 : -1, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_tokens = n;
   ls.reserve_upper = 0;
-  const int nc = stale_chunks(st->cfg, n);
   if (ls.n_summarised > nc) ls.n_summarised = nc;
   if (ls.n_gated > nc) ls.n_gated = 0;          // the carried LSTM state is past the cut: gate again from chunk 0
   if (ls.n_compacted > nc) {
@@ -426,8 +438,7 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   if (chunk_begin <= ls.n_summarised && chunk_end > ls.n_summarised) ls.n_summarised = chunk_end;
-  if (ls.n_compacted > chunk_begin) ls.n_compacted = chunk_begin;   // the compacted copies of these summaries are stale
-  return KVE_OK;
+  return lower_listed(st, layer, chunk_begin, s);                   // the compacted copies of these summaries are stale
 }
 
 int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE_lstm_weights* w, void* stream) {
@@ -457,8 +468,7 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_gated = chunk_end;
-  if (ls.n_compacted > chunk_begin) ls.n_compacted = chunk_begin;   // scores changed under the keep list
-  return KVE_OK;
+  return lower_listed(st, layer, chunk_begin, s);                   // scores changed under the keep list
 }
 
 int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {

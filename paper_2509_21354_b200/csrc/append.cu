@@ -74,11 +74,12 @@ __global__ void __launch_bounds__(256) kve_append_next_kernel(LayerView v, const
   if (threadIdx.x == 0) *ticket = 0;      // clean for the next launch
 }
 
-__global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n) {
+__global__ void kve_set_len_kernel(int32_t* seq_len, int B, int n, int32_t* n_listed, int listed) {
   pdl_launch_dependents();
   pdl_wait();
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) seq_len[b] = n;
+  if (b == 0 && listed >= 0) *n_listed = listed;
 }
 
 cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, int pos0, cudaStream_t st) {
@@ -98,8 +99,18 @@ cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void
                     static_cast<const uint4*>(v_new), n_new, ticket);
 }
 
-cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st) {
-  return launch_pdl(kve_set_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n);
+__global__ void kve_set_listed_kernel(int32_t* n_listed, int listed) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) *n_listed = listed;
+}
+
+cudaError_t launch_set_listed(const LayerView& v, int n_listed, cudaStream_t st) {
+  return launch_pdl(kve_set_listed_kernel, dim3(1), dim3(32), 0, st, v.n_listed, n_listed);
+}
+
+cudaError_t launch_set_len(const LayerView& v, int n, int n_listed, cudaStream_t st) {
+  return launch_pdl(kve_set_len_kernel, dim3((v.B + 127) / 128), dim3(128), 0, st, v.seq_len, v.B, n, v.n_listed, n_listed);
 }
 
 }  // namespace kve

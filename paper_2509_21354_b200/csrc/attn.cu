@@ -79,7 +79,8 @@ constexpr int TF_END = 4;      // no tile: the CTA's work is done
 
 struct AttnArgs {
   LayerView v;
-  int mode, n_chunks;
+  int mode;
+  int n_chunks;                // the host's count of chunks under the keep list: a prefetch hint; the kernel reads the device's
   int k;                       // parts per sequence
   const uint16_t* q;
   uint16_t* out;
@@ -99,6 +100,7 @@ struct AttnArgs {
 struct AttnGeo {
   int n_tail, raw0, TT, per;   // tail rows / tiles per sequence; rows a kept chunk contributes
   int n;                       // tokens attended to (the new one included when one is being appended)
+  int n_chunks;                // chunks the keep list covers (0 for full-cache attention)
   bool appending;              // the last tail row of every sequence is the new token, taken from k_new / v_new
   uint32_t I, P;               // parts in the launch (S k); CTAs that get any (min(G, I): none of them is empty)
 };
@@ -126,8 +128,8 @@ __device__ __forceinline__ void prefetch_sequence_metadata(const AttnArgs& a, in
 
 // rows the kept chunks of sequence s contribute
 __device__ __forceinline__ int lead_rows_of(const AttnArgs& a, const AttnGeo& g, int s) {
-  if (a.mode == ATTN_DENSE || a.n_chunks <= 0) return 0;
-  const int M = min(max(a.v.keep_cnt[s], 0), a.n_chunks);
+  if (a.mode == ATTN_DENSE || g.n_chunks <= 0) return 0;
+  const int M = min(max(a.v.keep_cnt[s], 0), g.n_chunks);
   return M * g.per;
 }
 
@@ -194,7 +196,10 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
     if (a.k_new != nullptr && !g.appending && blockIdx.x == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);   // cache full
     if (g.appending) n += 1;
     g.n = n;
-    g.raw0 = (a.mode == ATTN_DENSE) ? 0 : a.n_chunks * v.C;
+    // chunks the keep list covers: the device's own count, so that a launch replayed from a CUDA graph follows the
+    // gate triggers that happened since it was captured (the launch argument is only the host's view at capture time)
+    g.n_chunks = (a.mode == ATTN_DENSE) ? 0 : min(max(*v.n_listed, 0), v.max_chunks);
+    g.raw0 = g.n_chunks * v.C;
     g.n_tail = max(0, n - g.raw0);
     g.TT = (g.n_tail + AT_TILE - 1) / AT_TILE;
     g.per = (a.mode == ATTN_RAW) ? v.C : 1;
@@ -278,7 +283,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
           const int ci = L / v.C;
           r = L - ci * v.C;
           chunk = v.keep_idx[sb + ci];
-          if (chunk < 0 || chunk >= a.n_chunks) { set_status(v.status, ERR_CAPACITY); chunk = 0; }
+          if (chunk < 0 || chunk >= g.n_chunks) { set_status(v.status, ERR_CAPACITY); chunk = 0; }
         }
         long long page = v.page_table[sb + chunk];
         if (page < 0 || page >= v.n_pages) { set_status(v.status, ERR_CAPACITY); page = 0; }

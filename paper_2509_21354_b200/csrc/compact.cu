@@ -26,6 +26,7 @@ __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_kernel(LayerVi
   }
   for (int t = base + lane; t < v.max_chunks; t += 32) idx[t] = -1;
   if (lane == 0) v.keep_cnt[s] = base;
+  if (s == 0 && lane == 0) *v.n_listed = n_chunks;      // what the attention kernel reads: the list covers chunks [0, n_chunks)
 }
 
 // ---- what attention wants from a fresh keep list ---------------------------------------------------------
@@ -118,6 +119,7 @@ __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_topk_kernel(La
   }
   for (int t = base + lane; t < v.max_chunks; t += 32) idx[t] = -1;
   if (lane == 0) v.keep_cnt[s] = base;
+  if (s == 0 && lane == 0) *v.n_listed = n_chunks;
 }
 
 cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, void* kkept, void* vkept, cudaStream_t st) {

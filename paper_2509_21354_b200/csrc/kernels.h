@@ -44,6 +44,7 @@ struct LayerView {
   float* lstm_h;              // [S][d_g]
   float* lstm_c;
   int32_t* status;
+  int32_t* n_listed;          // one int: chunks [0, *n_listed) are covered by the keep list (device copy of the handle's count)
   int B, H, S, C, max_chunks, max_tokens;
 };
 
@@ -63,7 +64,9 @@ constexpr int ATTN_TILE_ROWS = 64;
 constexpr int ATTN_PARTIAL_FLOATS = 132;       // acc[128], m, l, 2 pad: keeps every record 16-byte aligned
 
 cudaError_t launch_append(const LayerView& v, const void* k_new, const void* v_new, int n_new, int pos0, cudaStream_t st);
-cudaError_t launch_set_len(const LayerView& v, int n, cudaStream_t st);
+cudaError_t launch_set_listed(const LayerView& v, int n_listed, cudaStream_t st);      // the device copy of the keep list's coverage
+// n_listed >= 0: also set the device copy of the keep list's coverage to it
+cudaError_t launch_set_len(const LayerView& v, int n, int n_listed, cudaStream_t st);
 cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, int32_t* ticket,
                                cudaStream_t st);
 cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st);

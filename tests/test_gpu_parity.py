@@ -564,8 +564,8 @@ def test_long_gate_chain_two_and_three_planes():
 
 
 def test_streaming_soak_reuses_reclaimed_pages_over_several_triggers():
-    """Sec. 3.3 as it runs: tokens arrive one by one (append at the device-held length + attention, replayed from one
-    CUDA graph); every C tokens a chunk leaves the window: true length to the host, that ONE chunk summarised and gated
+    """Sec. 3.3 as it runs: tokens arrive one by one (kvE_decode_step: append at the device-held length + attention in one
+    launch, captured ONCE in a CUDA graph and replayed for the whole run); every C tokens a chunk leaves the window: true length to the host, that ONE chunk summarised and gated
     with the carried (h, c), keep list rebuilt, the pages of all gated chunks handed back, and the freed pages given to
     the chunks that fill next.  After every trigger: attention against the oracle on the grown cache, the raw tail
     read back through the page table, the pages really re-used, status word clean."""
@@ -600,6 +600,14 @@ def test_streaming_soak_reuses_reclaimed_pages_over_several_triggers():
         return pb.o64.attn(q, np.ascontiguousarray(K[:, :n_now]), np.ascontiguousarray(V[:, :n_now]), C_, nc_now, idx, cnt,
                            pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)[0]
 
+    # ONE graph for the whole run: the step appends at the length the device holds and reads the number of chunks under the
+    # keep list from the device too, so the triggers that happen between replays need no new capture
+    graph = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            st.decode_step(0, k_in, v_in, q_in, out, n_reserve=n_triggers * C_)
+    torch.cuda.current_stream().wait_stream(side)
     for trig in range(n_triggers):
         # ---- hand back the pages of every gated chunk, give them to the chunks that fill next ----
         free_list, free_count = st.reclaim_pages(0, 0, nc, mode="gated")
@@ -613,14 +621,7 @@ def test_streaming_soak_reuses_reclaimed_pages_over_several_triggers():
         reused += S
         st.page_table[0].copy_(pt)
         next_slot += 1
-        # ---- C decode steps between two triggers, replayed from one graph ----
-        graph = torch.cuda.CUDAGraph()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(graph, stream=side):
-                st.append_next(0, k_in, v_in, n_reserve=C_)
-                st.decode_attn(0, q_in, out)
-        torch.cuda.current_stream().wait_stream(side)
+        # ---- C decode steps between two triggers: replays of the one graph ----
         for step in range(C_):
             q = wlm.gen_q(wl_full, 0, 1000 * trig + step)
             k_in.copy_(b.bits_to_bf16(K[:, n])); v_in.copy_(b.bits_to_bf16(V[:, n])); q_in.copy_(b.bits_to_bf16(q))
