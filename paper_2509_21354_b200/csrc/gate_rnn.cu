@@ -35,6 +35,27 @@
 
 namespace kve {
 
+// Optional cycle budget of one recurrence step (build with -DKVE_RNN_STAMPS, see rnn_stamps.py): warp 0 of CTA 0 adds
+// up, over all steps and groups, the clock64 cycles between five points of a step - 0: waiting for the peers' h,
+// 1: fragment loads + MMA chain, 2: prefetch of the next step's P, 3: cell update and plane split, 4: sending h,
+// 6: from the end of one round to the start of the next (the loaded P moves into place, barrier bookkeeping) - and
+// slot 5 counts the (step, group) rounds.  The marks are contiguous: the slots add up to the whole step loop.  Compiled out of the product library.
+#ifdef KVE_RNN_STAMPS
+__device__ unsigned long long g_rnn_cycles[8];
+#define KVE_RNN_MARK(slot)                                                                   \
+  do {                                                                                       \
+    if (blockIdx.x == 0 && warp == 0 && lane == 0) {                                         \
+      const long long now_ = clock64();                                                      \
+      atomicAdd(&g_rnn_cycles[slot], (unsigned long long)(now_ - mark_));                    \
+      mark_ = now_;                                                                          \
+    }                                                                                        \
+  } while (0)
+#define KVE_RNN_MARK_BEGIN() long long mark_ = clock64()
+#else
+#define KVE_RNN_MARK(slot) do { } while (0)
+#define KVE_RNN_MARK_BEGIN() do { } while (0)
+#endif
+
 // NG independent groups of 8 sequences per cluster.  A group is one pipeline (own h buffers, barriers,
 // staging and cell state); a warp works through the groups one after the other within a step, so
 // while group A's new h is on its way between the CTAs the warp is busy with group B.
@@ -130,6 +151,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   cluster_sync_all();
 
   bool alive = true;
+  KVE_RNN_MARK_BEGIN();
   for (int step = 0; step < a.n_range && alive; ++step) {
     const int buf = step & 1;
     const bool send_h = step + 1 < a.n_range;
@@ -144,6 +166,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       uint16_t* my_stage = stage + (gi * RNN_WARPS + warp) * STG_WARP;
       uint64_t* hbar_g = hbar + 2 * gi;
       const int seq_g = seq0 + gi * NS;
+      KVE_RNN_MARK(6);
       if (step > 0) {
         // h_{t-1} of this group from every CTA of the cluster (each buffer completes once per two steps)
         if (!mbar_wait_cluster_bounded(&hbar_g[buf], ((step - 1) >> 1) & 1)) {
@@ -154,6 +177,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         if (!alive) break;
       }
 
+      KVE_RNN_MARK(0);
       // ---- W_hh h_{t-1} on the tensor cores: one accumulator set per plane ---------------------------
       float acc[PL][2 * MP][4];
 #pragma unroll
@@ -185,6 +209,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
               mma_bf16_16816(acc[pl][mt], A[mt][2 * kp + half], bf[cur][pl][2 * half], bf[cur][pl][2 * half + 1]);
       }
 
+      KVE_RNN_MARK(1);
       // ---- P_{t+1} into registers while the MMAs drain ----------------------------------------------------
       float pnext[MP][4][2];
 #pragma unroll
@@ -203,6 +228,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           }
         }
 
+      KVE_RNN_MARK(2);
       // ---- cell update (thread-local), planes of h_t into the warp's staging area ---------------------
       asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       __syncwarp();      // earlier copies have read the staging areas
@@ -241,6 +267,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           }
         }
       }
+      KVE_RNN_MARK(3);
       // ---- the warp's k-blocks (8 units each: [plane][sequence][8], contiguous) to every CTA of the cluster ----
       if (send_h) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // staging writes -> visible to the bulk copies
@@ -261,6 +288,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         if (lane == 0) mbar_arrive(&hbar_g[buf ^ 1]);     // release: this warp's local pieces are in place
       }
 
+      KVE_RNN_MARK(4);
+#ifdef KVE_RNN_STAMPS
+      if (blockIdx.x == 0 && warp == 0 && lane == 0) atomicAdd(&g_rnn_cycles[5], 1ull);
+#endif
 #pragma unroll
       for (int p = 0; p < MP; ++p)
 #pragma unroll
@@ -354,3 +385,14 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
 }
 
 }  // namespace kve
+
+#ifdef KVE_RNN_STAMPS
+// instrumented build only: read and clear the cycle sums
+extern "C" int kve_rnn_cycles_read(unsigned long long* host) {
+  cudaError_t e = cudaMemcpyFromSymbol(host, kve::g_rnn_cycles, sizeof(kve::g_rnn_cycles));
+  void* p = nullptr;
+  if (e == cudaSuccess) e = cudaGetSymbolAddress(&p, kve::g_rnn_cycles);
+  if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(kve::g_rnn_cycles));
+  return (int)e;
+}
+#endif
