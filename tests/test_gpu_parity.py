@@ -159,6 +159,22 @@ def test_gate_sizes_and_chunk_sizes(d_g, C):
     full_check(wl, "summary")
 
 
+@pytest.mark.parametrize("d_g,B,H", [(64, 37, 33), (256, 9, 35)])
+def test_two_sequence_groups_per_cluster(d_g, B, H):
+    # more sequences than one group of 8 per cluster places in one wave: every cluster walks two groups, with
+    # the rounds of the two software-pipelined; S is ragged against 16 (a cluster's last group is partly or wholly empty)
+    wl = wlm.Workload("groups", B=B, H=H, n=9 * 16 + 40, C=16, W=32, d_g=d_g, agg="mean", key_offset_std=0.5, seed=d_g + B)
+    assert wl.S > 8 * (148 if d_g == 64 else 37)
+    st, pb, _, lstm_w = full_check(wl, "summary")
+    # one chunk at a time with the carried state: the same scores as the whole range
+    want = st.scores[0].clone()
+    for t in range(pb.Nc):
+        st.gate(0, t, t + 1, lstm_w)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    assert torch.equal(st.scores[0, :, :pb.Nc], want[:, :pb.Nc])
+
+
 def test_chunk_of_one_identity_keep_all_is_dense():
     # C = 1 with identity aggregation and tau = 0: the summary path reproduces dense attention
     b = _binding()
