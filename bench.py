@@ -546,33 +546,46 @@ def measure_config(rig, peaks, peak_kind, flush, headline=False):
 
 def trigger_leg(wl, attend, seed, steady_ms, n_triggers=24):
     """The aggregation-and-gating step of Sec. 3.3 as it happens while decoding: C more tokens have arrived, ONE chunk
-    per sequence leaves the window; it is summarised, takes one LSTM step with the carried (h, c), and the keep list
-    is rebuilt.  Timed per trigger (events around the three calls), n_triggers triggers in a row on a growing cache."""
+    per sequence leaves the window; it is summarised, takes one LSTM step with the carried (h, c), and joins the keep
+    list.  Timed per trigger (events around the calls), n_triggers triggers in a row on a growing cache, in two forms:
+    kvE_summarize_chunks + kvE_gate_next (the LSTM step, the score and the keep-list append in one launch) and the
+    general calls kvE_summarize_chunks + kvE_gate + kvE_compact (projection GEMM, recurrence, score head, compaction
+    and kept-row gather as separate launches)."""
     import torch
-    rig = Rig(wl, attend, seed, extra_tokens=(n_triggers + 1) * wl.C)
-    st = rig.st
-    kC = torch.randn((wl.S, wl.C, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-    vC = torch.randn((wl.S, wl.C, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-    ts = []
-    for i in range(n_triggers):
-        ready = st.append(0, kC, vC)
-        assert ready == 1
-        t = rig.Nc + i
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        st.summarize_chunks(0, t, t + 1, rig.aw)
-        st.gate(0, t, t + 1, rig.lw)
-        st.compact(0, wl.tau)
-        e1.record()
-        torch.cuda.synchronize()
-        if i >= 4:
-            ts.append(e0.elapsed_time(e1))
-    assert st.poll_status() == 0
-    trig = float(np.median(ts))
-    return {"what": "one chunk per sequence leaves the window: kvE_summarize_chunks(t, t+1) + kvE_gate(t, t+1) with carried "
-                    "state + kvE_compact, per layer; the amortised step spreads it over the C tokens between two triggers",
-            "trigger_ms": trig, "triggers_timed": len(ts), "steady_ms": steady_ms, "C": wl.C,
+    out = {}
+    for form in ("gate_next", "general"):
+        rig = Rig(wl, attend, seed, extra_tokens=(n_triggers + 1) * wl.C)
+        st = rig.st
+        kC = torch.randn((wl.S, wl.C, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        vC = torch.randn((wl.S, wl.C, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        ts = []
+        for i in range(n_triggers):
+            ready = st.append(0, kC, vC)
+            assert ready == 1
+            t = rig.Nc + i
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            st.summarize_chunks(0, t, t + 1, rig.aw)
+            if form == "gate_next":
+                st.gate_next(0, rig.lw, wl.tau)
+            else:
+                st.gate(0, t, t + 1, rig.lw)
+                st.compact(0, wl.tau)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 4:
+                ts.append(e0.elapsed_time(e1))
+        assert st.poll_status() == 0
+        out[form] = float(np.median(ts))
+        n_timed = len(ts)
+        st.close()
+    trig = out["gate_next"]
+    return {"what": "one chunk per sequence leaves the window: kvE_summarize_chunks(t, t+1) + kvE_gate_next (one LSTM step with "
+                    "carried state, score, keep-list append: one launch), per layer; the amortised step spreads it over the C "
+                    "tokens between two triggers",
+            "trigger_ms": trig, "trigger_ms_with_gate_and_compact": out["general"], "triggers_timed": n_timed,
+            "steady_ms": steady_ms, "C": wl.C,
             "amortised_ms_per_token": (wl.C * steady_ms + trig) / wl.C,
             "amortised_steps_per_s": 1e3 * wl.C / (wl.C * steady_ms + trig),
             "trigger_share_of_amortised_step": trig / (wl.C * steady_ms + trig)}

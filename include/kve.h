@@ -172,6 +172,16 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
 int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
              const kvE_lstm_weights* w, void* stream);
 
+/* Sec. 3.3, the gate's part of a trigger while decoding: ONE more chunk per sequence has left the window and has been
+ * summarised.  Gates chunk t = (number of chunks gated so far) with the carried (h, c) (Eq. 3), writes scores[t] and
+ * brings the keep list for `tau` up to date (Sec. 3.2): like kvE_gate(t, t + 1) + kvE_compact(tau).  When the keep
+ * list already covers chunks [0, t) under the same tau (kvE_compact, kvE_refresh or earlier calls of this one; t > 0)
+ * all of it is ONE launch: the LSTM step on the new summary, the score, and chunk t appended to keep_idx / keep_cnt
+ * and to the compacted summary rows; otherwise it runs the two calls.  The single launch sums in another order than
+ * kvE_gate: its scores agree with kvE_gate's to rounding (1e-6), not bit for bit.  KVE_ERR_STATE if chunk t has not
+ * been summarised.  Timed under KVE_K_GATE_RNN. */
+int kvE_gate_next(kvE_store* st, int layer, const kvE_lstm_weights* w, float tau, void* stream);
+
 /* Sec. 3.2 retention rule: keep chunk t iff scores[t] >= tau, over all gated chunks of `layer`;
  * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw.  Also copies the kept
  * chunks' summary rows into one contiguous run per sequence (workspace), which is what attention reads, and records

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libkve.so")
-SOURCES = ["api.cu", "append.cu", "summarize.cu", "summarize_token.cu", "gate_proj.cu", "gate_rnn.cu", "compact.cu", "attn.cu", "attn_block.cu", "attn_block_tc.cu", "selftest.cu"]
+SOURCES = ["api.cu", "append.cu", "summarize.cu", "summarize_token.cu", "gate_proj.cu", "gate_rnn.cu", "gate_step.cu", "compact.cu", "attn.cu", "attn_block.cu", "attn_block_tc.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -485,6 +485,31 @@ int kvE_compact(kvE_store* st, int layer, float tau, void* stream) {
   return KVE_OK;
 }
 
+int kvE_gate_next(kvE_store* st, int layer, const kvE_lstm_weights* w, float tau, void* stream) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
+  if (!w || !w->W_ih || !w->W_hh || !w->b_ih || !w->b_hh || !w->w_s) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  const int t = ls.n_gated;
+  if (t >= ls.n_summarised) return KVE_ERR_STATE;
+  if (t == 0 || ls.n_compacted != t || ls.by_topk || ls.tau != tau) {      // no list to append to: the general path
+    const int rc = kvE_gate(st, layer, t, t + 1, w, stream);
+    return rc != KVE_OK ? rc : kvE_compact(st, layer, tau, stream);
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const KeptRows kr = kept_rows(st, layer);
+  cudaError_t e;
+  {
+    Prof prof(st, KVE_K_GATE_RNN, s);
+    e = launch_gate_step(view(st, layer), t, static_cast<const uint16_t*>(w->W_ih), static_cast<const uint16_t*>(w->W_hh),
+                         w->b_ih, w->b_hh, w->w_s, w->b_s, tau, st->cfg.d_g, st->gate_planes,
+                         static_cast<uint16_t*>(kr.k), static_cast<uint16_t*>(kr.v), s);
+  }
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  ls.n_gated = ls.n_compacted = t + 1;
+  return KVE_OK;
+}
+
 int kvE_refresh(kvE_store* st, int layer, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, void* stream) {
   if (bad_layer(st, layer)) return KVE_ERR_ARG;
   const int nc = stale_chunks(st->cfg, st->layers[layer].n_tokens);

@@ -79,6 +79,11 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
 // planes: bf16 planes of the fp32 state h that enter the recurrent product (2, or 3 = exact products)
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
                             int d_g, float* P, bool reset_state, int planes, cudaStream_t st);
+// one LSTM step on chunk t with the carried state, its score, and chunk t appended to the keep list for tau (which must
+// cover chunks [0, t)), its summary rows appended to kkept / vkept, the device's coverage count set to t + 1
+cudaError_t launch_gate_step(const LayerView& v, int t, const uint16_t* W_ih, const uint16_t* W_hh, const float* b_ih,
+                             const float* b_hh, const float* w_s, float b_s, float tau, int d_g, int planes,
+                             uint16_t* kept_k, uint16_t* kept_v, cudaStream_t st);
 // both also leave the kept chunks' summary rows compacted in kkept / vkept [S][max_chunks][128] bf16, which is
 // what attention reads until the next keep list
 cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, void* kkept, void* vkept, cudaStream_t st);

@@ -331,6 +331,57 @@ def test_refresh_equals_the_stepwise_calls(agg):
     assert st.poll_status() == 0 and torch.equal(st.scores[0], got[0])
 
 
+@pytest.mark.parametrize("d_g,agg,planes,B,H", [(256, "mlp", 2, 3, 5), (256, "mean", 3, 3, 5), (128, "mean", 2, 3, 5), (64, "mean", 2, 3, 5),
+                                                  (64, "max", 3, 3, 5),
+                                                  # more groups of 8 sequences than clusters in a wave: 2 and 4 groups per cluster
+                                                  (256, "mean", 2, 9, 35), (256, "mean", 2, 19, 32), (256, "mean", 3, 19, 32),
+                                                  (128, "mean", 2, 37, 33), (64, "mean", 2, 75, 32)])
+def test_gate_next_extends_scores_and_keep_list_one_chunk_at_a_time(d_g, agg, planes, B, H):
+    """The trigger's gate step in one launch: from a keep list over the first chunks, kvE_gate_next takes the chunks one
+    by one; scores, carried state, keep list and the compacted summary rows (through attention) must match the oracle
+    exactly as kvE_gate + kvE_compact over the whole range do."""
+    b = _binding()
+    Nc = 21 if B * H < 100 else 7
+    wl = wlm.Workload("next", B=B, H=H, n=32 * Nc + 64 + 5, C=32, W=64, d_g=d_g, agg=agg, d_sum=128 if agg == "mlp" else 0,
+                      key_offset_std=0.5, seed=300 + d_g + planes + B)
+    pb = hz.Problem(wl, keep=0.5)
+    assert pb.Nc == Nc
+    aw = b.AggWeights(pb.mlp) if pb.mlp is not None else None
+    lw = b.LstmWeights(pb.lstm)
+    ref = make_store(wl)
+    load_kv(ref, 0, pb.K, pb.V)
+    ref.set_gate_planes(planes)
+    run_gpu_pipeline(ref, pb, 0, aw, lw)
+
+    st = make_store(wl)
+    load_kv(st, 0, pb.K, pb.V)
+    st.set_gate_planes(planes)
+    with pytest.raises(b.KveError) as e:                  # nothing summarised yet
+        st.gate_next(0, lw, pb.tau)
+    assert e.value.rc == -4
+    st.summarize_chunks(0, 0, pb.Nc, aw)
+    st.gate_next(0, lw, pb.tau)                           # chunk 0: no list yet, the general path
+    assert st.layer_state(0)["n_gated"] == 1 and st.layer_state(0)["n_compacted"] == 1
+    st.gate(0, 1, 4, lw)                                  # the list is stale now ...
+    assert st.layer_state(0)["n_compacted"] <= 1
+    st.gate_next(0, lw, pb.tau)                           # ... so this one re-lists as well
+    assert st.layer_state(0) == dict(n_tokens=wl.n, n_summarised=pb.Nc, n_gated=5, n_compacted=5)
+    for t in range(5, pb.Nc):
+        st.gate_next(0, lw, pb.tau)                       # one launch each
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    assert st.layer_state(0) == dict(n_tokens=wl.n, n_summarised=pb.Nc, n_gated=pb.Nc, n_compacted=pb.Nc)
+    check_gate_and_keep(st, pb)
+    check_attention(st, pb, "summary")
+    # against the range kernels on the same device: another summation order, nothing more
+    assert (st.scores[0, :, :pb.Nc] - ref.scores[0, :, :pb.Nc]).abs().max().item() <= 2e-6
+    assert (st.lstm_h[0] - ref.lstm_h[0]).abs().max().item() <= 2e-6
+    assert torch.equal(st.keep_idx[0], ref.keep_idx[0]) and torch.equal(st.keep_cnt[0], ref.keep_cnt[0])
+    with pytest.raises(b.KveError) as e:                  # every summarised chunk is gated
+        st.gate_next(0, lw, pb.tau)
+    assert e.value.rc == -4
+
+
 def test_layers_are_independent():
     b = _binding()
     wl = wlm.CFG1.small(n=1024, B=2, H=4, n_layers=3)
