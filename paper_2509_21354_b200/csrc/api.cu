@@ -651,7 +651,10 @@ static int decode_step_host(kvE_store* st, int layer, const void* k_new_host, co
     if (rc != KVE_OK) return rc;
   }
   const int g0 = ls.n_gated;
-  if (nc > g0) {
+  if (nc == g0 + 1) {      // the usual trigger: one chunk has left the window
+    rc = kvE_gate_next(st, layer, lw, tau, stream);
+    if (rc != KVE_OK) return rc;
+  } else if (nc > g0) {
     rc = kvE_gate(st, layer, g0, nc, lw, stream);
     if (rc != KVE_OK) return rc;
   }

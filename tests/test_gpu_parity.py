@@ -424,6 +424,39 @@ def test_decode_step_host_matches_stepwise_calls():
     assert torch.equal(out2, out)
 
 
+@pytest.mark.parametrize("agg", ["mean", "mlp"])
+def test_decode_step_host_streams_across_triggers(agg):
+    """The host-buffer step without the from-scratch refresh: tokens arrive one by one, and whenever a chunk has left
+    the window the step summarises it, gates it with the carried state (kvE_gate_next) and extends the keep list.
+    After 2 C + 3 steps - two triggers - everything must match the oracle on the final cache."""
+    b = _binding()
+    C_, W, n0 = 16, 32, 16 * 6 + 32 + 3
+    n1 = n0 + 2 * C_ + 3
+    wl1 = wlm.Workload("hoststream", B=2, H=5, n=n1, C=C_, W=W, d_g=128, agg=agg, d_sum=64 if agg == "mlp" else 0,
+                       key_offset_std=0.5, seed=77)
+    pb = hz.Problem(wl1, keep=0.5)
+    st = make_store(wl1)
+    aw = b.AggWeights(pb.mlp) if pb.mlp is not None else None
+    lw = b.LstmWeights(pb.lstm)
+    load_kv(st, 0, np.ascontiguousarray(pb.K[:, :n0]), np.ascontiguousarray(pb.V[:, :n0]))
+    st.refresh(0, aw, lw, pb.tau)
+    pin = lambda a: b.bits_to_bf16(np.ascontiguousarray(a), "cpu").pin_memory()
+    out = torch.zeros(wl1.S, 128, dtype=torch.bfloat16).pin_memory()
+    q = wlm.gen_q(wl1)
+    hq = pin(q)
+    gated = [st.layer_state(0)["n_gated"]]
+    for pos in range(n0, n1):
+        st.decode_step_host(0, pin(pb.K[:, pos]), pin(pb.V[:, pos]), hq, out, aw, lw, pb.tau, from_scratch=False)
+        gated.append(st.layer_state(0)["n_gated"])
+    assert st.poll_status() == 0
+    assert gated[0] == pb.Nc - 2 and gated[-1] == pb.Nc and sorted(set(gated)) == [pb.Nc - 2, pb.Nc - 1, pb.Nc]
+    assert st.layer_state(0) == dict(n_tokens=n1, n_summarised=pb.Nc, n_gated=pb.Nc, n_compacted=pb.Nc)
+    check_summaries(st, pb)
+    check_gate_and_keep(st, pb)
+    want, _, _, _ = pb.oracle_attn(q, "summary")
+    hz.check_output(b.bf16_to_bits(out), want, "host stream")
+
+
 def test_host_side_errors():
     b = _binding()
     wl = wlm.CFG1.small(n=512)
