@@ -237,6 +237,59 @@ def query_block_leg(wl, hbm, tensor_peak, peak_kind, seed):
     return res
 
 
+def host_free_loop_leg(wl, attend, seed, steady_ms, replays=6):
+    """Sec. 3.3 with the host out of the loop: ONE captured graph = C decode steps (kvE_decode_step) + the trigger in its
+    device-positioned form (kvE_refresh_next: the chunk that has just left the window is summarised, gated and appended
+    to the keep list, its index found on the device).  Every replay moves one layer C tokens ahead, trigger included;
+    the graph is replayed across several triggers without a new capture."""
+    import torch
+    rig = Rig(wl, attend, seed, extra_tokens=(replays + 3) * wl.C)
+    st, S, C_ = rig.st, wl.S, wl.C
+    # start on a chunk boundary of the stale range: C more tokens make exactly one chunk leave the window
+    n_start = wl.W + (rig.Nc + 1) * C_
+    fillk = torch.randn((S, n_start - wl.n, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    st.append(0, fillk, fillk)
+    st.refresh(0, rig.aw, rig.lw, wl.tau)
+    torch.cuda.synchronize()
+    k_in = torch.randn((C_, S, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    q_in = torch.randn((C_, S, 128), generator=rig.gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty_like(q_in)
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(C_):
+                st.decode_step(0, k_in[i], k_in[i], q_in[i], out[i], n_reserve=(replays + 2) * C_)
+            st.refresh_next(0, rig.aw, rig.lw, wl.tau)
+    torch.cuda.current_stream().wait_stream(side)
+    st.adopt_device_state(0)
+    gated0 = st.layer_state(0)["n_gated"]
+    graph.replay()                                         # warm-up: one replay = C tokens + one trigger
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(replays):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    st.adopt_device_state(0)
+    state = st.layer_state(0)
+    assert state["n_gated"] == gated0 + 1 + replays and state["n_tokens"] == n_start + (1 + replays) * C_
+    ms_replay = e0.elapsed_time(e1) / replays
+    st.close()
+    return {"what": f"one CUDA graph of C = {C_} x kvE_decode_step + kvE_refresh_next (trigger positioned on the device), one layer, "
+                    f"replayed {replays} times across as many triggers, no host work besides the replay",
+            "ms_per_replay": ms_replay, "us_per_token_trigger_included": 1e3 * ms_replay / C_,
+            "tokens_per_s": 1e3 * C_ / ms_replay, "steady_us_per_token_without_trigger": 1e3 * steady_ms,
+            "triggers_crossed": replays, "launches_per_replay": C_ + kernels_per_trigger(wl)}
+
+
+def kernels_per_trigger(wl):
+    """launches of the device-positioned trigger: chunk mean (+ MLP) + the gate step"""
+    return 3 if wl.agg == "mlp" else 2
+
+
 def graph_tick_leg(wl, n_layers, seed, replays=20, mem_cap=40e9, fused=True):
     """The decode loop of a whole model between two gate triggers: per token, for each of n_layers layers
     append the new token at the device-held length (kvE_append_next) and run the gated attention; all
@@ -859,6 +912,8 @@ def run_ours(args, rank, world, local_rank):
     per[short]["kernels_us"] = {k: {a: v[a] for a in ("us", "us_l2_flushed", "frac_of_hbm_peak_l2_flushed") if a in v} for k, v in kern.items()}
     if "trigger" in legs:
         res["trigger"] = trigger_leg(wl, args.attend, seed + 5, steady["ms_per_step"])
+        if wl.agg != "token_mlp":
+            res["host_free_loop"] = host_free_loop_leg(wl, args.attend, seed + 6, steady["ms_per_step"])
     rig.st.close()
     del rig, st
     torch.cuda.empty_cache()

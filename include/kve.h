@@ -182,6 +182,23 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end,
  * been summarised.  Timed under KVE_K_GATE_RNN. */
 int kvE_gate_next(kvE_store* st, int layer, const kvE_lstm_weights* w, float tau, void* stream);
 
+/* Sec. 3.3, the trigger with nothing about the position fixed at launch, so that it can sit in a captured CUDA graph
+ * behind the decode steps (kvE_decode_step) and be replayed: every execution looks on the DEVICE for the chunk right
+ * behind the keep list's coverage and, if the stored length says that chunk has left the window, summarises it (Eq. 2),
+ * gates it with the carried (h, c) (Eq. 3) and appends it to the keep list for `tau` (Sec. 3.2), as kvE_summarize_chunks
+ * + kvE_gate_next do; if no chunk is due the launches return at once.  A graph of C decode steps followed by this call
+ * replays for as long as the cache has room, with no host work besides the replay.  Needs, at the call: a keep list under
+ * the same tau that covers every gated chunk (at least one), and nothing summarised beyond it; else KVE_ERR_STATE.
+ * KVE_ERR_GEOMETRY for KVE_AGG_TOKEN_MLP.  The handle's own counters advance as for one execution on the state it
+ * knows; after replays, kvE_adopt_device_state brings them up to date.  Sequences of a layer have one common length. */
+int kvE_refresh_next(kvE_store* st, int layer, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, void* stream);
+
+/* Read the stored length and the keep list's coverage of `layer` back from the device (waits for `stream`) and make them
+ * the handle's: the token count, and - when the keep list covered every gated chunk before - the counts of summarised,
+ * gated and listed chunks.  For use after replaying captured kvE_append_next / kvE_decode_step / kvE_refresh_next
+ * launches, which move the device's counters without the host.  KVE_ERR_STATE if the device holds impossible values. */
+int kvE_adopt_device_state(kvE_store* st, int layer, void* stream);
+
 /* Sec. 3.2 retention rule: keep chunk t iff scores[t] >= tau, over all gated chunks of `layer`;
  * writes keep_idx / keep_cnt.  Attention then treats tokens from (gated chunks) * C on as raw.  Also copies the kept
  * chunks' summary rows into one contiguous run per sequence (workspace), which is what attention reads, and records

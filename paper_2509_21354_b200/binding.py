@@ -22,7 +22,7 @@ STATUS = {0: "KVE_OK", -1: "KVE_ERR_ARG", -2: "KVE_ERR_GEOMETRY", -3: "KVE_ERR_C
           -4: "KVE_ERR_STATE", -5: "KVE_ERR_CUDA", -6: "KVE_ERR_TIMEOUT"}
 
 EXPORTS = ["kvE_workspace_bytes", "kvE_create", "kvE_destroy", "kvE_set_attend", "kvE_set_gate_planes", "kvE_append", "kvE_append_next", "kvE_set_len",
-           "kvE_summarize_chunks", "kvE_gate", "kvE_gate_next", "kvE_refresh", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_step", "kvE_decode_attn_dense", "kvE_decode_attn_block",
+           "kvE_summarize_chunks", "kvE_gate", "kvE_gate_next", "kvE_refresh", "kvE_refresh_next", "kvE_adopt_device_state", "kvE_compact", "kvE_compact_topk", "kvE_decode_attn", "kvE_decode_step", "kvE_decode_attn_dense", "kvE_decode_attn_block",
            "kvE_decode_attn_static", "kvE_reclaim_pages", "kvE_decode_step_host", "kvE_decode_step_host_async", "kvE_poll_status", "kvE_layer_state", "kvE_last_cuda_error",
            "kvE_profile", "kvE_profile_read", "kvE_selftest_timeout"]
 KERNEL_IDS = ["append", "chunk_mean", "chunk_mlp", "gate_proj", "gate_rnn", "compact", "attn", "attn_dense", "attn_block"]
@@ -83,6 +83,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.kvE_summarize_chunks.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_agg_weights), C.c_void_p]
     lib.kvE_gate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(kvE_lstm_weights), C.c_void_p]
     lib.kvE_gate_next.argtypes = [C.c_void_p, C.c_int, C.POINTER(kvE_lstm_weights), C.c_float, C.c_void_p]
+    lib.kvE_refresh_next.argtypes = [C.c_void_p, C.c_int, C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float, C.c_void_p]
+    lib.kvE_adopt_device_state.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.kvE_compact.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_void_p]
     lib.kvE_refresh.argtypes = [C.c_void_p, C.c_int, C.POINTER(kvE_agg_weights), C.POINTER(kvE_lstm_weights), C.c_float, C.c_void_p]
     lib.kvE_compact_topk.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
@@ -265,6 +267,15 @@ class Store:
 
     def gate_next(self, layer, lstm_weights, tau, stream=None):
         kvE_gate_next(self, layer, lstm_weights, tau, stream)
+
+    def refresh_next(self, layer, agg_weights, lstm_weights, tau, stream=None):
+        """the trigger with its position taken from the device at execution time (replayable from a CUDA graph)"""
+        aw = C.byref(agg_weights.c) if agg_weights is not None else None
+        _check("kvE_refresh_next", self.lib.kvE_refresh_next(self.handle, layer, aw, C.byref(lstm_weights.c), C.c_float(tau),
+                                                             _stream(stream)), self.handle)
+
+    def adopt_device_state(self, layer, stream=None):
+        _check("kvE_adopt_device_state", self.lib.kvE_adopt_device_state(self.handle, layer, _stream(stream)), self.handle)
 
     def compact(self, layer, tau, stream=None):
         kvE_compact(self, layer, tau, stream)

@@ -124,7 +124,7 @@ Carve carve(const kvE_config& c) {
   const size_t sum_bytes = (size_t)c.n_layers * S * max_chunks * 128 * 2;
   k.off_kept_k = o;   o = align_up(o + sum_bytes);
   k.off_kept_v = o;   o = align_up(o + sum_bytes);
-  k.off_listed = o;   o = align_up(o + (size_t)c.n_layers * sizeof(int32_t));      // per layer: chunks the keep list covers
+  k.off_listed = o;   o = align_up(o + (size_t)c.n_layers * 2 * sizeof(int32_t));  // per layer: chunks the keep list covers; behind them, per layer: arrival ticket of the gate-step kernel
   k.total = o;
   return k;
 }
@@ -171,6 +171,7 @@ LayerView view(const kvE_store* st, int layer) {
   v.lstm_c = b.lstm_c + L * S * c.d_g;
   v.status = b.status_word;
   v.n_listed = reinterpret_cast<int32_t*>(static_cast<char*>(b.workspace) + st->off_listed) + layer;
+  v.step_ticket = v.n_listed + st->cfg.n_layers;
   v.B = c.B; v.H = c.Hkv; v.S = st->S; v.C = c.C; v.max_chunks = st->max_chunks; v.max_tokens = c.max_tokens;
   return v;
 }
@@ -418,7 +419,7 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
   cudaError_t e = cudaSuccess;
   if (!token_mlp) {
     Prof prof(st, KVE_K_CHUNK_MEAN, s);
-    e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, st->cfg.agg == KVE_AGG_MAX, s);
+    e = launch_chunk_mean(v, chunk_begin, chunk_end, !mlp, st->cfg.agg == KVE_AGG_MAX, s, -1);
   } else {
     Prof prof(st, KVE_K_CHUNK_MLP, s);
     MlpWeights mw;
@@ -434,7 +435,7 @@ int kvE_summarize_chunks(kvE_store* st, int layer, int chunk_begin, int chunk_en
     mw.W1K = static_cast<const uint16_t*>(w->W1K); mw.W2K = static_cast<const uint16_t*>(w->W2K);
     mw.W1V = static_cast<const uint16_t*>(w->W1V); mw.W2V = static_cast<const uint16_t*>(w->W2V);
     mw.b1K = w->b1K; mw.b2K = w->b2K; mw.b1V = w->b1V; mw.b2V = w->b2V;
-    e = launch_chunk_mlp(v, chunk_begin, chunk_end, mw, st->cfg.d_sum, s);
+    e = launch_chunk_mlp(v, chunk_begin, chunk_end, mw, st->cfg.d_sum, s, -1);
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   if (chunk_begin <= ls.n_summarised && chunk_end > ls.n_summarised) ls.n_summarised = chunk_end;
@@ -503,10 +504,70 @@ int kvE_gate_next(kvE_store* st, int layer, const kvE_lstm_weights* w, float tau
     Prof prof(st, KVE_K_GATE_RNN, s);
     e = launch_gate_step(view(st, layer), t, static_cast<const uint16_t*>(w->W_ih), static_cast<const uint16_t*>(w->W_hh),
                          w->b_ih, w->b_hh, w->w_s, w->b_s, tau, st->cfg.d_g, st->gate_planes,
-                         static_cast<uint16_t*>(kr.k), static_cast<uint16_t*>(kr.v), s);
+                         static_cast<uint16_t*>(kr.k), static_cast<uint16_t*>(kr.v), -1, s);
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_gated = ls.n_compacted = t + 1;
+  return KVE_OK;
+}
+
+int kvE_refresh_next(kvE_store* st, int layer, const kvE_agg_weights* aw, const kvE_lstm_weights* lw, float tau, void* stream) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
+  if (!lw || !lw->W_ih || !lw->W_hh || !lw->b_ih || !lw->b_hh || !lw->w_s) return KVE_ERR_ARG;
+  if (st->cfg.agg == KVE_AGG_TOKEN_MLP) return KVE_ERR_GEOMETRY;      // its kernels take their position from the launch only
+  const bool mlp = st->cfg.agg == KVE_AGG_MLP;
+  if (mlp && (!aw || !aw->W1K || !aw->W2K || !aw->W1V || !aw->W2V || !aw->b1K || !aw->b2K || !aw->b1V || !aw->b2V)) return KVE_ERR_ARG;
+  LayerState& ls = st->layers[layer];
+  // a keep list under this tau that covers everything gated, and nothing summarised ahead of it: the device appends to it
+  if (ls.n_compacted < 1 || ls.n_compacted != ls.n_gated || ls.n_summarised != ls.n_gated || ls.by_topk || ls.tau != tau)
+    return KVE_ERR_STATE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const LayerView v = view(st, layer);
+  const int W = st->cfg.W;
+  cudaError_t e;
+  {
+    Prof prof(st, KVE_K_CHUNK_MEAN, s);
+    e = launch_chunk_mean(v, 0, 1, !mlp, st->cfg.agg == KVE_AGG_MAX, s, W);
+  }
+  if (e == cudaSuccess && mlp) {
+    Prof prof(st, KVE_K_CHUNK_MLP, s);
+    MlpWeights mw;
+    mw.W1K = static_cast<const uint16_t*>(aw->W1K); mw.W2K = static_cast<const uint16_t*>(aw->W2K);
+    mw.W1V = static_cast<const uint16_t*>(aw->W1V); mw.W2V = static_cast<const uint16_t*>(aw->W2V);
+    mw.b1K = aw->b1K; mw.b2K = aw->b2K; mw.b1V = aw->b1V; mw.b2V = aw->b2V;
+    e = launch_chunk_mlp(v, 0, 1, mw, st->cfg.d_sum, s, W);
+  }
+  if (e == cudaSuccess) {
+    Prof prof(st, KVE_K_GATE_RNN, s);
+    const KeptRows kr = kept_rows(st, layer);
+    e = launch_gate_step(v, 0, static_cast<const uint16_t*>(lw->W_ih), static_cast<const uint16_t*>(lw->W_hh), lw->b_ih,
+                         lw->b_hh, lw->w_s, lw->b_s, tau, st->cfg.d_g, st->gate_planes, static_cast<uint16_t*>(kr.k),
+                         static_cast<uint16_t*>(kr.v), W, s);
+  }
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  // what this call does when it executes once on the state the host knows of
+  if (stale_chunks(st->cfg, ls.n_tokens) > ls.n_gated && ls.n_gated < st->max_chunks)
+    ls.n_summarised = ls.n_gated = ls.n_compacted = ls.n_gated + 1;
+  return KVE_OK;
+}
+
+int kvE_adopt_device_state(kvE_store* st, int layer, void* stream) {
+  if (bad_layer(st, layer)) return KVE_ERR_ARG;
+  if (wrong_device(st)) return KVE_ERR_STATE;
+  LayerState& ls = st->layers[layer];
+  const LayerView v = view(st, layer);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t len = 0, listed = 0;
+  cudaError_t e = cudaMemcpyAsync(&len, v.seq_len, sizeof(len), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&listed, v.n_listed, sizeof(listed), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(st, e);
+  if (len < 0 || len > st->cfg.max_tokens || listed < 0 || listed > stale_chunks(st->cfg, len)) return KVE_ERR_STATE;
+  ls.n_tokens = len;
+  ls.reserve_upper = 0;
+  if (ls.n_compacted > 0 && ls.n_compacted == ls.n_gated && ls.n_summarised == ls.n_gated && listed > 0)
+    ls.n_summarised = ls.n_gated = ls.n_compacted = listed;      // triggers executed on the device move all three together
   return KVE_OK;
 }
 

@@ -148,6 +148,18 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// A launch whose position comes from the DEVICE (a trigger replayed from a CUDA graph): the chunk to work on is the one
+// right behind the keep list's coverage, and it is due once the stored length says it has left the window.
+struct NextChunk { int t; bool due; };
+__device__ __forceinline__ NextChunk next_chunk(const int32_t* n_listed, const int32_t* seq_len, int C, int window, int max_chunks) {
+  NextChunk nx;
+  nx.t = *n_listed;
+  const int n = seq_len[0];      // lengths are uniform over the sequences of a layer
+  const int stale = n > window ? (n - window) / C : 0;
+  nx.due = nx.t >= 0 && nx.t < stale && nx.t < max_chunks;
+  return nx;
+}
+
 // host side: launch with the programmatic-serialisation attribute
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {

@@ -31,9 +31,11 @@ struct GateStepArgs {
   float b_s, tau;
   const uint16_t *ksum, *vsum;      // bf16 [S][max_chunks][128]
   float *scores, *lstm_h, *lstm_c;
-  int32_t *keep_idx, *keep_cnt, *n_listed;
+  int32_t *keep_idx, *keep_cnt, *n_listed, *ticket;
+  const int32_t* seq_len;
   uint16_t *kept_k, *kept_v;        // bf16 [S][max_chunks][128]
   int S, max_chunks, t;
+  int C, dev_window;      // dev_window >= 0: t comes from the device (the chunk behind the keep list, if it has left the window)
 };
 
 constexpr int STEP_MAX_SEQ = 32;      // sequences per cluster at most (NG = 4)
@@ -61,6 +63,12 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
 
   pdl_launch_dependents();
   pdl_wait();
+  if (a.dev_window >= 0) {
+    // every CTA reads the same count: it only moves when the last cluster of this launch has arrived at the end
+    const NextChunk nx = next_chunk(a.n_listed, a.seq_len, a.C, a.dev_window, a.max_chunks);
+    if (!nx.due) return;
+    a.t = nx.t;
+  }
 
   // ---- B operands into shared memory -----------------------------------------------------------------------------------
   for (int i = tid; i < NSEQ * 32; i += RNN_THREADS) {      // 16-byte pieces of the summary rows: 16 of Kbar, 16 of Vbar
@@ -218,7 +226,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     }
     kept_slot[tid] = slot;
   }
-  if (blockIdx.x == 0 && tid == 0) *a.n_listed = a.t + 1;
+  if (a.dev_window < 0 && blockIdx.x == 0 && tid == 0) *a.n_listed = a.t + 1;
   __syncthreads();
   // a warp copies a kept sequence's summary rows (K and V: 2 x 256 bytes) behind its compacted run
   for (int j = warp; j < NSEQ; j += RNN_WARPS) {
@@ -227,6 +235,18 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     const long long src = ((long long)s * a.max_chunks + a.t) * D, dst = ((long long)s * a.max_chunks + kept_slot[j]) * D;
     if (lane < 16) reinterpret_cast<uint4*>(a.kept_k + dst)[lane] = reinterpret_cast<const uint4*>(a.ksum + src)[lane];
     else reinterpret_cast<uint4*>(a.kept_v + dst)[lane - 16] = reinterpret_cast<const uint4*>(a.vsum + src)[lane - 16];
+  }
+  if (a.dev_window >= 0) {
+    // the coverage count moves when the last cluster is through: until then every CTA of the launch finds the same t
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      const int clusters = gridDim.x / CL;
+      if (atomicAdd(a.ticket, 1) == clusters - 1) {
+        *a.ticket = 0;
+        *a.n_listed = a.t + 1;
+      }
+    }
   }
 }
 
@@ -264,13 +284,14 @@ static cudaError_t launch_step_planes(const GateStepArgs& a, int d_g, cudaStream
 
 cudaError_t launch_gate_step(const LayerView& v, int t, const uint16_t* W_ih, const uint16_t* W_hh, const float* b_ih,
                              const float* b_hh, const float* w_s, float b_s, float tau, int d_g, int planes,
-                             uint16_t* kept_k, uint16_t* kept_v, cudaStream_t st) {
+                             uint16_t* kept_k, uint16_t* kept_v, int dev_window, cudaStream_t st) {
   if (v.S <= 0) return cudaSuccess;
   GateStepArgs a;
   a.W_ih = W_ih; a.W_hh = W_hh; a.b_ih = b_ih; a.b_hh = b_hh; a.w_s = w_s; a.b_s = b_s; a.tau = tau;
   a.ksum = v.ksum_bf16; a.vsum = v.vsum_bf16; a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c;
   a.keep_idx = v.keep_idx; a.keep_cnt = v.keep_cnt; a.n_listed = v.n_listed; a.kept_k = kept_k; a.kept_v = kept_v;
   a.S = v.S; a.max_chunks = v.max_chunks; a.t = t;
+  a.ticket = v.step_ticket; a.seq_len = v.seq_len; a.C = v.C; a.dev_window = dev_window;
   return planes == 3 ? launch_step_planes<3>(a, d_g, st) : launch_step_planes<2>(a, d_g, st);
 }
 

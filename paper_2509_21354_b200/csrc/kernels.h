@@ -45,6 +45,7 @@ struct LayerView {
   float* lstm_c;
   int32_t* status;
   int32_t* n_listed;          // one int: chunks [0, *n_listed) are covered by the keep list (device copy of the handle's count)
+  int32_t* step_ticket;       // one int, zero between launches: arrivals of the gate-step kernel's clusters
   int B, H, S, C, max_chunks, max_tokens;
 };
 
@@ -69,8 +70,11 @@ cudaError_t launch_set_listed(const LayerView& v, int n_listed, cudaStream_t st)
 cudaError_t launch_set_len(const LayerView& v, int n, int n_listed, cudaStream_t st);
 cudaError_t launch_append_next(const LayerView& v, const void* k_new, const void* v_new, int n_new, int32_t* ticket,
                                cudaStream_t st);
-cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st);
-cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st);
+// dev_window < 0: chunks [t0, t1).  dev_window >= 0 (the window size W): ONE chunk per sequence whose index the kernel
+// finds on the device - the chunk behind the keep list's coverage, if the stored length says it has left the window,
+// else the launch does nothing (a trigger that is replayed from a CUDA graph)
+cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st, int dev_window);
+cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st, int dev_window);
 // per-token MLP aggregator: hid = scratch of 2 * S * (t1 - t0) * d_sum floats
 bool token_mlp_supported(int C, int d_sum);
 cudaError_t launch_chunk_token_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, float* hid, cudaStream_t st);
@@ -80,10 +84,11 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
                             int d_g, float* P, bool reset_state, int planes, cudaStream_t st);
 // one LSTM step on chunk t with the carried state, its score, and chunk t appended to the keep list for tau (which must
-// cover chunks [0, t)), its summary rows appended to kkept / vkept, the device's coverage count set to t + 1
+// cover chunks [0, t)), its summary rows appended to kkept / vkept, the device's coverage count set to t + 1.
+// dev_window >= 0: t is found on the device as above (the argument t is ignored), nothing happens if no chunk is due
 cudaError_t launch_gate_step(const LayerView& v, int t, const uint16_t* W_ih, const uint16_t* W_hh, const float* b_ih,
                              const float* b_hh, const float* w_s, float b_s, float tau, int d_g, int planes,
-                             uint16_t* kept_k, uint16_t* kept_v, cudaStream_t st);
+                             uint16_t* kept_k, uint16_t* kept_v, int dev_window, cudaStream_t st);
 // both also leave the kept chunks' summary rows compacted in kkept / vkept [S][max_chunks][128] bf16, which is
 // what attention reads until the next keep list
 cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, void* kkept, void* vkept, cudaStream_t st);

@@ -31,9 +31,14 @@ __device__ __forceinline__ void max_row(float (&acc)[8], const uint4& w) {
 // POOL_MAX: element-wise maximum of the chunk instead of its mean (the "pooling" aggregator of Sec. 3.1)
 template <bool POOL_MAX>
 __global__ void __launch_bounds__(MEAN_WARPS * 32) kve_chunk_mean_kernel(LayerView v, int t0, int n_range,
-                                                                        long long n_units, int final_output) {
+                                                                        long long n_units, int final_output, int dev_window) {
   pdl_launch_dependents();
   pdl_wait();
+  if (dev_window >= 0) {      // one chunk per sequence, found on the device
+    const NextChunk nx = next_chunk(v.n_listed, v.seq_len, v.C, dev_window, v.max_chunks);
+    if (!nx.due) return;
+    t0 = nx.t;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // persistent warps: unit = global warp id, then strides of the whole grid
   for (long long unit = (long long)blockIdx.x * MEAN_WARPS + warp; unit < n_units; unit += (long long)gridDim.x * MEAN_WARPS) {
@@ -101,15 +106,15 @@ static int mean_ctas_per_sm() {
 // That only holds if the CTAs land on an empty GPU: the kernel is therefore launched WITHOUT the programmatic edge the
 // other kernels use.  (Launched early, beside the tail of its predecessor, its CTAs spread unevenly over the SMs
 // and the static striding turns that into a tail: measured +25 % on 4 GB of stale KV.)
-cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st) {
-  const int n_range = t1 - t0;
+cudaError_t launch_chunk_mean(const LayerView& v, int t0, int t1, bool final_output, bool pool_max, cudaStream_t st, int dev_window) {
+  const int n_range = dev_window >= 0 ? 1 : t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
   long long blocks = (n_units + MEAN_WARPS - 1) / MEAN_WARPS;
   const long long wave = (long long)sm_count() * (pool_max ? mean_ctas_per_sm<true>() : mean_ctas_per_sm<false>());
   if (blocks > wave) blocks = wave;
-  if (pool_max) kve_chunk_mean_kernel<true><<<dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st>>>(v, t0, n_range, n_units, 1);
-  else kve_chunk_mean_kernel<false><<<dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st>>>(v, t0, n_range, n_units, final_output ? 1 : 0);
+  if (pool_max) kve_chunk_mean_kernel<true><<<dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st>>>(v, t0, n_range, n_units, 1, dev_window);
+  else kve_chunk_mean_kernel<false><<<dim3((unsigned)blocks), dim3(MEAN_WARPS * 32), 0, st>>>(v, t0, n_range, n_units, final_output ? 1 : 0, dev_window);
   return cudaGetLastError();
 }
 
@@ -128,9 +133,14 @@ __device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8]) {
 }
 
 __global__ void __launch_bounds__(MLP_THREADS) kve_chunk_mlp_kernel(LayerView v, int t0, int n_range, long long n_units,
-                                                                   MlpWeights w, int d_sum) {
+                                                                   MlpWeights w, int d_sum, int dev_window) {
   pdl_launch_dependents();
   pdl_wait();
+  if (dev_window >= 0) {      // one chunk per sequence, found on the device
+    const NextChunk nx = next_chunk(v.n_listed, v.seq_len, v.C, dev_window, v.max_chunks);
+    if (!nx.due) return;
+    t0 = nx.t;
+  }
   extern __shared__ __align__(16) float smem[];
   float* Xs = smem;                    // [MLP_ROWS][128]
   float* Hs = smem + MLP_ROWS * D;     // [MLP_ROWS][d_sum]
@@ -259,7 +269,7 @@ __device__ __forceinline__ void store_split8(const float (&x)[8], unsigned char*
 }
 
 __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerView v, int t0, int n_range, long long n_units,
-                                                                         MlpWeights w, int d_sum) {
+                                                                         MlpWeights w, int d_sum, int dev_window) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* As = smem + MT_SMEM_A;
@@ -318,8 +328,13 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
 
   pdl_wait();      // weights, barriers and tensor memory are set up; the chunk means come from the previous kernel
   uint32_t ph_h = 0, ph_buf[2] = {0, 0};
-  bool failed = false;
-  for (long long tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
+  bool failed = false, due = true;
+  if (dev_window >= 0) {      // one chunk per sequence, found on the device
+    const NextChunk nx = next_chunk(v.n_listed, v.seq_len, v.C, dev_window, v.max_chunks);
+    due = nx.due;
+    t0 = nx.t;
+  }
+  for (long long tile = blockIdx.x; tile < n_tiles && !failed && due; tile += gridDim.x) {
     const long long unit0 = tile * MT_M;
     // ---- chunk means -> three bf16 planes (layer-1 A operand) ------------------------------------------
     {
@@ -472,8 +487,8 @@ __global__ void __launch_bounds__(MT_THREADS, 1) kve_chunk_mlp_tc_kernel(LayerVi
   if (warp == 0) umma::tmem_dealloc(tmem_h, MT_TMEM_COLS);
 }
 
-cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st) {
-  const int n_range = t1 - t0;
+cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeights& w, int d_sum, cudaStream_t st, int dev_window) {
+  const int n_range = dev_window >= 0 ? 1 : t1 - t0;
   const long long n_units = (long long)v.S * n_range;
   if (n_units <= 0) return cudaSuccess;
   if (d_sum % 64 == 0 && d_sum <= MT_MAX_DSUM && n_units + MT_M < (1LL << 31) &&
@@ -487,7 +502,7 @@ cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeight
     const long long half = sm_count() / 2;
     const long long per_side = n_tiles < half ? n_tiles : half;  // one CTA per SM: half of the SMs per side
     dim3 grid((unsigned)per_side, 2);
-    return launch_pdl(kve_chunk_mlp_tc_kernel, grid, dim3(MT_THREADS), MT_SMEM_BYTES, st, v, t0, n_range, n_units, w, d_sum);
+    return launch_pdl(kve_chunk_mlp_tc_kernel, grid, dim3(MT_THREADS), MT_SMEM_BYTES, st, v, t0, n_range, n_units, w, d_sum, dev_window);
   }
   const size_t smem = sizeof(float) * (size_t)MLP_ROWS * (D + d_sum);
   static DeviceFlags opted;
@@ -496,7 +511,7 @@ cudaError_t launch_chunk_mlp(const LayerView& v, int t0, int t1, const MlpWeight
     if (e != cudaSuccess) return e;
   }
   dim3 grid((unsigned)((n_units + MLP_ROWS - 1) / MLP_ROWS), 2);
-  return launch_pdl(kve_chunk_mlp_kernel, grid, dim3(MLP_THREADS), smem, st, v, t0, n_range, n_units, w, d_sum);
+  return launch_pdl(kve_chunk_mlp_kernel, grid, dim3(MLP_THREADS), smem, st, v, t0, n_range, n_units, w, d_sum, dev_window);
 }
 
 }  // namespace kve

@@ -760,6 +760,86 @@ def test_streaming_soak_reuses_reclaimed_pages_over_several_triggers():
     assert n == wl_full.n and nc == pb.Nc and reused == n_triggers * S
 
 
+@pytest.mark.parametrize("agg,d_g,B,H", [("mean", 64, 1, 4), ("mlp", 256, 2, 5), ("max", 128, 3, 3), ("mean", 256, 9, 35)])
+def test_one_graph_runs_decode_steps_and_triggers_without_the_host(agg, d_g, B, H):
+    """Sec. 3.3 with the host out of the loop: ONE captured graph holds C decode steps (kvE_decode_step) followed by the
+    trigger in its device-positioned form (kvE_refresh_next).  Every replay appends C tokens, attends after each, and
+    takes the chunk that has left the window through summary, gate and keep list.  After each replay: scores, keep lists
+    and the carried state against the oracle, attention outputs of the last step too; the handle then adopts the device's
+    counters and a host-issued step continues from there."""
+    b = _binding()
+    C_, W, n_replays = 16, 32, 5
+    n0 = W + 3 * C_                                  # three chunks gated before the graph takes over; (n0 - W) % C == 0
+    wl_full = wlm.Workload("graphtrig", B=B, H=H, n=n0 + n_replays * C_ + 1, C=C_, W=W, d_g=d_g, agg=agg,
+                           d_sum=64 if agg == "mlp" else 0, key_offset_std=0.5, seed=500 + d_g + B)
+    pb = hz.Problem(wl_full)
+    K, V, S = pb.K, pb.V, wl_full.S
+    st = make_store(wl_full)
+    aw = b.AggWeights(pb.mlp) if pb.mlp is not None else None
+    lw = b.LstmWeights(pb.lstm)
+    st.append(0, b.bits_to_bf16(np.ascontiguousarray(K[:, :n0])), b.bits_to_bf16(np.ascontiguousarray(V[:, :n0])))
+    nc = wl_full.n_stale_chunks(n0)
+    assert nc == 3
+    with pytest.raises(b.KveError) as e:             # no keep list yet: nothing for the device to append to
+        st.refresh_next(0, aw, lw, pb.tau)
+    assert e.value.rc == -4
+    st.refresh(0, aw, lw, pb.tau)
+    # per-step inputs of one replay live in [C] slots that the graph's launches read
+    k_in = torch.zeros((C_, S, 128), dtype=torch.bfloat16, device="cuda")
+    v_in, q_in, out = torch.zeros_like(k_in), torch.zeros_like(k_in), torch.zeros_like(k_in)
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(C_):
+                st.decode_step(0, k_in[i], v_in[i], q_in[i], out[i], n_reserve=n_replays * C_)
+            st.refresh_next(0, aw, lw, pb.tau)
+    torch.cuda.current_stream().wait_stream(side)
+    st.adopt_device_state(0)                         # capture advanced the handle's counters, nothing ran
+    assert st.layer_state(0) == dict(n_tokens=n0, n_summarised=3, n_gated=3, n_compacted=3)
+
+    def oracle_out(q, n_now, nc_now):
+        idx, cnt = pb.o64.compact(pb.sc64, nc_now, pb.tau)
+        return pb.o64.attn(q, np.ascontiguousarray(K[:, :n_now]), np.ascontiguousarray(V[:, :n_now]), C_, nc_now, idx, cnt,
+                           pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)[0]
+
+    n = n0
+    for rep in range(n_replays):
+        qs = [wlm.gen_q(wl_full, 0, 100 * rep + i) for i in range(C_)]
+        k_in.copy_(b.bits_to_bf16(np.ascontiguousarray(K[:, n:n + C_].transpose(1, 0, 2))))
+        v_in.copy_(b.bits_to_bf16(np.ascontiguousarray(V[:, n:n + C_].transpose(1, 0, 2))))
+        q_in.copy_(b.bits_to_bf16(np.stack(qs)))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        # step i of the replay saw n + i + 1 tokens and the keep list over nc chunks; the trigger came after the last step
+        for i in (0, C_ // 2, C_ - 1):
+            hz.check_output(b.bf16_to_bits(out[i]), oracle_out(qs[i], n + i + 1, nc), f"replay {rep}, step {i}")
+        n += C_
+        nc += 1
+        assert int(st.seq_len[0, 0]) == n
+        sc = st.scores[0, :, :nc].cpu().numpy()
+        assert np.abs(sc - pb.sc64[:, :nc]).max() <= 2e-4
+        idx, cnt = pb.o64.compact(pb.sc64, nc, pb.tau)
+        assert np.array_equal(st.keep_cnt[0].cpu().numpy(), cnt) and np.array_equal(st.keep_idx[0, :, :nc].cpu().numpy(), idx[:, :nc])
+    # the host takes over again: its counters come from the device, the next step is issued directly
+    st.adopt_device_state(0)
+    assert st.layer_state(0) == dict(n_tokens=n, n_summarised=nc, n_gated=nc, n_compacted=nc)
+    q = wlm.gen_q(wl_full, 0, 9999)
+    got = torch.zeros((S, 128), dtype=torch.bfloat16, device="cuda")
+    st.decode_step(0, b.bits_to_bf16(np.ascontiguousarray(K[:, n])), b.bits_to_bf16(np.ascontiguousarray(V[:, n])), b.bits_to_bf16(q), got)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    hz.check_output(b.bf16_to_bits(got), oracle_out(q, n + 1, nc), "host step after the graph")
+    assert n + 1 == wl_full.n and nc == pb.Nc
+    # a trigger that is not due does nothing
+    before = (st.scores[0].clone(), st.keep_cnt[0].clone(), st.lstm_h[0].clone())
+    st.refresh_next(0, aw, lw, pb.tau)
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0 and st.layer_state(0)["n_gated"] == nc
+    assert all(torch.equal(a_, b_) for a_, b_ in zip(before, (st.scores[0], st.keep_cnt[0], st.lstm_h[0])))
+
+
 # ---- Sec. 3.3 memory reduction: pages of gated chunks handed back ---------------------------------
 @pytest.mark.parametrize("attend,mode", [("summary", "discarded"), ("summary", "gated"), ("raw", "discarded")])
 def test_reclaim_pages_matches_oracle_and_leaves_attention_unchanged(attend, mode):
