@@ -127,10 +127,13 @@ __device__ __forceinline__ void prefetch_sequence_metadata(const AttnArgs& a, in
 }
 
 // rows the kept chunks of sequence s contribute
+__device__ __forceinline__ int lead_rows_from(const AttnArgs& a, const AttnGeo& g, int keep_cnt) {
+  if (a.mode == ATTN_DENSE || g.n_chunks <= 0) return 0;
+  return min(max(keep_cnt, 0), g.n_chunks) * g.per;
+}
 __device__ __forceinline__ int lead_rows_of(const AttnArgs& a, const AttnGeo& g, int s) {
   if (a.mode == ATTN_DENSE || g.n_chunks <= 0) return 0;
-  const int M = min(max(a.v.keep_cnt[s], 0), g.n_chunks);
-  return M * g.per;
+  return lead_rows_from(a, g, a.v.keep_cnt[s]);
 }
 
 #define KVE_TR_ROUND(OFF, CNT)                                                        \
@@ -171,6 +174,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
     const uint32_t I = (uint32_t)v.S * (uint32_t)a.k, P = min(gridDim.x, I);
     if (blockIdx.x < P) prefetch_sequence_metadata(a, (int)(piece_begin(blockIdx.x, I, P) / (uint32_t)a.k), lane);
     if (lane == 31) prefetch_l2(v.seq_len);
+    if (lane == 30) prefetch_l2(v.n_listed);
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < AT_STAGES; ++i) {
@@ -187,27 +191,35 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
   pdl_wait();      // lengths, keep lists, summaries and the new token come from earlier kernels
   KVE_STAMP(threadIdx.x == 0, 1);
 
+  // this CTA's parts follow from the launch arguments; the producer asks for its first sequence's keep count at once,
+  // together with the length and the coverage below: three look-ups in flight instead of one after the other
+  const uint32_t c = blockIdx.x, uk = (uint32_t)a.k;
+  const uint32_t n_items = (uint32_t)v.S * uk, n_pieces = min(gridDim.x, n_items);
+  const uint32_t i0 = piece_begin(c, n_items, n_pieces), i1 = piece_begin(c + 1, n_items, n_pieces);
+  int keep_cnt_first = 0;
+  if (warp == AT_PRODUCER && i0 < i1 && a.mode != ATTN_DENSE) keep_cnt_first = v.keep_cnt[i0 / uk];
+
   // ---- geometry (every thread) ---------------------------------------------------------------------------
   AttnGeo g;
   {
     int n = v.seq_len[0];
+    // chunks the keep list covers: the device's own count, so that a launch replayed from a CUDA graph follows the
+    // gate triggers that happened since it was captured (the launch argument is only the host's view at capture time).
+    // Requested together with the length: nothing that could alias stands between the two loads.
+    const int listed = (a.mode == ATTN_DENSE) ? 0 : *v.n_listed;
     n = min(max(n, 0), v.max_tokens);
     g.appending = a.k_new != nullptr && n < v.max_tokens;
     if (a.k_new != nullptr && !g.appending && blockIdx.x == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);   // cache full
     if (g.appending) n += 1;
     g.n = n;
-    // chunks the keep list covers: the device's own count, so that a launch replayed from a CUDA graph follows the
-    // gate triggers that happened since it was captured (the launch argument is only the host's view at capture time)
-    g.n_chunks = (a.mode == ATTN_DENSE) ? 0 : min(max(*v.n_listed, 0), v.max_chunks);
+    g.n_chunks = min(max(listed, 0), v.max_chunks);
     g.raw0 = g.n_chunks * v.C;
     g.n_tail = max(0, n - g.raw0);
     g.TT = (g.n_tail + AT_TILE - 1) / AT_TILE;
     g.per = (a.mode == ATTN_RAW) ? v.C : 1;
-    g.I = (uint32_t)v.S * (uint32_t)a.k;
-    g.P = min(gridDim.x, g.I);
+    g.I = n_items;
+    g.P = n_pieces;
   }
-  const uint32_t c = blockIdx.x, uk = (uint32_t)a.k;
-  const uint32_t i0 = piece_begin(c, g.I, g.P), i1 = piece_begin(c + 1, g.I, g.P);      // this CTA's parts
 
   if (warp == AT_PRODUCER) {
     // ================= producer warp =================
@@ -218,7 +230,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
     bool fresh = true;                      // the next tile is the first one of sequence s in this CTA
     auto enter_sequence = [&]() {
       if (s < s_last) prefetch_sequence_metadata(a, s + 1, lane);      // the next one's look-ups will hit L2
-      lt_rows = lead_rows_of(a, g, s);
+      lt_rows = (s == s_first) ? lead_rows_from(a, g, keep_cnt_first) : lead_rows_of(a, g, s);
       tiles = g.TT + (lt_rows + AT_TILE - 1) / AT_TILE;
       // part p of the sequence's tiles: [p tiles / k, (p + 1) tiles / k); p <= 32 and tiles < 2^20, so 32 bits do
       const uint32_t p_lo = (s == s_first) ? i0 - (uint32_t)s * uk : 0u;
