@@ -91,15 +91,8 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
   const LayerView& v = a.v;
   const int s = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  pdl_wait();      // lengths, keep lists, summaries and the queries come from earlier kernels
 
-  const BlockGeom gm = block_geometry(a, s, split);
-  // the sequence has outgrown what this launch was sized for (a replayed launch): rows would be dropped
-  if (gm.outgrown && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
-  if (split >= gm.n_splits) return;
-  const int n_tiles = gm.n_tiles;
-
-  // ---- set-up: barriers, tensor memory, Q as the A operand, P cleared --------------------------------
+  // ---- set-up that needs nothing from earlier kernels: barriers, tensor memory, P cleared -----------------
   if (threadIdx.x == 0) {
     for (int i = 0; i < TC_STAGES; ++i) {
       mbar_init(&full[i], 1);
@@ -115,13 +108,6 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
     mbar_fence_init();
   }
   if (warp == 1) umma::tmem_alloc(tmem_slot, TC_TMEM_COLS);
-  for (int idx = threadIdx.x; idx < 128 * 16; idx += TC_THREADS) {
-    const int arow = idx >> 4, p16 = idx & 15;      // row of the A operand = tensor-memory lane of S
-    const int qrow = arow % (128 / REP);             // the query block repeats REP times down the lanes
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (qrow < a.R) val = *reinterpret_cast<const uint4*>(a.q + q_row_offset(a, s, qrow) + p16 * 8);
-    *reinterpret_cast<uint4*>(Qs + (p16 >> 3) * (128 * 128) + arow * 128 + (((p16 & 7) ^ (arow & 7)) << 4)) = val;
-  }
   for (int idx = threadIdx.x; idx < 2 * TC_PLANES * TC_P_BYTES / 16; idx += TC_THREADS)
     *reinterpret_cast<uint4*>(Ps + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
   umma::fence_smem_to_async();
@@ -130,6 +116,30 @@ kve_decode_attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmK, const _
   umma::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_o = tmem_base, tmem_s = tmem_base + 256;
+
+  pdl_wait();      // lengths, keep lists, summaries and the queries come from earlier kernels
+
+  const BlockGeom gm = block_geometry(a, s, split);
+  // the sequence has outgrown what this launch was sized for (a replayed launch): rows would be dropped
+  if (gm.outgrown && split == 0 && threadIdx.x == 0) set_status(v.status, ERR_CAPACITY);
+  if (split >= gm.n_splits) {      // nothing for this CTA
+    if (warp == 1) umma::tmem_dealloc(tmem_base, TC_TMEM_COLS);
+    return;
+  }
+  const int n_tiles = gm.n_tiles;
+
+  // ---- Q as the A operand: staged by everybody but the producer warp, which is already fetching tiles ----------------
+  if (warp != 0) {
+    for (int idx = threadIdx.x - 32; idx < 128 * 16; idx += TC_THREADS - 32) {
+      const int arow = idx >> 4, p16 = idx & 15;      // row of the A operand = tensor-memory lane of S
+      const int qrow = arow % (128 / REP);             // the query block repeats REP times down the lanes
+      uint4 val = make_uint4(0u, 0u, 0u, 0u);
+      if (qrow < a.R) val = *reinterpret_cast<const uint4*>(a.q + q_row_offset(a, s, qrow) + p16 * 8);
+      *reinterpret_cast<uint4*>(Qs + (p16 >> 3) * (128 * 128) + arow * 128 + (((p16 & 7) ^ (arow & 7)) << 4)) = val;
+    }
+    umma::fence_smem_to_async();
+    asm volatile("bar.sync 2, %0;" ::"n"(TC_THREADS - 32) : "memory");
+  }
 
   if (warp == 0) {
     // ================= producer warp =================
