@@ -51,9 +51,19 @@ __device__ unsigned long long g_rnn_cycles[8];
     }                                                                                        \
   } while (0)
 #define KVE_RNN_MARK_BEGIN() long long mark_ = clock64()
+__device__ unsigned long long g_rnn_once[8];
+#define KVE_RNN_ONCE(slot)                                                                   \
+  do {                                                                                       \
+    if (blockIdx.x == 0 && threadIdx.x == 0) {                                               \
+      unsigned long long t_;                                                                 \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                 \
+      g_rnn_once[slot] = t_;                                                                 \
+    }                                                                                        \
+  } while (0)
 #else
 #define KVE_RNN_MARK(slot) do { } while (0)
 #define KVE_RNN_MARK_BEGIN() do { } while (0)
+#define KVE_RNN_ONCE(slot) do { } while (0)
 #endif
 
 // NG independent groups of 8 sequences per cluster.  A group is one pipeline (own h buffers, barriers,
@@ -87,6 +97,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   const int seq0 = cid * NS * NG;        // group gi owns sequences seq0 + 8 gi .. + 7
 
   pdl_launch_dependents();
+  KVE_RNN_ONCE(0);
   if (tid == 0) {
     for (int i = 0; i < 2 * NG; ++i) mbar_init(&hbar[i], 1 + RNN_WARPS);
     mbar_fence_init();
@@ -106,7 +117,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     }
   }
 
+  KVE_RNN_ONCE(1);
   pdl_wait();      // W_hh is in registers; the carried state and P come from earlier kernels
+  KVE_RNN_ONCE(2);
   // ---- initial state: every CTA needs the full h of its sequences as planes in buffer 0 of each group -------------
   for (int i = tid; i < NG * NS * (DG / 2); i += RNN_THREADS) {
     const int js = i / (DG / 2), k2 = i % (DG / 2);      // js: sequence of the cluster, 0 .. 8 NG - 1
@@ -148,7 +161,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   const uint32_t peer_bar = map_to_rank(smem_u32(&hbar[0]), lane < CL ? lane : 0);
 
   // barriers initialised and buffer 0 filled in every CTA before anyone sends
+  KVE_RNN_ONCE(3);
   cluster_sync_all();
+  KVE_RNN_ONCE(4);
 
   bool alive = true;
   KVE_RNN_MARK_BEGIN();
@@ -301,6 +316,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
     }
   }
 
+  KVE_RNN_ONCE(5);
   // ---- carried state out ---------------------------------------------------------------------------
 #pragma unroll
   for (int gi = 0; gi < NG; ++gi)
@@ -317,6 +333,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
       }
   // nobody leaves while a peer may still be sending into its shared memory
   cluster_sync_all();
+  KVE_RNN_ONCE(6);
 }
 
 // ---- score head: s_t = sigmoid(w_s . h_t + b_s), one warp per (sequence, chunk) --------------------------
@@ -388,6 +405,9 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
 
 #ifdef KVE_RNN_STAMPS
 // instrumented build only: read and clear the cycle sums
+extern "C" int kve_rnn_once_read(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, kve::g_rnn_once, sizeof(kve::g_rnn_once));
+}
 extern "C" int kve_rnn_cycles_read(unsigned long long* host) {
   cudaError_t e = cudaMemcpyFromSymbol(host, kve::g_rnn_cycles, sizeof(kve::g_rnn_cycles));
   void* p = nullptr;

@@ -50,6 +50,8 @@ def main(cfgs):
             us_kernel = rig.st.profile_read()["gate_rnn"]
             rig.st.profile(False)
             lib.kve_rnn_cycles_read(buf.ctypes.data)
+            once = np.zeros(8, np.uint64)
+            lib.kve_rnn_once_read(once.ctypes.data)
             rounds = int(buf[5])
             groups = max(1, rounds // rig.Nc)
             print(f"== {rig.wl.name}: {rig.Nc} steps, {rig.wl.S} sequences, {groups} group(s) of 8 sequences per cluster, "
@@ -59,6 +61,9 @@ def main(cfgs):
                 cyc = float(buf[i]) / max(rounds, 1)
                 tot += cyc
                 print(f"  {nm:52s} {cyc:8.0f} cycles  {cyc / mhz:6.3f} us   (per step and group)")
+            o = (once.astype(np.int64) - int(once[0])) / 1e3
+            print(f"  CTA 0, us after its entry: W_hh fragments loaded {o[1]:.2f}, predecessor waited for {o[2]:.2f}, initial state and "
+                  f"first P {o[3]:.2f}, cluster barrier {o[4]:.2f}, step loop done {o[5]:.2f}, state out + cluster barrier {o[6]:.2f}")
             loop_us = tot * rounds / mhz
             print(f"  {'sum':52s} {tot:8.0f} cycles  {tot / mhz:6.3f} us   x {groups} group(s) = {tot * groups / mhz:.3f} us per step; "
                   f"step loop {loop_us:.1f} us of the {us_kernel:.1f} us (rest: W_hh fragments into registers, first P, "
