@@ -104,16 +104,50 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   }
 
   // ---- W_hh rows of this CTA as A fragments, resident in registers --------------------------------
+  // Register j of the fragment of k tile kt holds the two bf16 at k = 16 kt + 8 (j >> 1) + 2 tig of row (j & 1): word
+  // 8 kt + 4 (j >> 1) + tig of the row.  The four lanes of a group (equal g) fetch 16 consecutive words of the row with one
+  // 16-byte load each (lane tig: words 4 tig ..) and turn the 4 x 4 block among themselves with shuffles, so that lane tig
+  // ends up with words tig, 4 + tig, 8 + tig, 12 + tig: a quarter of the load instructions of word-by-word fetches (5 -> 2 us).
+  // With two groups per cluster the kernel sits at the register limit and that order of definition cost 10 % in the step
+  // loop (measured), so there the words are fetched one by one.
   uint32_t A[2 * MP][KT][4];
+  static_assert(KT % 2 == 0, "k tiles are fetched in pairs");
+  if constexpr (NG == 1) {
 #pragma unroll
-  for (int mt = 0; mt < 2 * MP; ++mt) {
-    const int ug = (int)rank * HU + warp * UW + (mt >> 1) * 8 + g;
+    for (int mt = 0; mt < 2 * MP; ++mt) {
+      const int ug = (int)rank * HU + warp * UW + (mt >> 1) * 8 + g;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int gate = (mt & 1) * 2 + (j & 1);
-      const uint32_t* wrow = reinterpret_cast<const uint32_t*>(a.W_hh + ((long long)gate * DG + ug) * DG);
+      for (int rs = 0; rs < 2; ++rs) {
+        const int gate = (mt & 1) * 2 + rs;
+        const uint4* wrow = reinterpret_cast<const uint4*>(a.W_hh + ((long long)gate * DG + ug) * DG) + tig;
 #pragma unroll
-      for (int kt = 0; kt < KT; ++kt) A[mt][kt][j] = __ldg(wrow + kt * 8 + (j >> 1) * 4 + tig);
+        for (int kp = 0; kp < KT / 2; ++kp) {
+          const uint4 w = __ldg(wrow + kp * 4);
+          const bool hi = (tig & 2) != 0, lo = (tig & 1) != 0;
+          // lanes t and t ^ 2 swap halves: afterwards y0, y1 come from lane (t & 1), y2, y3 from lane (t & 1) + 2, words 2 hi, 2 hi + 1
+          const uint32_t r0 = __shfl_xor_sync(0xffffffffu, hi ? w.x : w.z, 2), r1 = __shfl_xor_sync(0xffffffffu, hi ? w.y : w.w, 2);
+          const uint32_t y0 = hi ? r0 : w.x, y1 = hi ? r1 : w.y, y2 = hi ? w.z : r0, y3 = hi ? w.w : r1;
+          // lanes t and t ^ 1 swap the word the other one wants
+          const uint32_t u0 = __shfl_xor_sync(0xffffffffu, lo ? y0 : y1, 1), u1 = __shfl_xor_sync(0xffffffffu, lo ? y2 : y3, 1);
+          const uint32_t k0 = lo ? y1 : y0, k1 = lo ? y3 : y2;
+          A[mt][2 * kp][rs] = lo ? u0 : k0;              // word tig of the lane group's 16
+          A[mt][2 * kp][rs + 2] = lo ? k0 : u0;          // word 4 + tig
+          A[mt][2 * kp + 1][rs] = lo ? u1 : k1;          // word 8 + tig
+          A[mt][2 * kp + 1][rs + 2] = lo ? k1 : u1;      // word 12 + tig
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int mt = 0; mt < 2 * MP; ++mt) {
+      const int ug = (int)rank * HU + warp * UW + (mt >> 1) * 8 + g;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gate = (mt & 1) * 2 + (j & 1);
+        const uint32_t* wrow = reinterpret_cast<const uint32_t*>(a.W_hh + ((long long)gate * DG + ug) * DG);
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) A[mt][kt][j] = __ldg(wrow + kt * 8 + (j >> 1) * 4 + tig);
+      }
     }
   }
 
