@@ -840,6 +840,63 @@ def test_one_graph_runs_decode_steps_and_triggers_without_the_host(agg, d_g, B, 
     assert all(torch.equal(a_, b_) for a_, b_ in zip(before, (st.scores[0], st.keep_cnt[0], st.lstm_h[0])))
 
 
+def test_one_graph_serves_two_layers_with_their_own_triggers():
+    """Two layers with different data and weights in ONE graph: per token the decode step of layer 0, then of layer 1; after
+    C tokens the device-positioned trigger of each.  The layers' counters, tickets and keep lists must not mix."""
+    b = _binding()
+    C_, W, n_replays, n_layers = 16, 32, 3, 2
+    n0 = W + 2 * C_
+    wl = wlm.Workload("graph2", B=2, H=4, n=n0 + n_replays * C_, C=C_, W=W, d_g=256, agg="mean", key_offset_std=0.5, seed=640,
+                      n_layers=n_layers)
+    pbs = [hz.Problem(wl.small(seed=wl.seed + L), layer=L) for L in range(n_layers)]
+    S = wl.S
+    st = make_store(wl, n_layers=n_layers)
+    lws = [b.LstmWeights(pb.lstm) for pb in pbs]
+    for L, pb in enumerate(pbs):
+        st.append(L, b.bits_to_bf16(np.ascontiguousarray(pb.K[:, :n0])), b.bits_to_bf16(np.ascontiguousarray(pb.V[:, :n0])))
+        st.refresh(L, None, lws[L], pb.tau)
+    k_in = torch.zeros((n_layers, C_, S, 128), dtype=torch.bfloat16, device="cuda")
+    v_in, q_in, out = torch.zeros_like(k_in), torch.zeros_like(k_in), torch.zeros_like(k_in)
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(C_):
+                for L in range(n_layers):
+                    st.decode_step(L, k_in[L, i], v_in[L, i], q_in[L, i], out[L, i], n_reserve=n_replays * C_)
+            for L in range(n_layers):
+                st.refresh_next(L, None, lws[L], pbs[L].tau)
+    torch.cuda.current_stream().wait_stream(side)
+    for L in range(n_layers):
+        st.adopt_device_state(L)
+    n, nc = n0, 2
+    for rep in range(n_replays):
+        qs = [[wlm.gen_q(wl, L, 100 * rep + i) for i in range(C_)] for L in range(n_layers)]
+        for L, pb in enumerate(pbs):
+            k_in[L].copy_(b.bits_to_bf16(np.ascontiguousarray(pb.K[:, n:n + C_].transpose(1, 0, 2))))
+            v_in[L].copy_(b.bits_to_bf16(np.ascontiguousarray(pb.V[:, n:n + C_].transpose(1, 0, 2))))
+            q_in[L].copy_(b.bits_to_bf16(np.stack(qs[L])))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        for L, pb in enumerate(pbs):
+            idx, cnt = pb.o64.compact(pb.sc64, nc, pb.tau)
+            i = C_ - 1
+            want = pb.o64.attn(qs[L][i], np.ascontiguousarray(pb.K[:, :n + i + 1]), np.ascontiguousarray(pb.V[:, :n + i + 1]), C_, nc,
+                               idx, cnt, pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)[0]
+            hz.check_output(b.bf16_to_bits(out[L, i]), want, f"layer {L}, replay {rep}")
+            idx1, cnt1 = pb.o64.compact(pb.sc64, nc + 1, pb.tau)
+            assert np.abs(st.scores[L, :, :nc + 1].cpu().numpy() - pb.sc64[:, :nc + 1]).max() <= 2e-4
+            assert np.array_equal(st.keep_cnt[L].cpu().numpy(), cnt1)
+            assert np.array_equal(st.keep_idx[L, :, :nc + 1].cpu().numpy(), idx1[:, :nc + 1])
+        n += C_
+        nc += 1
+    for L in range(n_layers):
+        st.adopt_device_state(L)
+        assert st.layer_state(L) == dict(n_tokens=n, n_summarised=nc, n_gated=nc, n_compacted=nc)
+    assert n == wl.n and nc == pbs[0].Nc
+
+
 # ---- Sec. 3.3 memory reduction: pages of gated chunks handed back ---------------------------------
 @pytest.mark.parametrize("attend,mode", [("summary", "discarded"), ("summary", "gated"), ("raw", "discarded")])
 def test_reclaim_pages_matches_oracle_and_leaves_attention_unchanged(attend, mode):
