@@ -370,30 +370,63 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
   KVE_RNN_ONCE(6);
 }
 
-// ---- score head: s_t = sigmoid(w_s . h_t + b_s), one warp per (sequence, chunk) --------------------------
+// ---- score head: s_t = sigmoid(w_s . h_t + b_s), one warp per SCORE_ROWS (sequence, chunk) rows --------------------
 // h_t sits in columns [0, d_g) of row (s, t) of P.  Lane l sums elements l*4 .. l*4+3 (+128 per round) in
-// order, then a butterfly over the lanes: the same order for every launch.
-__global__ void __launch_bounds__(256) kve_gate_score_kernel(const float* __restrict__ P, const float* __restrict__ w_s,
-                                                             float b_s, float* __restrict__ scores, long long n_rows,
-                                                             int n_range, int t0, int max_chunks, int d_g) {
+// order, then a butterfly over the lanes: the same order for every launch.  A warp has the loads of all its rows in
+// flight before it starts to add (the rows are 1 KB pieces 4 KB apart: latency, not bytes, is what a lone row waits for).
+constexpr int SCORE_ROWS = 4;
+constexpr int SCORE_WARPS = 8;
+
+template <int DG>
+__global__ void __launch_bounds__(SCORE_WARPS * 32) kve_gate_score_kernel(const float* __restrict__ P, const float* __restrict__ w_s,
+                                                                         float b_s, float* __restrict__ scores, long long n_rows,
+                                                                         int n_range, int t0, int max_chunks) {
+  constexpr int ROUNDS = (DG / 4 + 31) / 32;      // 16-byte pieces per lane and row
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31;
-  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (row >= n_rows) return;
-  const float4* h = reinterpret_cast<const float4*>(P + row * 4 * d_g);
+  const long long row0 = ((long long)blockIdx.x * SCORE_WARPS + (threadIdx.x >> 5)) * SCORE_ROWS;
+  if (row0 >= n_rows) return;
   const float4* w = reinterpret_cast<const float4*>(w_s);
-  float acc = 0.f;
-  for (int i = lane; i < d_g / 4; i += 32) {
-    const float4 hv = __ldcs(h + i), wv = __ldg(w + i);
-    acc = fmaf(hv.x, wv.x, acc); acc = fmaf(hv.y, wv.y, acc);
-    acc = fmaf(hv.z, wv.z, acc); acc = fmaf(hv.w, wv.w, acc);
+  float4 hv[SCORE_ROWS][ROUNDS];
+#pragma unroll
+  for (int r = 0; r < SCORE_ROWS; ++r) {
+    const float4* h = reinterpret_cast<const float4*>(P + (row0 + r) * 4 * DG);
+#pragma unroll
+    for (int i = 0; i < ROUNDS; ++i)
+      hv[r][i] = (row0 + r < n_rows && lane + 32 * i < DG / 4) ? __ldcs(h + lane + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  acc = warp_sum(acc);
-  if (lane == 0) {
-    const int s = (int)(row / n_range);
-    const int t = t0 + (int)(row - (long long)s * n_range);
-    scores[(long long)s * max_chunks + t] = 1.f / (1.f + expf(-(acc + b_s)));
+  float4 wv[ROUNDS];
+#pragma unroll
+  for (int i = 0; i < ROUNDS; ++i) wv[i] = (lane + 32 * i < DG / 4) ? __ldg(w + lane + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+  for (int r = 0; r < SCORE_ROWS; ++r) {
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < ROUNDS; ++i) {
+      if (lane + 32 * i < DG / 4) {
+        acc = fmaf(hv[r][i].x, wv[i].x, acc); acc = fmaf(hv[r][i].y, wv[i].y, acc);
+        acc = fmaf(hv[r][i].z, wv[i].z, acc); acc = fmaf(hv[r][i].w, wv[i].w, acc);
+      }
+    }
+    acc = warp_sum(acc);
+    const long long row = row0 + r;
+    if (lane == 0 && row < n_rows) {
+      const int s = (int)(row / n_range);
+      const int t = t0 + (int)(row - (long long)s * n_range);
+      scores[(long long)s * max_chunks + t] = 1.f / (1.f + expf(-(acc + b_s)));
+    }
+  }
+}
+
+static cudaError_t launch_score(const float* P, const float* w_s, float b_s, float* scores, long long n_rows, int n_range, int t0,
+                                int max_chunks, int d_g, cudaStream_t st) {
+  const dim3 grid((unsigned)((n_rows + SCORE_WARPS * SCORE_ROWS - 1) / (SCORE_WARPS * SCORE_ROWS))), block(SCORE_WARPS * 32);
+  switch (d_g) {
+    case 256: return launch_pdl(kve_gate_score_kernel<256>, grid, block, 0, st, P, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
+    case 128: return launch_pdl(kve_gate_score_kernel<128>, grid, block, 0, st, P, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
+    case 64:  return launch_pdl(kve_gate_score_kernel<64>, grid, block, 0, st, P, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
+    default:  return cudaErrorInvalidValue;
   }
 }
 
@@ -431,8 +464,7 @@ cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* 
   const cudaError_t e = planes == 3 ? launch_rnn_planes<3>(a, d_g, st) : launch_rnn_planes<2>(a, d_g, st);
   if (e != cudaSuccess) return e;
   const long long n_rows = (long long)v.S * a.n_range;
-  return launch_pdl(kve_gate_score_kernel, dim3((unsigned)((n_rows + 7) / 8)), dim3(256), 0, st, (const float*)P, w_s, b_s, v.scores, n_rows,
-                    a.n_range, t0, v.max_chunks, d_g);
+  return launch_score(P, w_s, b_s, v.scores, n_rows, a.n_range, t0, v.max_chunks, d_g, st);
 }
 
 }  // namespace kve
