@@ -108,7 +108,7 @@ typedef struct {
 
 typedef struct kvE_store kvE_store;
 
-/* Bytes of workspace the handle needs: the gate projection buffer, the split-K partial records and tickets of
+/* Bytes of workspace the handle needs: the gate projection buffer and the h_t rows of one kvE_gate call, the split-K partial records and tickets of
  * the attention kernels (those of kvE_decode_attn_block only when cfg.max_query_tokens > 0), staging rows of the
  * host-buffer step, scratch of kvE_reclaim_pages.  0 if the geometry is not supported. */
 size_t kvE_workspace_bytes(const kvE_config* cfg);

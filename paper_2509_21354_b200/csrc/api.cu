@@ -28,7 +28,7 @@ struct kvE_store {
   int device = -1;       // the device that was current at kvE_create: owner of every buffer; calls check it
   int S, max_chunks;
   // workspace carve-up (byte offsets)
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, off_listed, ws_needed;
+  size_t off_P, off_H, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, off_listed, ws_needed;
   int attn_grid_max;     // most CTAs an attention launch uses (two per SM of the handle's device): sizes the partial records
   // block-of-queries attention: tensor maps over the page pools and the summary store (encoded at
   // create when cfg.max_query_tokens > 0), rows per page box, split cap the workspace was sized for
@@ -87,7 +87,7 @@ int check_config(const kvE_config* c) {
 }
 
 struct Carve {
-  size_t off_P, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, off_listed, total;
+  size_t off_P, off_H, off_partials, off_counters, off_stage, off_reclaim, off_ticket, off_block, off_kept_k, off_kept_v, off_listed, total;
 };
 // most CTAs of one attention launch: two resident per SM (148 SMs assumed where no device can be asked)
 int attn_grid_cap() {
@@ -109,6 +109,8 @@ Carve carve(const kvE_config& c) {
   size_t p_floats = S * max_chunks * 4 * (size_t)c.d_g;
   if (c.agg == KVE_AGG_TOKEN_MLP && 2 * S * max_chunks * (size_t)c.d_sum > p_floats) p_floats = 2 * S * max_chunks * (size_t)c.d_sum;
   k.off_P = o;        o = align_up(o + p_floats * sizeof(float));
+  // h_t of every gated (sequence, chunk) of one kvE_gate call, [S max_chunks][d_g]: what the score head reads
+  k.off_H = o;        o = align_up(o + S * max_chunks * (size_t)c.d_g * sizeof(float));
   // attention partial records: the one of (sequence s, CTA c) at s + c, at most ATTN_GRID_LIMIT CTAs
   k.off_partials = o; o = align_up(o + (S + ATTN_GRID_LIMIT) * ATTN_PARTIAL_FLOATS * sizeof(float));
   k.off_counters = o; o = align_up(o + S * sizeof(int32_t));
@@ -295,7 +297,7 @@ int kvE_create(const kvE_config* cfg, const kvE_buffers* buf, kvE_store** out) {
   }
   st->S = cfg->B * cfg->Hkv;
   st->max_chunks = (cfg->max_tokens + cfg->C - 1) / cfg->C;
-  st->off_P = k.off_P; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
+  st->off_P = k.off_P; st->off_H = k.off_H; st->off_partials = k.off_partials; st->off_counters = k.off_counters;
   st->off_stage = k.off_stage; st->off_reclaim = k.off_reclaim; st->off_ticket = k.off_ticket; st->off_block = k.off_block;
   st->off_kept_k = k.off_kept_k; st->off_kept_v = k.off_kept_v; st->off_listed = k.off_listed; st->ws_needed = k.total;
   st->attn_grid_max = attn_grid_cap();
@@ -465,7 +467,8 @@ int kvE_gate(kvE_store* st, int layer, int chunk_begin, int chunk_end, const kvE
   if (e == cudaSuccess) {
     Prof prof(st, KVE_K_GATE_RNN, s);
     e = launch_gate_rnn(v, chunk_begin, chunk_end, static_cast<const uint16_t*>(w->W_hh), w->w_s, w->b_s, st->cfg.d_g,
-                        P, chunk_begin == 0, st->gate_planes, s);
+                        P, reinterpret_cast<float*>(static_cast<char*>(st->buf.workspace) + st->off_H), chunk_begin == 0,
+                        st->gate_planes, s);
   }
   if (e != cudaSuccess) return cuda_fail(st, e);
   ls.n_gated = chunk_end;

@@ -1,5 +1,6 @@
 // Gate input projection (Eq. 3, the W_ih x_t term for all chunks at once):
 //   P[s, t, :] = W_ih [Kbar_t ; Vbar_t] + b_ih + b_hh      a GEMM [S * n_range, 256] x [256, 4 d_g]
+// stored with the four gates of a hidden unit side by side (column 4 u + gate)
 // bf16 operands (the rounded summaries and bf16 weights, so every product is exact), fp32
 // accumulation in tensor memory (tcgen05.mma, M = 128, N = 256 per instruction), bias fused in the
 // epilogue.
@@ -55,10 +56,16 @@ __global__ void __launch_bounds__(PJ_THREADS, 1) kve_gate_proj_kernel(LayerView 
   // ---- one-time set-up: weight slice, bias, tensor memory, barrier ---------------------------------
   for (int i = tid; i < PJ_N * 32; i += PJ_THREADS) {
     const int r = i >> 5, p = i & 31;                 // p: 16-byte piece of the 512-byte weight row
+    // column c of P holds gate c & 3 of hidden unit c >> 2 (the four pre-activations of a unit side by side: the
+    // recurrence fetches them with one 16-byte load): row (c & 3) d_g + (c >> 2) of W_ih
+    const int c = col0 + r, d_g = n_cols >> 2;
     cp_async16(Bs + (p >> 3) * PJ_B_KB_BYTES + umma::piece_offset(r, p & 7),
-               reinterpret_cast<const uint4*>(W_ih + (long long)(col0 + r) * PJ_K) + p, true);
+               reinterpret_cast<const uint4*>(W_ih + (long long)((c & 3) * d_g + (c >> 2)) * PJ_K) + p, true);
   }
-  for (int i = tid; i < PJ_N; i += PJ_THREADS) bias[i] = b_ih[col0 + i] + b_hh[col0 + i];
+  for (int i = tid; i < PJ_N; i += PJ_THREADS) {
+    const int c = col0 + i, row = (c & 3) * (n_cols >> 2) + (c >> 2);
+    bias[i] = b_ih[row] + b_hh[row];
+  }
   if (warp == 0) umma::tmem_alloc(tmem_slot, 2 * PJ_N);      // two accumulators: MMAs of tile i+1 overlap the epilogue of tile i
   if (tid == 0) {
     mbar_init(bar, 1);

@@ -25,10 +25,11 @@
 //    receiving CTA, so a step costs one one-way transfer and no
 //    cluster-wide barrier.  A CTA can only be sent step t+1 data after it has itself sent step t
 //    data, i.e. after all its warps have finished reading the buffer that is being overwritten.
-//  * The score head is not part of the chain: h_t is stored into the (already consumed) gate-0
-//    slot of row (s, t) of P, and a second, fully parallel kernel computes
-//    s_t = sigmoid(w_s . h_t + b_s) for all (s, t) afterwards, with a fixed summation order.
-//  * P_{t+1} is fetched into registers while step t computes.
+//  * The score head is not part of the chain: h_t is stored as row (s, t) of a buffer of its own, and a
+//    second, fully parallel kernel computes s_t = sigmoid(w_s . h_t + b_s) for all (s, t) afterwards, with
+//    a fixed summation order.
+//  * P_{t+1} is fetched into registers while step t computes: the projection kernel stores the four
+//    pre-activations of a hidden unit side by side, so a thread takes them with one 16-byte load.
 // Every mbarrier wait is bounded (one second); on give-up the status word gets KVE_ERR_TIMEOUT and
 // the CTA stops sending, which lets its peers run into their own limits and leave as well.
 #include "gate_rnn.cuh"
@@ -185,9 +186,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
         const bool live = !a.reset && s < a.S;
         c[gi][p][e] = live ? a.lstm_c[(long long)s * DG + ug] : 0.f;
         hlast[gi][p][e] = live ? a.lstm_h[(long long)s * DG + ug] : 0.f;
-        const float* prow = a.P + ((long long)s * a.n_range) * n_cols + ug;
-#pragma unroll
-        for (int gate = 0; gate < 4; ++gate) pin[gi][p][gate][e] = (s < a.S) ? __ldcs(prow + gate * DG) : 0.f;
+        // the four pre-activations of a unit lie side by side in P: one 16-byte load
+        const float4 pv = (s < a.S) ? __ldcs(reinterpret_cast<const float4*>(a.P + ((long long)s * a.n_range) * n_cols) + ug)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+        pin[gi][p][0][e] = pv.x; pin[gi][p][1][e] = pv.y; pin[gi][p][2][e] = pv.z; pin[gi][p][3][e] = pv.w;
       }
 
   // lane r < CL feeds peer r: that CTA's h buffers and barriers, as addresses in the cluster window
@@ -268,13 +270,11 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           const int s = seq_g + tig * 2 + e;
           const int ug = (int)rank * HU + warp * UW + p * 8 + g;
           const bool live = s < a.S && send_h;
-          const float* prow = a.P + ((long long)s * a.n_range + step + 1) * n_cols + ug;
-#pragma unroll
-          for (int gate = 0; gate < 4; ++gate) pnext[p][gate][e] = live ? __ldcs(prow + gate * DG) : 0.f;
-          if (s < a.S && step + 2 < a.n_range) {
-#pragma unroll
-            for (int gate = 0; gate < 4; ++gate) asm volatile("prefetch.global.L2 [%0];" ::"l"(prow + n_cols + gate * DG));
-          }
+          const float4* prow = reinterpret_cast<const float4*>(a.P + ((long long)s * a.n_range + step + 1) * n_cols) + ug;
+          const float4 pv = live ? __ldcs(prow) : make_float4(0.f, 0.f, 0.f, 0.f);
+          pnext[p][0][e] = pv.x; pnext[p][1][e] = pv.y; pnext[p][2][e] = pv.z; pnext[p][3][e] = pv.w;
+          // the 8 lanes of a group cover one 128-byte line of the row after it: one of them asks L2 for it
+          if (s < a.S && step + 2 < a.n_range && g == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(prow + n_cols / 4));
         }
 
       KVE_RNN_MARK(2);
@@ -303,9 +303,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
           const float hv = og * fast_tanh(cn);
           hlast[gi][p][e] = hv;
           {
-            // P_t of this (unit, sequence) is consumed: its gate-0 slot carries h_t to the score kernel
+            // h_t for the score kernel
             const int sq = seq_g + tig * 2 + e;
-            if (sq < a.S) a.P[((long long)sq * a.n_range + step) * n_cols + (int)rank * HU + warp * UW + p * 8 + g] = hv;
+            if (sq < a.S) a.H[((long long)sq * a.n_range + step) * DG + (int)rank * HU + warp * UW + p * 8 + g] = hv;
           }
           if (send_h) {
             uint32_t pl3[3];
@@ -371,14 +371,14 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(RNN_THREADS, 1) kve
 }
 
 // ---- score head: s_t = sigmoid(w_s . h_t + b_s), one warp per SCORE_ROWS (sequence, chunk) rows --------------------
-// h_t sits in columns [0, d_g) of row (s, t) of P.  Lane l sums elements l*4 .. l*4+3 (+128 per round) in
+// h_t is row (s, t) of H.  Lane l sums elements l*4 .. l*4+3 (+128 per round) in
 // order, then a butterfly over the lanes: the same order for every launch.  A warp has the loads of all its rows in
-// flight before it starts to add (the rows are 1 KB pieces 4 KB apart: latency, not bytes, is what a lone row waits for).
+// flight before it starts to add.
 constexpr int SCORE_ROWS = 4;
 constexpr int SCORE_WARPS = 8;
 
 template <int DG>
-__global__ void __launch_bounds__(SCORE_WARPS * 32) kve_gate_score_kernel(const float* __restrict__ P, const float* __restrict__ w_s,
+__global__ void __launch_bounds__(SCORE_WARPS * 32) kve_gate_score_kernel(const float* __restrict__ H, const float* __restrict__ w_s,
                                                                          float b_s, float* __restrict__ scores, long long n_rows,
                                                                          int n_range, int t0, int max_chunks) {
   constexpr int ROUNDS = (DG / 4 + 31) / 32;      // 16-byte pieces per lane and row
@@ -391,7 +391,7 @@ __global__ void __launch_bounds__(SCORE_WARPS * 32) kve_gate_score_kernel(const 
   float4 hv[SCORE_ROWS][ROUNDS];
 #pragma unroll
   for (int r = 0; r < SCORE_ROWS; ++r) {
-    const float4* h = reinterpret_cast<const float4*>(P + (row0 + r) * 4 * DG);
+    const float4* h = reinterpret_cast<const float4*>(H + (row0 + r) * DG);
 #pragma unroll
     for (int i = 0; i < ROUNDS; ++i)
       hv[r][i] = (row0 + r < n_rows && lane + 32 * i < DG / 4) ? __ldcs(h + lane + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -419,13 +419,13 @@ __global__ void __launch_bounds__(SCORE_WARPS * 32) kve_gate_score_kernel(const 
   }
 }
 
-static cudaError_t launch_score(const float* P, const float* w_s, float b_s, float* scores, long long n_rows, int n_range, int t0,
+static cudaError_t launch_score(const float* H, const float* w_s, float b_s, float* scores, long long n_rows, int n_range, int t0,
                                 int max_chunks, int d_g, cudaStream_t st) {
   const dim3 grid((unsigned)((n_rows + SCORE_WARPS * SCORE_ROWS - 1) / (SCORE_WARPS * SCORE_ROWS))), block(SCORE_WARPS * 32);
   switch (d_g) {
-    case 256: return launch_pdl(kve_gate_score_kernel<256>, grid, block, 0, st, P, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
-    case 128: return launch_pdl(kve_gate_score_kernel<128>, grid, block, 0, st, P, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
-    case 64:  return launch_pdl(kve_gate_score_kernel<64>, grid, block, 0, st, P, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
+    case 256: return launch_pdl(kve_gate_score_kernel<256>, grid, block, 0, st, H, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
+    case 128: return launch_pdl(kve_gate_score_kernel<128>, grid, block, 0, st, H, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
+    case 64:  return launch_pdl(kve_gate_score_kernel<64>, grid, block, 0, st, H, w_s, b_s, scores, n_rows, n_range, t0, max_chunks);
     default:  return cudaErrorInvalidValue;
   }
 }
@@ -455,16 +455,16 @@ static cudaError_t launch_rnn_planes(const RnnArgs& a, int d_g, cudaStream_t st)
 }
 
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
-                            int d_g, float* P, bool reset_state, int planes, cudaStream_t st) {
+                            int d_g, const float* P, float* H, bool reset_state, int planes, cudaStream_t st) {
   if (t1 <= t0 || v.S <= 0) return cudaSuccess;
   RnnArgs a;
-  a.P = P; a.W_hh = W_hh; a.w_s = w_s; a.b_s = b_s;
+  a.P = P; a.H = H; a.W_hh = W_hh; a.w_s = w_s; a.b_s = b_s;
   a.scores = v.scores; a.lstm_h = v.lstm_h; a.lstm_c = v.lstm_c; a.status = v.status;
   a.S = v.S; a.max_chunks = v.max_chunks; a.t0 = t0; a.n_range = t1 - t0; a.reset = reset_state ? 1 : 0;
   const cudaError_t e = planes == 3 ? launch_rnn_planes<3>(a, d_g, st) : launch_rnn_planes<2>(a, d_g, st);
   if (e != cudaSuccess) return e;
   const long long n_rows = (long long)v.S * a.n_range;
-  return launch_score(P, w_s, b_s, v.scores, n_rows, a.n_range, t0, v.max_chunks, d_g, st);
+  return launch_score(H, w_s, b_s, v.scores, n_rows, a.n_range, t0, v.max_chunks, d_g, st);
 }
 
 }  // namespace kve

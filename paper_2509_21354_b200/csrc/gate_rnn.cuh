@@ -11,7 +11,8 @@ constexpr int RNN_WARPS = 8;
 constexpr int RNN_THREADS = RNN_WARPS * 32;
 
 struct RnnArgs {
-  float* P;                // [S * n_range][4 d_g]; columns [0, d_g) of row (s, t) receive h_t once P_t is consumed
+  const float* P;          // [S * n_range][4 d_g], column 4 u + gate: the pre-activations W_ih x + b of unit u
+  float* H;                // [S * n_range][d_g]: h_t for the score kernel
   const uint16_t* W_hh;    // bf16 [4 d_g][d_g]
   const float* w_s;        // [d_g] (score kernel)
   float b_s;

@@ -82,7 +82,7 @@ cudaError_t launch_gate_proj(const LayerView& v, int t0, int t1, const uint16_t*
                              const float* b_hh, int d_g, float* P, cudaStream_t st);
 // planes: bf16 planes of the fp32 state h that enter the recurrent product (2, or 3 = exact products)
 cudaError_t launch_gate_rnn(const LayerView& v, int t0, int t1, const uint16_t* W_hh, const float* w_s, float b_s,
-                            int d_g, float* P, bool reset_state, int planes, cudaStream_t st);
+                            int d_g, const float* P, float* H, bool reset_state, int planes, cudaStream_t st);
 // one LSTM step on chunk t with the carried state, its score, and chunk t appended to the keep list for tau (which must
 // cover chunks [0, t)), its summary rows appended to kkept / vkept, the device's coverage count set to t + 1.
 // dev_window >= 0: t is found on the device as above (the argument t is ignored), nothing happens if no chunk is due
