@@ -215,7 +215,7 @@ int kvE_refresh(kvE_store* st, int layer, const kvE_agg_weights* aw, const kvE_l
 /* The gating-strategy variant the paper names for its ablations (Sec. 5): keep the k highest-scoring gated
  * chunks of every sequence instead of thresholding.  Equal scores: the older chunk ranks first, so the
  * list is unique.  Writes keep_idx / keep_cnt like kvE_compact (ascending ids; k <= 0 keeps nothing,
- * k >= gated chunks keeps all).  At most 2048 gated chunks, else KVE_ERR_GEOMETRY.  After it,
+ * k >= gated chunks keeps all).  Work grows with the square of the gated chunks per sequence.  After it,
  * kvE_reclaim_pages(KVE_RECLAIM_DISCARDED) returns KVE_ERR_STATE (there is no threshold to judge by). */
 int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream);
 

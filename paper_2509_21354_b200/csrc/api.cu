@@ -587,7 +587,6 @@ int kvE_compact_topk(kvE_store* st, int layer, int k, void* stream) {
   if (bad_layer(st, layer)) return KVE_ERR_ARG;
   if (wrong_device(st)) return KVE_ERR_STATE;
   LayerState& ls = st->layers[layer];
-  if (ls.n_gated > 2048) return KVE_ERR_GEOMETRY;      // the kernel stages one sequence's scores per warp
   Prof prof(st, KVE_K_COMPACT, static_cast<cudaStream_t>(stream));
   const KeptRows kr = kept_rows(st, layer);
   cudaError_t e = launch_compact_topk(view(st, layer), ls.n_gated, k, kr.k, kr.v, static_cast<cudaStream_t>(stream));

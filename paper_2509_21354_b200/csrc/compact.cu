@@ -84,22 +84,28 @@ cudaError_t launch_compact(const LayerView& v, int n_chunks, float tau, void* kk
 // ---- kvE_compact_topk kernel: keep the k highest-scoring chunks of every sequence --------------------------
 // One warp per sequence.  Chunk t is kept iff fewer than k chunks rank before it; u ranks before t when
 // s_u > s_t, or s_u == s_t and u < t (the older chunk first), so the result is unique.  Each lane counts
-// the chunks ranking before its own by walking the sequence's scores in shared memory; the kept ids are
-// then written in ascending order with the same ballot + popcount as the threshold rule.
-constexpr int TOPK_MAX_CHUNKS = 2048;      // scores of one sequence staged per warp
+// the chunks ranking before its own by walking the sequence's scores - in shared memory while a sequence's scores
+// fit there (STAGED), straight from global memory beyond that; the kept ids are then written in ascending order
+// with the same ballot + popcount as the threshold rule.
+constexpr int TOPK_STAGED_CHUNKS = 2048;      // scores of one sequence staged per warp up to here
 
+template <bool STAGED>
 __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_topk_kernel(LayerView v, int n_chunks, int k) {
-  extern __shared__ float topk_scores[];   // [COMPACT_WARPS][n_chunks]
+  extern __shared__ float topk_scores[];   // STAGED: [COMPACT_WARPS][n_chunks]
   pdl_launch_dependents();
   pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int s = blockIdx.x * COMPACT_WARPS + warp;
   if (s >= v.S) return;
   const float* sc = v.scores + (long long)s * v.max_chunks;
-  float* mine = topk_scores + warp * n_chunks;
+  const float* mine = sc;
   int32_t* idx = v.keep_idx + (long long)s * v.max_chunks;
-  for (int t = lane; t < n_chunks; t += 32) mine[t] = sc[t];
-  __syncwarp();
+  if (STAGED) {
+    float* stage = topk_scores + warp * n_chunks;
+    for (int t = lane; t < n_chunks; t += 32) stage[t] = sc[t];
+    __syncwarp();
+    mine = stage;
+  }
   int base = 0;
   for (int t0 = 0; t0 < n_chunks; t0 += 32) {
     const int t = t0 + lane;
@@ -123,10 +129,16 @@ __global__ void __launch_bounds__(COMPACT_WARPS * 32) kve_compact_topk_kernel(La
 }
 
 cudaError_t launch_compact_topk(const LayerView& v, int n_chunks, int k, void* kkept, void* vkept, cudaStream_t st) {
-  if (n_chunks > TOPK_MAX_CHUNKS) return cudaErrorInvalidValue;
-  const size_t smem = sizeof(float) * (size_t)COMPACT_WARPS * (n_chunks > 0 ? n_chunks : 1);
-  cudaError_t e = launch_pdl(kve_compact_topk_kernel, dim3((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), dim3(COMPACT_WARPS * 32), smem, st,
-                             v, n_chunks, k);
+  const dim3 grid((v.S + COMPACT_WARPS - 1) / COMPACT_WARPS), block(COMPACT_WARPS * 32);
+  cudaError_t e;
+  if (n_chunks <= TOPK_STAGED_CHUNKS) {
+    const size_t smem = sizeof(float) * (size_t)COMPACT_WARPS * (n_chunks > 0 ? n_chunks : 1);
+    static DeviceFlags opted;
+    e = smem_opt_in(opted, kve_compact_topk_kernel<true>, (int)(sizeof(float) * COMPACT_WARPS * TOPK_STAGED_CHUNKS));
+    if (e == cudaSuccess) e = launch_pdl(kve_compact_topk_kernel<true>, grid, block, smem, st, v, n_chunks, k);
+  } else {
+    e = launch_pdl(kve_compact_topk_kernel<false>, grid, block, 0, st, v, n_chunks, k);
+  }
   return e == cudaSuccess ? launch_keep_gather(v, n_chunks, kkept, vkept, st) : e;
 }
 

@@ -161,8 +161,8 @@ def test_gate_sizes_and_chunk_sizes(d_g, C):
 
 @pytest.mark.parametrize("d_g,B,H", [(64, 37, 33), (256, 9, 35)])
 def test_two_sequence_groups_per_cluster(d_g, B, H):
-    # more sequences than one group of 8 per cluster places in one wave: every cluster walks two groups, with
-    # the rounds of the two software-pipelined; S is ragged against 16 (a cluster's last group is partly or wholly empty)
+    # more sequences than one group of 8 per cluster places in one wave: every cluster walks two groups;
+    # S is ragged against 16 (a cluster's last group is partly or wholly empty)
     wl = wlm.Workload("groups", B=B, H=H, n=9 * 16 + 40, C=16, W=32, d_g=d_g, agg="mean", key_offset_std=0.5, seed=d_g + B)
     assert wl.S > 8 * (148 if d_g == 64 else 37)
     st, pb, _, lstm_w = full_check(wl, "summary")
@@ -955,6 +955,37 @@ def test_reclaim_pages_host_errors_and_overflow():
     _, cnt = st.reclaim_pages(0, 0, 0, "discarded")             # empty range
     torch.cuda.synchronize()
     assert int(cnt.item()) == 0 and st.poll_status() == 0
+
+
+def test_compact_topk_beyond_the_staged_range():
+    """More gated chunks per sequence than the top-k kernel stages in shared memory (2048): the ranking then walks the
+    scores in global memory.  Chunks of one token keep the case small; the list must equal the oracle's ranking of the
+    same fp32 scores bit for bit, and attention over it the oracle's."""
+    b = _binding()
+    wl = wlm.Workload("topk_long", B=1, H=3, n=2300 + 40, C=1, W=40, d_g=64, agg="identity", seed=17, tau=0.0)
+    pb = hz.Problem(wl, keep=None, tau=0.0, margin_eps=0.0)
+    assert pb.Nc == 2300
+    st = make_store(wl)
+    load_kv(st, 0, pb.K, pb.V)
+    lw = b.LstmWeights(pb.lstm)
+    st.summarize_chunks(0, 0, pb.Nc)
+    st.gate(0, 0, pb.Nc, lw)
+    sc_gpu = st.scores[0].cpu().numpy()
+    for k in (1, 700, 2299):
+        st.compact_topk(0, k)
+        torch.cuda.synchronize()
+        assert st.poll_status() == 0
+        want_idx, want_cnt = pb.o32.compact_topk(sc_gpu.astype(np.float32), pb.Nc, k)
+        assert np.array_equal(st.keep_cnt[0].cpu().numpy(), want_cnt)
+        assert np.array_equal(st.keep_idx[0].cpu().numpy(), want_idx)
+    st.compact_topk(0, 700)
+    q = wlm.gen_q(wl, 0, 1)
+    out = st.decode_attn(0, b.bits_to_bf16(q))
+    torch.cuda.synchronize()
+    assert st.poll_status() == 0
+    idx, cnt = st.keep_idx[0].cpu().numpy(), st.keep_cnt[0].cpu().numpy()
+    want = pb.o64.attn(q, pb.K, pb.V, wl.C, pb.Nc, idx, cnt, pb.sm64["ksum_b16"], pb.sm64["vsum_b16"], hz.ATT["summary"], hz.SCALE)[0]
+    hz.check_output(b.bf16_to_bits(out), want, "attn after a long top-k")
 
 
 # ---- gating variant: top-k retention ---------------------------------------------------------------
