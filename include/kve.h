@@ -92,14 +92,15 @@ typedef struct {
 
 /* Aggregator MLP_K / MLP_V of Eq. 2 (KVE_AGG_MLP: y = W2 gelu(W1 m + b1) + b2, m the chunk mean; KVE_AGG_TOKEN_MLP:
  * the same MLP applied to every token of the chunk, the outputs averaged).
- * DEVICE pointers; W1 [d_sum][d], W2 [d][d_sum] bf16; b1 [d_sum], b2 [d] fp32. */
+ * DEVICE pointers; W1 [d_sum][d], W2 [d][d_sum] bf16; b1 [d_sum], b2 [d] fp32; matrices on 16-byte boundaries. */
 typedef struct {
   const void *W1K, *W2K, *W1V, *W2V;
   const float *b1K, *b2K, *b1V, *b2V;
 } kvE_agg_weights;
 
 /* LSTM gate of Eq. 3.  DEVICE pointers; W_ih [4 d_g][2 d], W_hh [4 d_g][d_g] bf16, gate rows in the
- * order i, f, g, o; b_ih, b_hh [4 d_g], w_s [d_g] fp32; b_s by value. */
+ * order i, f, g, o; b_ih, b_hh [4 d_g], w_s [d_g] fp32; b_s by value.  Matrices and w_s start on 16-byte boundaries
+ * (the kernels fetch them 16 bytes at a time). */
 typedef struct {
   const void *W_ih, *W_hh;
   const float *b_ih, *b_hh, *w_s;
