@@ -494,13 +494,17 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
         float* mine = a.partials + (long long)(s + c) * ATTN_PARTIAL_FLOATS;
         *reinterpret_cast<float4*>(mine + lane * 4) = make_float4(accC[0], accC[1], accC[2], accC[3]);
         if (lane == 0) { mine[128] = mC; mine[129] = lC; }
-        __threadfence();
+        // The ticket is an acquire-release atomic at device scope: taken by lane 0 after the warp has synchronised, it
+        // publishes the whole warp's record (release is cumulative over what the barrier ordered before it) and, for the
+        // last arriver, makes the other CTAs' records visible to the warp once it has synchronised again - one round
+        // trip to L2 instead of fence, atomic, fence.
         __syncwarp();
         int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(a.counters + s, 1);
+        if (lane == 0)
+          asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(ticket) : "l"(a.counters + s) : "memory");
         ticket = __shfl_sync(0xffffffffu, ticket, 0);
         if (ticket != n_parts - 1) continue;       // somebody else finishes later and merges
-        __threadfence();
+        __syncwarp();
         // records of sequence s: CTAs c0 .. c1, at s + c0 .. s + c1; lanes fetch the (m, l) pairs side by side
         const float* base = a.partials + (long long)(s + c0) * ATTN_PARTIAL_FLOATS;
         mC = -INFINITY;
@@ -537,8 +541,9 @@ __global__ void __launch_bounds__(AT_THREADS, 2) kve_decode_attn_kernel(AttnArgs
       __syncwarp();
       int last = 0;
       if (lane == 0) {
-        __threadfence();
-        last = atomicAdd(a.ticket, 1) == (int)gridDim.x - 1;
+        int arrived;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(arrived) : "l"(a.ticket) : "memory");
+        last = arrived == (int)gridDim.x - 1;
       }
       last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
